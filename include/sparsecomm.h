@@ -1,0 +1,122 @@
+/*
+ * sparsecomm.h -- C ABI of the sparsified-SGD gradient compressor for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-step hot path of "Sparsified SGD with
+ * error-feedback" (Algorithm 1 of "Sparse Communication for Training Deep
+ * Networks"): for every worker w
+ *     p   = g + e            accumulate the residual   (Algorithm 1, accumulate line; gamma folded into g)
+ *     q^w = C(p)             keep k coordinates        (Methodology: Top-k, Random-k, Block-random-k)
+ *     e'  = p - q^w          kept coordinates become 0 (Methodology prose on error feedback)
+ * and, after the exchange,
+ *     q   = (sum_w q^w) / W  dense average             (Algorithm 1, aggregate line; abstract: "average")
+ *
+ * Conventions
+ *  - All data pointers are DEVICE pointers owned by the caller unless a name
+ *    starts with h_ (then it is a HOST pointer).  The library never frees them.
+ *  - fp32 IEEE-754 round-to-nearest, denormals kept; coordinates are uint32.
+ *  - Every call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL
+ *    is the legacy default stream) and returns a status code, never throws.
+ *    Argument errors are detected on the host before any launch and leave every
+ *    buffer untouched.  Problems seen on the device (a bounded wait that ran out,
+ *    a coordinate outside its range) set a sticky status word read by
+ *    sc_sync_status().
+ *  - A context owns scratch memory and is bound to the device that was current
+ *    in sc_create().  Use one context per stream; calls on one context must not
+ *    overlap on the GPU.
+ *  - grad/residual/out must not alias; base pointers must be 16-byte aligned.
+ *  - Messages: coordinates ascending and distinct, vals[j] = p[idx[j]].  With a
+ *    segment table (layer-wise scope, Methodology "scope of sparsification")
+ *    segment s owns message slots [K_s, K_s + k_s), K_s = sum of earlier k, and
+ *    its coordinates are global (segment offset added).  Segment s of a call
+ *    draws its coordinates from the seed mix64(seed, s).
+ */
+#ifndef SPARSECOMM_H
+#define SPARSECOMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sc_ctx sc_ctx;
+
+/* Compressor C(.) -- Methodology, "compressor or sparsification scheme". */
+enum { SC_TOPK = 0,       /* k largest |p|, ties to the lowest coordinate            */
+       SC_RANDK = 1,      /* k distinct coordinates from a seeded bijection of [0,n)  */
+       SC_RANDBLOCK = 2   /* one seeded start a in [0,n-k], coordinates a..a+k-1      */ };
+
+enum { SC_OK = 0,
+       SC_ERR_INVALID = -1,      /* null pointer, misaligned base pointer, unknown scheme, bad table */
+       SC_ERR_RANGE = -2,        /* k > n, n >= 2^32, W < 1, sizes beyond what the context was made for */
+       SC_ERR_WORKSPACE = -3,    /* scratch allocation failed */
+       SC_ERR_CUDA = -4,         /* a CUDA runtime call failed */
+       SC_ERR_TIMEOUT = -5,      /* a bounded device-side wait gave up (reported by sc_sync_status) */
+       SC_ERR_UNSUPPORTED = -6,
+       SC_ERR_DEVICE_CHECK = -7  /* a device-side range check failed (e.g. unsorted message) */ };
+
+/* One tensor of the gradient: elements [offset, offset+n) keep k coordinates. */
+typedef struct { uint64_t offset, n, k; } sc_segment;
+
+/* Allocates the context and all scratch for problems up to max_n elements per
+ * worker, max_W workers and max_segments segments (cudaMalloc; synchronous). */
+int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments);
+void sc_destroy(sc_ctx* ctx);
+const char* sc_strerror(int code);
+
+/* Synchronises `stream`, then returns (and clears) the sticky device status. */
+int sc_sync_status(sc_ctx* ctx, void* stream);
+
+/* Bytes of device scratch the context holds; kernels launched so far. */
+size_t sc_scratch_bytes(const sc_ctx* ctx);
+uint64_t sc_launch_count(const sc_ctx* ctx);
+
+/* Algorithm 1, accumulate + compress + residual lines, one worker, global scope.
+ * grad[n] read-only; residual[n] in/out (reads e, writes e'); out_vals[k],
+ * out_idx[k] written.  k == 0 is allowed (residual <- g + e). */
+int sc_compress(sc_ctx* ctx, int scheme, const float* grad, float* residual, size_t n, size_t k,
+                uint64_t seed, float* out_vals, uint32_t* out_idx, void* stream);
+
+/* Same for W workers and a segment table in one call.  grads and residuals are
+ * W rows of n elements (row w at +w*n); segs is a HOST array of nseg segments,
+ * ascending and non-overlapping inside [0,n); elements outside every segment
+ * are left alone.  h_seeds is a HOST array of W seeds; equal seeds give equal
+ * coordinates (the paper's "same seed state").  Messages: row w of out_vals /
+ * out_idx has K = sum k_s entries (row w at +w*K). */
+int sc_compress_batch(sc_ctx* ctx, int scheme, int W, const float* grads, float* residuals, size_t n,
+                      const sc_segment* segs, int nseg, const uint64_t* h_seeds,
+                      float* out_vals, uint32_t* out_idx, void* stream);
+
+/* Algorithm 1, aggregate line, read as an average: out[i] = (sum over w = 0..W-1,
+ * in that order, starting from +0.0, of q^w[i]) / (float)W; untouched i give
+ * +0.0.  vals and idx are W rows of k entries, each row ascending and distinct,
+ * all coordinates < n.  out[n] is fully overwritten. */
+int sc_aggregate(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                 float* out, void* stream);
+
+/* The same when all workers kept the same coordinates (the paper's allReduce
+ * case): vals is W rows of k, idx is ONE row of k. */
+int sc_aggregate_shared(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                        float* out, void* stream);
+
+/* One whole step: sc_compress_batch followed by the aggregate over the W
+ * messages it produced (the shared-coordinate form when all seeds are equal and
+ * the scheme is not top-k).  out[n] receives the dense average. */
+int sc_step(sc_ctx* ctx, int scheme, int W, const float* grads, float* residuals, size_t n,
+            const sc_segment* segs, int nseg, const uint64_t* h_seeds,
+            float* out_vals, uint32_t* out_idx, float* out, void* stream);
+
+/* One whole step with the step's inputs and result in HOST memory: h_grads
+ * (W rows of n, ideally pinned) is copied to device staging owned by the
+ * context, worker by worker, overlapped with the compression of the previous
+ * worker; the dense average is copied back to h_out[n].  residuals stay on the
+ * device (they are the only state carried between steps).  The first call
+ * allocates the staging (cudaMalloc).  Returns after the result is in h_out. */
+int sc_step_host(sc_ctx* ctx, int scheme, int W, const float* h_grads, float* residuals, size_t n,
+                 const sc_segment* segs, int nseg, const uint64_t* h_seeds, float* h_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSECOMM_H */

@@ -1,0 +1,456 @@
+// Host side of the C ABI declared in include/sparsecomm.h: argument checks, scratch
+// ownership, the device-side segment table and the launch sequences.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/sparsecomm.h"
+#include "sc_aggregate.cuh"
+#include "sc_common.cuh"
+#include "sc_pack.cuh"
+#include "sc_random.cuh"
+#include "sc_topk.cuh"
+
+using namespace sc;
+
+struct sc_ctx {
+    int device = 0;
+    int sm_count = 0;
+    size_t max_n = 0;
+    int max_W = 0, max_seg = 0;
+    size_t max_tiles_per_worker = 0;
+    size_t max_mask_words = 0;      // per seed group
+    size_t max_atiles = 0;
+    size_t scratch_bytes = 0;
+
+    SegEntry* d_segs = nullptr;
+    uint32_t* d_hist = nullptr;
+    TopkState* d_state = nullptr;
+    unsigned long long* d_desc = nullptr;
+    unsigned long long* d_ticket = nullptr;
+    uint32_t* d_mask = nullptr;
+    uint32_t* d_bounds = nullptr;
+    uint64_t* d_seeds = nullptr;
+    int* d_status = nullptr;
+
+    std::vector<sc_segment> cached_segs;
+    size_t cached_n = 0;
+    bool layout_valid = false;
+    Layout layout{};
+
+    unsigned long long ticket_base = 0;
+    uint32_t epoch = 0;
+    uint64_t launches = 0;
+
+    int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1;
+
+    // host-buffer entry point
+    float* d_stage_grads = nullptr;
+    float* d_stage_vals = nullptr;
+    uint32_t* d_stage_idx = nullptr;
+    float* d_stage_out = nullptr;
+    size_t stage_grads_elems = 0, stage_msg_elems = 0, stage_out_elems = 0;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_start = nullptr;
+    std::vector<cudaEvent_t> ev_worker;
+};
+
+namespace {
+
+#define SC_CUDA(call)                                   \
+    do {                                                \
+        cudaError_t err__ = (call);                     \
+        if (err__ != cudaSuccess) return SC_ERR_CUDA;   \
+    } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+int dev_alloc(sc_ctx* c, T** p, size_t count) {
+    size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
+    if (cudaMalloc(reinterpret_cast<void**>(p), bytes) != cudaSuccess) { *p = nullptr; return SC_ERR_WORKSPACE; }
+    c->scratch_bytes += bytes;
+    return SC_OK;
+}
+
+class DeviceGuard {
+  public:
+    explicit DeviceGuard(int dev) { cudaGetDevice(&prev_); if (prev_ != dev) { cudaSetDevice(dev); set_ = true; } }
+    ~DeviceGuard() { if (set_) cudaSetDevice(prev_); }
+  private:
+    int prev_ = 0;
+    bool set_ = false;
+};
+
+// Validates the segment table and (re)builds the device copy when it changed.
+int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaStream_t stream) {
+    if (c->layout_valid && c->cached_n == n && (int)c->cached_segs.size() == nseg &&
+        std::memcmp(c->cached_segs.data(), segs, sizeof(sc_segment) * nseg) == 0)
+        return SC_OK;
+    std::vector<SegEntry> h(nseg + 1);
+    uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0;
+    for (int s = 0; s < nseg; ++s) {
+        const sc_segment& g = segs[s];
+        if (g.offset < end_prev || g.offset > n || g.n > n - g.offset) return SC_ERR_INVALID;
+        if (g.k > g.n) return SC_ERR_RANGE;
+        end_prev = g.offset + g.n;
+        SegEntry e{};
+        e.offset = g.offset; e.n = (uint32_t)g.n; e.k = (uint32_t)g.k;
+        e.msg_off = (uint32_t)msg; e.tile_begin = (uint32_t)tiles; e.scat_begin = (uint32_t)scat;
+        e.mask_word_begin = maskw;
+        h[s] = e;
+        tiles += (g.n + 3 + TILE - 1) / TILE;
+        scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
+        maskw += (g.n + 31) / 32;
+        msg += g.k;
+    }
+    if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
+    SegEntry sentinel{};
+    sentinel.offset = n; sentinel.msg_off = (uint32_t)msg; sentinel.tile_begin = (uint32_t)tiles;
+    sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw;
+    h[nseg] = sentinel;
+    SC_CUDA(cudaMemcpyAsync(c->d_segs, h.data(), sizeof(SegEntry) * (nseg + 1), cudaMemcpyHostToDevice, stream));
+    Layout L{};
+    L.segs = c->d_segs; L.nseg = (uint32_t)nseg; L.tiles_per_worker = (uint32_t)tiles;
+    L.scat_per_group = (uint32_t)scat; L.K_total = (uint32_t)msg; L.n_total = n; L.mask_words_per_group = maskw;
+    c->layout = L;
+    c->cached_segs.assign(segs, segs + nseg);
+    c->cached_n = n;
+    c->layout_valid = true;
+    return SC_OK;
+}
+
+int check_batch_args(const sc_ctx* c, int scheme, int W, const void* grads, const void* residuals, size_t n,
+                     const sc_segment* segs, int nseg, const uint64_t* seeds, const void* out_vals,
+                     const void* out_idx) {
+    if (!c || !segs || !seeds) return SC_ERR_INVALID;
+    if (scheme != SC_TOPK && scheme != SC_RANDK && scheme != SC_RANDBLOCK) return SC_ERR_INVALID;
+    if (W < 1 || W > c->max_W || nseg < 1 || nseg > c->max_seg) return SC_ERR_RANGE;
+    if (n >= (1ull << 32) || n > c->max_n) return SC_ERR_RANGE;
+    uint64_t K = 0;
+    for (int s = 0; s < nseg; ++s) {
+        if (segs[s].k > segs[s].n) return SC_ERR_RANGE;
+        K += segs[s].k;
+    }
+    if (n > 0 && (!grads || !residuals)) return SC_ERR_INVALID;
+    if (K > 0 && (!out_vals || !out_idx)) return SC_ERR_INVALID;
+    if (!aligned16(grads) || !aligned16(residuals)) return SC_ERR_INVALID;
+    return SC_OK;
+}
+
+inline uint32_t persistent_grid(const sc_ctx* c, int occ, uint64_t items) {
+    uint64_t cap = (uint64_t)c->sm_count * (uint64_t)std::max(occ, 1);
+    return (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(items, cap));
+}
+
+// Compression of rows [0, W) of the given base pointers.  `mask_ready` tells the
+// random-k path that the membership mask of seed group 0 is already built (used
+// when one shared-seed step is issued worker by worker).
+int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
+                  const uint64_t* h_seeds, bool shared_seeds, bool mask_ready,
+                  float* out_vals, uint32_t* out_idx, cudaStream_t stream) {
+    const Layout& L = c->layout;
+    if (n == 0 || L.tiles_per_worker == 0) return SC_OK;
+    const uint64_t items64 = (uint64_t)W * L.tiles_per_worker;
+    if (items64 > 0xFFFFFFF0ull) return SC_ERR_RANGE;
+    const uint32_t items = (uint32_t)items64;
+    const uint32_t P = (uint32_t)W * L.nseg;
+
+    if (scheme == SC_TOPK) {
+        SC_CUDA(cudaMemsetAsync(c->d_hist, 0, (size_t)P * HIST_WORDS * sizeof(uint32_t), stream));
+        topk_hist0_kernel<true><<<persistent_grid(c, c->occ_hist, items), THREADS, 0, stream>>>(
+            L, grads, residuals, c->d_hist, items);
+        topk_resolve_kernel<0><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status);
+        topk_refine_kernel<1><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
+            L, residuals, c->d_hist, c->d_state, items);
+        topk_resolve_kernel<1><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status);
+        topk_refine_kernel<2><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
+            L, residuals, c->d_hist, c->d_state, items);
+        topk_resolve_kernel<2><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status);
+        c->launches += 6;
+    } else {
+        SC_CUDA(cudaMemcpyAsync(c->d_seeds, h_seeds, sizeof(uint64_t) * W, cudaMemcpyHostToDevice, stream));
+    }
+
+    if (scheme == SC_RANDBLOCK) {
+        randblock_kernel<<<persistent_grid(c, c->occ_block, items), THREADS, 0, stream>>>(
+            L, grads, residuals, c->d_seeds, out_vals, out_idx, items);
+        c->launches += 1;
+        SC_CUDA(cudaGetLastError());
+        return SC_OK;
+    }
+
+    if (scheme == SC_RANDK && !mask_ready) {
+        const uint32_t groups = shared_seeds ? 1u : (uint32_t)W;
+        SC_CUDA(cudaMemsetAsync(c->d_mask, 0, (size_t)groups * L.mask_words_per_group * sizeof(uint32_t), stream));
+        const uint64_t blocks = (uint64_t)groups * L.scat_per_group;
+        if (blocks > 0x7FFFFFFFull) return SC_ERR_RANGE;
+        if (blocks > 0) {
+            randk_scatter_kernel<<<(uint32_t)blocks, THREADS, 0, stream>>>(L, c->d_seeds, c->d_mask, c->d_status);
+            c->launches += 1;
+        }
+    }
+
+    PackParams pp{};
+    pp.L = L; pp.grads = grads; pp.residuals = residuals; pp.out_vals = out_vals; pp.out_idx = out_idx;
+    pp.state = c->d_state; pp.mask = c->d_mask; pp.mask_per_worker = shared_seeds ? 0u : 1u;
+    if (++c->epoch >= (1u << 28)) {            // tags wrapped: forget every old word
+        SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), stream));
+        c->epoch = 1;
+    }
+    pp.epoch = c->epoch; pp.total_items = items;
+    pp.ticket = c->d_ticket; pp.ticket_base = c->ticket_base;
+    pp.desc = c->d_desc; pp.status = c->d_status;
+    uint32_t grid;
+    if (scheme == SC_TOPK) {
+        grid = persistent_grid(c, c->occ_pack_topk, items);
+        pack_kernel<PACK_TOPK><<<grid, THREADS, 0, stream>>>(pp);
+    } else {
+        grid = persistent_grid(c, c->occ_pack_mask, items);
+        pack_kernel<PACK_MASK><<<grid, THREADS, 0, stream>>>(pp);
+    }
+    c->ticket_base += (unsigned long long)items + grid;   // every CTA draws exactly one ticket past the end
+    c->launches += 1;
+    SC_CUDA(cudaGetLastError());
+    return SC_OK;
+}
+
+int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, bool shared_idx, size_t k, size_t n,
+                   float* out, cudaStream_t stream) {
+    if (n == 0) return SC_OK;
+    const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
+    const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
+    const uint64_t threads = (uint64_t)rows * (ntiles + 1ull);
+    agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
+        idx, rows, (uint32_t)k, ntiles, c->d_bounds);
+    agg_tiles_kernel<<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, stream>>>(
+        vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+    c->launches += 2;
+    SC_CUDA(cudaGetLastError());
+    return SC_OK;
+}
+
+int check_aggregate_args(const sc_ctx* c, int W, const void* vals, const void* idx, size_t k, size_t n, const void* out) {
+    if (!c) return SC_ERR_INVALID;
+    if (W < 1 || W > c->max_W) return SC_ERR_RANGE;
+    if (n >= (1ull << 32) || n > c->max_n || k > n) return SC_ERR_RANGE;
+    if (n > 0 && !out) return SC_ERR_INVALID;
+    if (k > 0 && (!vals || !idx)) return SC_ERR_INVALID;
+    if (!aligned16(out)) return SC_ERR_INVALID;
+    return SC_OK;
+}
+
+bool all_equal(const uint64_t* s, int W) {
+    for (int w = 1; w < W; ++w) if (s[w] != s[0]) return false;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sc_strerror(int code) {
+    switch (code) {
+        case SC_OK: return "ok";
+        case SC_ERR_INVALID: return "invalid argument";
+        case SC_ERR_RANGE: return "size out of range";
+        case SC_ERR_WORKSPACE: return "scratch allocation failed";
+        case SC_ERR_CUDA: return "CUDA runtime error";
+        case SC_ERR_TIMEOUT: return "bounded device wait timed out";
+        case SC_ERR_UNSUPPORTED: return "unsupported";
+        case SC_ERR_DEVICE_CHECK: return "device-side range check failed";
+        default: return "unknown status";
+    }
+}
+
+int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
+    if (!out) return SC_ERR_INVALID;
+    *out = nullptr;
+    if (max_W < 1 || max_segments < 1 || max_n >= (1ull << 32)) return SC_ERR_RANGE;
+    sc_ctx* c = new (std::nothrow) sc_ctx();
+    if (!c) return SC_ERR_WORKSPACE;
+    if (cudaGetDevice(&c->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
+        delete c;
+        return SC_ERR_CUDA;
+    }
+    c->max_n = max_n; c->max_W = max_W; c->max_seg = max_segments;
+    c->max_tiles_per_worker = (max_n + 3 + TILE - 1) / TILE + (size_t)max_segments + 1;
+    c->max_mask_words = (max_n + 31) / 32 + (size_t)max_segments;
+    c->max_atiles = (max_n + ATILE - 1) / ATILE;
+    const size_t P = (size_t)max_W * max_segments;
+    int rc = SC_OK;
+    if ((rc = dev_alloc(c, &c->d_segs, (size_t)max_segments + 1)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_hist, P * HIST_WORDS)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_state, P)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_desc, (size_t)max_W * c->max_tiles_per_worker * 2)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_ticket, 1)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_mask, (size_t)max_W * c->max_mask_words)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_bounds, (size_t)max_W * (c->max_atiles + 1))) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_seeds, (size_t)max_W)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_status, 1)) == SC_OK) {
+        bool ok = cudaMemset(c->d_desc, 0, (size_t)max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long)) == cudaSuccess &&
+                  cudaMemset(c->d_ticket, 0, sizeof(unsigned long long)) == cudaSuccess &&
+                  cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess &&
+                  cudaMemset(c->d_state, 0, P * sizeof(TopkState)) == cudaSuccess;
+        if (!ok) rc = SC_ERR_CUDA;
+    }
+    if (rc == SC_OK) {
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel<true>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_refine, topk_refine_kernel<1>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_topk, pack_kernel<PACK_TOPK>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_mask, pack_kernel<PACK_MASK>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_block, randblock_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel, THREADS, 0);
+        if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
+    }
+    if (rc != SC_OK) { sc_destroy(c); return rc; }
+    *out = c;
+    return SC_OK;
+}
+
+void sc_destroy(sc_ctx* c) {
+    if (!c) return;
+    DeviceGuard guard(c->device);
+    cudaFree(c->d_segs); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
+    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_seeds); cudaFree(c->d_status);
+    cudaFree(c->d_stage_grads); cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); cudaFree(c->d_stage_out);
+    for (cudaEvent_t e : c->ev_worker) cudaEventDestroy(e);
+    if (c->ev_start) cudaEventDestroy(c->ev_start);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    delete c;
+}
+
+int sc_sync_status(sc_ctx* c, void* stream) {
+    if (!c) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SC_CUDA(cudaStreamSynchronize(st));
+    int h = 0;
+    SC_CUDA(cudaMemcpyAsync(&h, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    SC_CUDA(cudaStreamSynchronize(st));
+    if (h != 0) {
+        SC_CUDA(cudaMemsetAsync(c->d_status, 0, sizeof(int), st));
+        SC_CUDA(cudaStreamSynchronize(st));
+    }
+    return h;
+}
+
+size_t sc_scratch_bytes(const sc_ctx* c) { return c ? c->scratch_bytes : 0; }
+uint64_t sc_launch_count(const sc_ctx* c) { return c ? c->launches : 0; }
+
+int sc_compress_batch(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
+                      const sc_segment* segs, int nseg, const uint64_t* h_seeds,
+                      float* out_vals, uint32_t* out_idx, void* stream) {
+    int rc = check_batch_args(c, scheme, W, grads, residuals, n, segs, nseg, h_seeds, out_vals, out_idx);
+    if (rc != SC_OK) return rc;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = prepare_layout(c, n, segs, nseg, st)) != SC_OK) return rc;
+    return compress_rows(c, scheme, W, grads, residuals, n, h_seeds, all_equal(h_seeds, W), false, out_vals, out_idx, st);
+}
+
+int sc_compress(sc_ctx* c, int scheme, const float* grad, float* residual, size_t n, size_t k,
+                uint64_t seed, float* out_vals, uint32_t* out_idx, void* stream) {
+    sc_segment seg{0, n, k};
+    return sc_compress_batch(c, scheme, 1, grad, residual, n, &seg, 1, &seed, out_vals, out_idx, stream);
+}
+
+int sc_aggregate(sc_ctx* c, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                 float* out, void* stream) {
+    int rc = check_aggregate_args(c, W, vals, idx, k, n, out);
+    if (rc != SC_OK) return rc;
+    DeviceGuard guard(c->device);
+    return aggregate_rows(c, W, vals, idx, false, k, n, out, static_cast<cudaStream_t>(stream));
+}
+
+int sc_aggregate_shared(sc_ctx* c, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                        float* out, void* stream) {
+    int rc = check_aggregate_args(c, W, vals, idx, k, n, out);
+    if (rc != SC_OK) return rc;
+    DeviceGuard guard(c->device);
+    return aggregate_rows(c, W, vals, idx, true, k, n, out, static_cast<cudaStream_t>(stream));
+}
+
+int sc_step(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
+            const sc_segment* segs, int nseg, const uint64_t* h_seeds,
+            float* out_vals, uint32_t* out_idx, float* out, void* stream) {
+    int rc = check_batch_args(c, scheme, W, grads, residuals, n, segs, nseg, h_seeds, out_vals, out_idx);
+    if (rc != SC_OK) return rc;
+    if ((n > 0 && !out) || !aligned16(out)) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = prepare_layout(c, n, segs, nseg, st)) != SC_OK) return rc;
+    const bool shared = all_equal(h_seeds, W);
+    if ((rc = compress_rows(c, scheme, W, grads, residuals, n, h_seeds, shared, false, out_vals, out_idx, st)) != SC_OK)
+        return rc;
+    return aggregate_rows(c, W, out_vals, out_idx, shared && scheme != SC_TOPK, c->layout.K_total, n, out, st);
+}
+
+int sc_step_host(sc_ctx* c, int scheme, int W, const float* h_grads, float* residuals, size_t n,
+                 const sc_segment* segs, int nseg, const uint64_t* h_seeds, float* h_out, void* stream) {
+    // message pointers are internal here; pass non-null placeholders to the checker
+    int rc = check_batch_args(c, scheme, W, h_grads, residuals, n, segs, nseg, h_seeds, c, c);
+    if (rc != SC_OK) return rc;
+    if (n > 0 && !h_out) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = prepare_layout(c, n, segs, nseg, st)) != SC_OK) return rc;
+    const size_t K = c->layout.K_total;
+    // staging, grown on demand (first call, or a larger problem)
+    if (c->stage_grads_elems < (size_t)W * n) {
+        SC_CUDA(cudaStreamSynchronize(st));
+        cudaFree(c->d_stage_grads); c->d_stage_grads = nullptr; c->stage_grads_elems = 0;
+        if (cudaMalloc(reinterpret_cast<void**>(&c->d_stage_grads), std::max<size_t>((size_t)W * n, 4) * sizeof(float)) != cudaSuccess)
+            return SC_ERR_WORKSPACE;
+        c->stage_grads_elems = (size_t)W * n;
+    }
+    if (c->stage_msg_elems < (size_t)W * K) {
+        SC_CUDA(cudaStreamSynchronize(st));
+        cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); c->d_stage_vals = nullptr; c->d_stage_idx = nullptr;
+        c->stage_msg_elems = 0;
+        if (cudaMalloc(reinterpret_cast<void**>(&c->d_stage_vals), std::max<size_t>((size_t)W * K, 4) * sizeof(float)) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&c->d_stage_idx), std::max<size_t>((size_t)W * K, 4) * sizeof(uint32_t)) != cudaSuccess)
+            return SC_ERR_WORKSPACE;
+        c->stage_msg_elems = (size_t)W * K;
+    }
+    if (c->stage_out_elems < n) {
+        SC_CUDA(cudaStreamSynchronize(st));
+        cudaFree(c->d_stage_out); c->d_stage_out = nullptr; c->stage_out_elems = 0;
+        if (cudaMalloc(reinterpret_cast<void**>(&c->d_stage_out), std::max<size_t>(n, 4) * sizeof(float)) != cudaSuccess)
+            return SC_ERR_WORKSPACE;
+        c->stage_out_elems = n;
+    }
+    if (!c->copy_stream) SC_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+    if (!c->ev_start) SC_CUDA(cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming));
+    while ((int)c->ev_worker.size() < W) {
+        cudaEvent_t e;
+        SC_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        c->ev_worker.push_back(e);
+    }
+    // copies of worker w+1.. overlap the compression of worker w
+    SC_CUDA(cudaEventRecord(c->ev_start, st));
+    SC_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_start, 0));
+    for (int w = 0; w < W; ++w) {
+        SC_CUDA(cudaMemcpyAsync(c->d_stage_grads + (size_t)w * n, h_grads + (size_t)w * n, n * sizeof(float),
+                                cudaMemcpyHostToDevice, c->copy_stream));
+        SC_CUDA(cudaEventRecord(c->ev_worker[w], c->copy_stream));
+    }
+    const bool shared = all_equal(h_seeds, W);
+    for (int w = 0; w < W; ++w) {
+        SC_CUDA(cudaStreamWaitEvent(st, c->ev_worker[w], 0));
+        rc = compress_rows(c, scheme, 1, c->d_stage_grads + (size_t)w * n, residuals + (size_t)w * n, n,
+                           h_seeds + w, shared, shared && w > 0,
+                           c->d_stage_vals + (size_t)w * K, c->d_stage_idx + (size_t)w * K, st);
+        if (rc != SC_OK) return rc;
+    }
+    rc = aggregate_rows(c, W, c->d_stage_vals, c->d_stage_idx, shared && scheme != SC_TOPK, K, n, c->d_stage_out, st);
+    if (rc != SC_OK) return rc;
+    SC_CUDA(cudaMemcpyAsync(h_out, c->d_stage_out, n * sizeof(float), cudaMemcpyDeviceToHost, st));
+    SC_CUDA(cudaStreamSynchronize(st));
+    return SC_OK;
+}
+
+}  // extern "C"

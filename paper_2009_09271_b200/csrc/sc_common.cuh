@@ -1,0 +1,206 @@
+// Shared device-side definitions for the sparsified-SGD compressor kernels (sm_100a).
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace sc {
+
+constexpr int THREADS = 256;            // threads per CTA in every tile kernel
+constexpr int QUADS = 4;                // float4 per thread per tile
+constexpr int TILE = THREADS * QUADS * 4;   // 4096 elements = 16 KB per operand per tile
+constexpr int WARPS = THREADS / 32;
+
+constexpr uint32_t HIST0_BINS = 2048;   // key bits 30..20
+constexpr uint32_t HIST1_BINS = 1024;   // key bits 19..10
+constexpr uint32_t HIST2_BINS = 1024;   // key bits  9..0
+constexpr uint32_t HIST_WORDS = HIST0_BINS + HIST1_BINS + HIST2_BINS;
+
+// device status codes (mirrors the public header)
+constexpr int ST_TIMEOUT = -5;
+constexpr int ST_DEVICE_CHECK = -7;
+
+// One tensor of the gradient as the kernels see it.
+struct SegEntry {
+    uint64_t offset;          // first element inside a worker row
+    uint64_t mask_word_begin; // first 32-bit word of this segment's membership mask
+    uint32_t n, k;
+    uint32_t msg_off;         // K_s: first message slot of the segment
+    uint32_t tile_begin;      // first tile of the segment inside a worker
+    uint32_t scat_begin;      // first scatter chunk of the segment inside a seed group
+    uint32_t pad;
+};
+
+struct Layout {
+    const SegEntry* segs;     // device array, nseg + 1 entries (last = sentinel with the totals)
+    uint32_t nseg;
+    uint32_t tiles_per_worker;
+    uint32_t scat_per_group;
+    uint32_t K_total;         // message entries per worker
+    uint64_t n_total;         // elements per worker row
+    uint64_t mask_words_per_group;
+};
+
+// Per (worker, segment) result of the radix select.
+struct TopkState {
+    uint32_t prefix;   // key bits fixed so far
+    uint32_t need;     // how many elements of the current bucket are still to be taken
+    uint32_t active;   // 1 while the threshold is not final
+    uint32_t T;        // threshold key: every key > T is kept
+    uint32_t r;        // number of elements with key == T that are kept (lowest coordinates first)
+    uint32_t dual;     // 1 if only some of the ties are kept (r < number of ties)
+    uint32_t pad0, pad1;
+};
+
+// ---------------------------------------------------------------------------
+// integer hashing (the generator specification; integer-only, so host, device
+// and any other implementation agree bit for bit)
+// ---------------------------------------------------------------------------
+__host__ __device__ inline uint64_t mix64(uint64_t a, uint64_t b) {
+    uint64_t z = a + (b + 1ull) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+__host__ __device__ inline uint32_t mix32(uint32_t x) {
+    x ^= x >> 16; x *= 0x6A09E667u;
+    x ^= x >> 15; x *= 0xBB67AE85u;
+    x ^= x >> 16;
+    return x;
+}
+
+constexpr uint64_t SALT_BLOCK = 0x626C6F636Bull;
+constexpr uint64_t SALT_RANDK = 0x72616E646B00ull;
+constexpr int FEISTEL_ROUNDS = 6;
+
+__device__ inline uint32_t block_start(uint64_t seed_s, uint32_t n, uint32_t k) {
+    uint64_t h = mix64(seed_s, SALT_BLOCK);
+    return (uint32_t)__umul64hi(h, (uint64_t)(n - k) + 1ull);
+}
+
+struct Feistel {
+    uint32_t keys[FEISTEL_ROUNDS];
+    uint32_t left, right, mask_l, mask_r;
+};
+
+__device__ inline Feistel feistel_setup(uint64_t seed_s, uint32_t n) {
+    Feistel f;
+    uint32_t b = (n <= 1u) ? 0u : 32u - (uint32_t)__clz((int)(n - 1u));
+    if (b < 2u) b = 2u;
+    f.left = b >> 1;
+    f.right = b - f.left;
+    f.mask_l = (1u << f.left) - 1u;
+    f.mask_r = (f.right >= 32u) ? 0xFFFFFFFFu : ((1u << f.right) - 1u);
+#pragma unroll
+    for (int r = 0; r < FEISTEL_ROUNDS; ++r) f.keys[r] = (uint32_t)(mix64(seed_s, SALT_RANDK + (uint64_t)r) >> 32);
+    return f;
+}
+
+__device__ inline uint32_t feistel_once(const Feistel& f, uint32_t x) {
+    uint32_t L = (x >> f.right) & f.mask_l;
+    uint32_t R = x & f.mask_r;
+#pragma unroll
+    for (int r = 0; r < FEISTEL_ROUNDS; ++r) {
+        if ((r & 1) == 0) L ^= mix32(R ^ f.keys[r]) & f.mask_l;
+        else              R ^= mix32(L ^ f.keys[r]) & f.mask_r;
+    }
+    return (L << f.right) | R;
+}
+
+// ---------------------------------------------------------------------------
+// tile addressing
+// ---------------------------------------------------------------------------
+// Finds the segment that owns local tile `lt` (thread-uniform, a few cached loads).
+__device__ inline uint32_t find_by_tile(const Layout& L, uint32_t lt) {
+    uint32_t lo = 0, hi = L.nseg;
+    while (hi - lo > 1) {
+        uint32_t mid = (lo + hi) >> 1;
+        if (L.segs[mid].tile_begin <= lt) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+__device__ inline uint32_t find_by_scat(const Layout& L, uint32_t ls) {
+    uint32_t lo = 0, hi = L.nseg;
+    while (hi - lo > 1) {
+        uint32_t mid = (lo + hi) >> 1;
+        if (L.segs[mid].scat_begin <= ls) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// A quad is four consecutive elements starting at segment-local element `base`
+// (which may be negative or reach past n for the ragged first/last quad).  The
+// address seg + base is 16-byte aligned by construction.
+__device__ inline uint32_t load_quad(const float* __restrict__ seg, long long base, uint32_t n, float v[4]) {
+    if (base >= 0 && base + 3 < (long long)n) {
+        float4 q = *reinterpret_cast<const float4*>(seg + base);
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+        return 0xFu;
+    }
+    uint32_t m = 0;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        long long i = base + c;
+        if (i >= 0 && i < (long long)n) { v[c] = seg[i]; m |= 1u << c; } else v[c] = 0.0f;
+    }
+    return m;
+}
+__device__ inline uint32_t load_quad_stream(const float* __restrict__ seg, long long base, uint32_t n, float v[4]) {
+    if (base >= 0 && base + 3 < (long long)n) {
+        float4 q = __ldcs(reinterpret_cast<const float4*>(seg + base));
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+        return 0xFu;
+    }
+    uint32_t m = 0;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        long long i = base + c;
+        if (i >= 0 && i < (long long)n) { v[c] = __ldcs(seg + i); m |= 1u << c; } else v[c] = 0.0f;
+    }
+    return m;
+}
+__device__ inline void store_quad(float* __restrict__ seg, long long base, uint32_t valid, const float v[4]) {
+    if (valid == 0xFu) {
+        *reinterpret_cast<float4*>(seg + base) = make_float4(v[0], v[1], v[2], v[3]);
+        return;
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        if ((valid >> c) & 1u) seg[base + c] = v[c];
+}
+
+__device__ inline uint32_t key_of(float p) { return __float_as_uint(p) & 0x7FFFFFFFu; }
+
+__device__ inline uint32_t misalign_of(const void* p) { return (uint32_t)((reinterpret_cast<uintptr_t>(p) >> 2) & 3u); }
+
+// block-wide exclusive scan of one value per thread (THREADS threads); returns
+// the exclusive prefix, *total receives the block sum.  smem: WARPS + 1 words.
+__device__ inline uint32_t block_exclusive_scan(uint32_t v, uint32_t* smem, uint32_t* total) {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= (uint32_t)d) inc += t;
+    }
+    if (lane == 31u) smem[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = (lane < (uint32_t)WARPS) ? smem[lane] : 0u;
+        uint32_t winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t t = __shfl_up_sync(0xFFFFFFFFu, winc, d);
+            if (lane >= (uint32_t)d) winc += t;
+        }
+        if (lane < (uint32_t)WARPS) smem[lane] = winc - w;
+        if (lane == (uint32_t)WARPS - 1u) smem[WARPS] = winc;
+    }
+    __syncthreads();
+    uint32_t res = smem[warp] + inc - v;
+    *total = smem[WARPS];
+    __syncthreads();
+    return res;
+}
+
+}  // namespace sc

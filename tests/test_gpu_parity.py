@@ -1,0 +1,227 @@
+"""GPU parity: the CUDA library against the CPU oracle, bit for bit, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2009_09271_b200 as sc
+import workloads as wl
+from oracle import sparsify_oracle as O
+from parity_util import assert_bits_equal, run_step_both
+
+pytestmark = pytest.mark.gpu
+
+SCHEMES = [sc.SC_TOPK, sc.SC_RANDK, sc.SC_RANDBLOCK]
+TILE = 4096
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = sc.Context(max_n=1 << 21, max_W=8, max_segments=64)
+    yield c
+    c.close()
+
+
+def rand(n, seed, scale=1e-3):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randn(n, generator=g) * scale
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+@pytest.mark.parametrize("n", [1, 2, 3, 31, 32, 33, 1023, 1024, 1025, TILE - 1, TILE, TILE + 1,
+                               2 * TILE - 3, 3 * TILE + 5, 100_003])
+def test_single_worker_sizes(ctx, scheme, n):
+    g = rand(n, n).view(1, n)
+    e = rand(n, n + 1).view(1, n)
+    for k in sorted({0, 1, (n + 99) // 100, n // 2, n - 1, n} & set(range(n + 1))):
+        run_step_both(ctx, scheme, g, e, [(0, n, k)], [1234 + k])
+
+
+def test_topk_massive_ties_and_special_values(ctx):
+    n = 3 * TILE + 17
+    g = torch.zeros(1, n)
+    e = torch.zeros(1, n)
+    pos = torch.randperm(n, generator=torch.Generator().manual_seed(0))
+    g[0, pos[:200]] = 1.0          # 200 equal large values, the rest exact zeros
+    g[0, pos[200:300]] = -1.0
+    for k in (1, 150, 299, 300, 301, 2000, n - 1):
+        run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, k)], [0])
+    sp = rand(n, 5).view(1, n)
+    sp[0, 5] = float("inf"); sp[0, 77] = float("-inf"); sp[0, 4096] = float("nan")
+    sp[0, 9:20] = 0.0; sp[0, 30:40] = -0.0
+    tiny = torch.from_numpy(np.array([1, 2, 0x80000001, 0x80000003], np.uint32).view(np.float32).copy())
+    sp[0, 100:104] = tiny
+    for k in (1, 2, 3, 50, n - 30, n - 5, n):
+        run_step_both(ctx, sc.SC_TOPK, sp, e, [(0, n, k)], [0])
+    # all values equal: the first k coordinates win
+    eq = torch.full((1, n), 0.25)
+    for k in (1, 100, TILE, TILE + 1, n):
+        run_step_both(ctx, sc.SC_TOPK, eq, e, [(0, n, k)], [0])
+    # small integers: thousands of ties at every level
+    ints = torch.randint(-5, 6, (1, n), generator=torch.Generator().manual_seed(2)).float()
+    for k in (10, 1000, 5000, n // 2):
+        run_step_both(ctx, sc.SC_TOPK, ints, e, [(0, n, k)], [0])
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+def test_segments_unaligned_multiworker(ctx, scheme):
+    sizes = [5, 64, 1, 4099, 33, 8192, 7, 12289, 2, 1000]
+    W = 5
+    segs = wl.segment_table(sizes, 1, 10)
+    n = sum(sizes)
+    g = torch.stack([rand(n, 100 + w) for w in range(W)])
+    e = torch.stack([rand(n, 200 + w) for w in range(W)])
+    run_step_both(ctx, scheme, g, e, segs, [7] * W)                       # shared coordinates
+    run_step_both(ctx, scheme, g, e, segs, [7, 8, 9, 10, 11])             # per-worker coordinates
+    run_step_both(ctx, scheme, g, e, segs, [7] * W, use="split")
+    # a table with gaps: elements outside every segment are left alone
+    gap = [(3, 100, 10), (200, 4096, 41), (5000, 13, 13), (6000, 9000, 0)]
+    run_step_both(ctx, scheme, g, e, gap, [3] * W)
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+def test_row_length_not_multiple_of_four(ctx, scheme):
+    W, n = 3, 2 * TILE + 1            # rows 1 and 2 start misaligned
+    g = torch.stack([rand(n, 300 + w) for w in range(W)])
+    e = torch.stack([rand(n, 400 + w) for w in range(W)])
+    run_step_both(ctx, scheme, g, e, [(0, n, 97)], [1, 1, 1])
+    run_step_both(ctx, scheme, g, e, [(1, 4000, 40), (4001, n - 4001, 400)], [1, 2, 3])
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+def test_multistep_error_feedback_c1(ctx, scheme):
+    """Workload 1 at full size: n = 2^20, W = 4, k = 10,486, three steps with the
+    residual carried from step to step."""
+    w1 = wl.workload("c1")
+    segs = wl.flat_table(w1.n, 1, 100)
+    assert segs[0].k == 10_486
+    e = torch.zeros(w1.W, w1.n)
+    for t in range(w1.steps):
+        g = torch.stack([wl.generate(w1, w, t, "cpu") for w in range(w1.W)])
+        e = run_step_both(ctx, scheme, g, e, segs, [wl.step_seed(w1.base_seed, t)] * w1.W)
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+def test_telescoping_on_integer_gradients(ctx, scheme):
+    n, k, W, T = 20_000, 200, 2, 12
+    e = torch.zeros(W, n)
+    total = torch.zeros(W, n, dtype=torch.float64)
+    sent = torch.zeros(W, n, dtype=torch.float64)
+    dev_ctx = ctx
+    for t in range(T):
+        g = torch.stack([wl.gen_small_integers(n, wl.make_generator(9, w, t, "cpu"), "cpu") for w in range(W)])
+        total += g
+        gd, ed = g.cuda(), e.cuda()
+        vals = torch.empty(W, k, device="cuda"); idx = torch.empty(W, k, device="cuda", dtype=torch.int32)
+        dev_ctx.sc_compress_batch(scheme, gd, ed, [(0, n, k)], [t, t + 100], vals, idx)
+        assert dev_ctx.sc_sync_status() == 0
+        for w in range(W):
+            sent[w, idx[w].long().cpu()] += vals[w].double().cpu()
+        e = ed.cpu()
+    assert torch.equal(sent + e.double(), total)
+
+
+def test_reduced_resnet_shapes(ctx):
+    """Workloads 2 and 3 with every tensor shrunk 16x (same count of segments, same mix
+    of tiny and large tensors), 3 steps each with error feedback."""
+    for name, schemes in (("c2", [sc.SC_RANDBLOCK]), ("c3", SCHEMES)):
+        w = wl.workload(name)
+        sizes = [max(1, s // 16) for s in w.sizes][:64] if name == "c3" else [max(1, s // 16) for s in w.sizes]
+        num, den = w.densities[0]
+        segs = wl.segment_table(sizes, num, den)
+        n = sum(sizes)
+        W = 4
+        for scheme in schemes:
+            e = torch.zeros(W, n)
+            for t in range(3):
+                g = torch.stack([wl.generate(w, ww, t, "cpu", sizes=sizes) for ww in range(W)])
+                e = run_step_both(ctx, scheme, g, e, segs, [wl.step_seed(w.base_seed, t)] * W)
+
+
+def test_lstm_like_zero_rows(ctx):
+    """Workload 4 structure: embedding tensors with 95 % exactly-zero rows, so that the
+    top-k threshold is zero and most kept entries are ties."""
+    sizes = [650 * 300, 20_000, 20_000, 650 * 300, 301, 50_000]
+    w4 = wl.workload("c4")
+    W = 3
+    n = sum(sizes)
+    for num, den in ((1, 1000), (1, 100), (1, 10)):
+        for scheme in (sc.SC_TOPK, sc.SC_RANDBLOCK):
+            for segs in (wl.segment_table(sizes, num, den), wl.flat_table(n, num, den)):
+                e = torch.zeros(W, n)
+                for t in range(2):
+                    g = torch.stack([wl.generate(w4, ww, t, "cpu", sizes=sizes) for ww in range(W)])
+                    e = run_step_both(ctx, scheme, g, e, segs, [wl.step_seed(3, t)] * W)
+
+
+def test_aggregate_generic_shared_and_collisions(ctx):
+    rng = np.random.default_rng(0)
+    W, n, k = 7, 50_001, 5000
+    idx = np.stack([np.sort(rng.choice(n, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+    vals = (rng.standard_normal((W, k)) * 10.0 ** rng.uniform(-3, 3, (W, k))).astype(np.float32)
+    vals[0, :10] = -0.0
+    d_idx = torch.from_numpy(idx.view(np.int32)).cuda()
+    d_vals = torch.from_numpy(vals).cuda()
+    out = torch.full((n,), float("nan"), device="cuda")
+    ctx.sc_aggregate(W, d_vals, d_idx, k, n, out)
+    assert ctx.sc_sync_status() == 0
+    assert_bits_equal(out, O.aggregate(list(vals), list(idx), n), "generic aggregate")
+    out.fill_(float("nan"))
+    ctx.sc_aggregate_shared(W, d_vals, d_idx[0].contiguous(), k, n, out)
+    assert ctx.sc_sync_status() == 0
+    assert_bits_equal(out, O.aggregate(list(vals), [idx[0]] * W, n), "shared aggregate")
+    # k = 0: all zeros
+    ctx.sc_aggregate(W, d_vals, d_idx, 0, n, out)
+    assert ctx.sc_sync_status() == 0
+    assert not out.any() and not (out.view(torch.int32) != 0).any()
+    # every worker sends the same single coordinate, at the very end
+    one_i = torch.full((W, 1), n - 1, dtype=torch.int32, device="cuda")
+    one_v = torch.arange(1, W + 1, dtype=torch.float32, device="cuda").view(W, 1) * 0.1
+    ctx.sc_aggregate(W, one_v, one_i, 1, n, out)
+    want = O.aggregate(list(one_v.cpu().numpy()), list(one_i.cpu().numpy().view(np.uint32)), n)
+    assert_bits_equal(out, want, "single coordinate")
+
+
+def test_host_buffer_step(ctx):
+    W, n = 4, 3 * TILE + 9
+    g = torch.stack([rand(n, 500 + w) for w in range(W)])
+    e = torch.stack([rand(n, 600 + w) for w in range(W)])
+    for scheme in SCHEMES:
+        run_step_both(ctx, scheme, g, e, [(0, n, 123)], [5] * W, use="host")
+        run_step_both(ctx, scheme, g, e, [(0, n, 123)], [5, 6, 7, 8], use="host")
+
+
+def test_repeatable(ctx):
+    """The same call twice gives the same bits (no dependence on scheduling)."""
+    W, n, k = 4, 200_003, 2001
+    g = torch.stack([rand(n, 700 + w) for w in range(W)]).cuda()
+    e0 = torch.stack([rand(n, 800 + w) for w in range(W)]).cuda()
+    res = []
+    for _ in range(2):
+        e = e0.clone()
+        vals = torch.empty(W, k, device="cuda"); idx = torch.empty(W, k, device="cuda", dtype=torch.int32)
+        out = torch.empty(n, device="cuda")
+        ctx.sc_step(sc.SC_TOPK, g, e, [(0, n, k)], [0, 1, 2, 3], vals, idx, out)
+        assert ctx.sc_sync_status() == 0
+        res.append((vals.clone(), idx.clone(), out.clone(), e.clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+def test_argument_errors_leave_buffers_untouched(ctx):
+    n, k = 1000, 10
+    g = rand(n, 1).cuda(); e = rand(n, 2).cuda(); e0 = e.clone()
+    vals = torch.zeros(k, device="cuda"); idx = torch.zeros(k, device="cuda", dtype=torch.int32)
+    lib = sc.load_library()
+    h = ctx._h
+    assert lib.sc_compress(h, 7, g.data_ptr(), e.data_ptr(), n, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -1
+    assert lib.sc_compress(h, 0, g.data_ptr(), e.data_ptr(), n, n + 1, 0, vals.data_ptr(), idx.data_ptr(), None) == -2
+    assert lib.sc_compress(h, 0, None, e.data_ptr(), n, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -1
+    assert lib.sc_compress(h, 0, g.data_ptr() + 4, e.data_ptr(), n - 1, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -1
+    assert lib.sc_compress(h, 0, g.data_ptr(), e.data_ptr(), (1 << 21) + 1, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -2
+    assert lib.sc_aggregate(h, 0, vals.data_ptr(), idx.data_ptr(), k, n, e.data_ptr(), None) == -2
+    assert lib.sc_aggregate(h, 1, vals.data_ptr(), idx.data_ptr(), n + 1, n, e.data_ptr(), None) == -2
+    torch.cuda.synchronize()
+    assert torch.equal(e, e0) and not vals.any()
+    with pytest.raises(sc.SparseCommError):
+        ctx.sc_compress(9, g, e, k, 0, vals, idx)
+    assert sc.strerror(-2) == "size out of range"
