@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the sparsified-SGD compress + aggregate step on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic
+gradients: for each sparsifier of the workload (top-k, random-k, block-random-k)
+W workers are compressed (error-feedback add, selection, packing, residual
+writeback) and their messages are aggregated into one dense average.  The
+metric is gradient elements compressed per second (W * n * schemes / time).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compress+aggregate gradient elements/s"
+UNIT = "elements/s"
+CONTRACT_PEAK_GBS = 8000.0        # the nominal B200 HBM figure the target is stated against
+FALLBACK_PEAK_GBS = 6650.0        # used only if MEASURED_PEAKS.json is absent
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c5", help="c1..c5 (default: the largest, flat 350M x 16 workers)")
+    ap.add_argument("--density", default="1/100", help="kept fraction num/den (default: the paper's 1 %%)")
+    ap.add_argument("--schemes", default="", help="comma list; default: all schemes of the workload")
+    ap.add_argument("--n", type=int, default=0, help="override elements per worker (flat workloads only)")
+    ap.add_argument("--workers", type=int, default=0, help="override W")
+    ap.add_argument("--pool", type=int, default=2, help="distinct gradient sets cycled through the steps")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-div", type=int, default=4, help="oracle sample = n / this of one worker")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_PEAK_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid, self.proc, self.path = uuid, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="sc_clocks_", suffix=".csv")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=fd, stderr=subprocess.DEVNULL)
+            os.close(fd)
+            time.sleep(0.3)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.strip().split(",") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+                for name, v in zip(names, r[3:7]):
+                    if v.strip().lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        if sm:
+            busy = [c for c, p in zip(sm, pw) if p >= 0.5 * max(pw)] or sm
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(pw))
+        return out
+
+
+def algorithmic_bytes(kind: str, n: int, W: int, K: int, shared: bool) -> float:
+    """Bytes one launch of a kernel must move by the definition of its step
+    (operands read once, results written once)."""
+    return {
+        "topk_hist0": 12.0 * n * W,                      # read g, read e, write p
+        "topk_refine": 4.0 * n * W,                      # read p
+        "pack_topk": 4.0 * n * W + 12.0 * K * W,         # read p; write vals, idx and the kept zeros
+        "randk_pack": 12.0 * n * W + n / 8.0 * W + 8.0 * K * W,  # read g, e, mask; write e', vals, idx
+        "mask_count": n / 8.0, "row_scan": 8.0 * (n / 4096.0),
+        "randblock": 12.0 * n * W + 8.0 * K * W,
+        "randk_scatter": 4.0 * K,
+        "agg_tiles": 4.0 * n + (4.0 * K * W + 4.0 * K if shared else 8.0 * K * W),
+        "agg_bounds": 4.0 * (n / 4096.0) * (1 if shared else W),
+        "topk_resolve": 0.0,
+    }.get(kind, 0.0)
+
+
+def step_min_bytes(scheme: str, n: int, W: int, K: int, shared: bool) -> float:
+    """Minimum traffic of one whole step: read g and e, write e', write and read the messages,
+    write the dense average."""
+    if scheme == "topk" or not shared:
+        return 12.0 * n * W + 16.0 * K * W + 4.0 * n
+    return 12.0 * n * W + 8.0 * K * W + 8.0 * K + 4.0 * n
+
+
+def build_problem(args):
+    import workloads as wl
+    w = wl.workload(args.workload)
+    num, den = (int(x) for x in args.density.split("/"))
+    sizes = list(w.sizes)
+    if args.n:
+        sizes = [args.n]
+    W = args.workers or w.W
+    schemes = [s for s in (args.schemes.split(",") if args.schemes else w.schemes) if s]
+    segs = wl.segment_table(sizes, num, den)
+    return w, sizes, W, schemes, segs, (num, den)
+
+
+def run_reference(args, rank: int):
+    """Times the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    import workloads as wl
+    from oracle import sparsify_oracle as O
+    w, sizes, W, schemes, segs, (num, den) = build_problem(args)
+    n_full = sum(sizes)
+    # sample: one worker, the first n/div elements of a flat vector (or the whole table if it is small)
+    if len(sizes) == 1 and n_full > 50_000_000:
+        sizes = [n_full // args.cpu_sample_div]
+    segs = wl.segment_table(sizes, num, den)
+    n = sum(sizes)
+    seg_t = [(s.offset, s.n, s.k) for s in segs]
+    torch.manual_seed(0)
+    times = []
+    e = {s: np.zeros(n, np.float32) for s in schemes}
+    for t in range(args.warmup + args.steps):
+        g = wl.generate(w, 0, t, "cpu", sizes=sizes).numpy()
+        t0 = time.perf_counter()
+        for s in schemes:
+            v, i, e_new = O.compress_segments(O.SCHEMES[s], g, e[s], seg_t, wl.step_seed(w.base_seed, t))
+            O.aggregate([v], [i], n)
+            e[s] = e_new
+        if t >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    total = sum(times)
+    value = n * len(schemes) * len(times) / total
+    sample = (f"worker 0 only, {n} of {n_full} elements per step, schemes {','.join(schemes)}, density {num}/{den}, "
+              f"compress + aggregate of that one message (W=1)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: n={n_full} W={W} density={num}/{den}", "kind": "numpy oracle on host cores"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+    import paper_2009_09271_b200 as sc
+    import workloads as wl
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w, sizes, W, schemes, segs, (num, den) = build_problem(args)
+    n = sum(sizes)
+    K = sum(s.k for s in segs)
+    seg_t = [(s.offset, s.n, s.k) for s in segs]
+    codes = [sc.SCHEMES[s] for s in schemes]
+    pool = max(1, args.pool)
+
+    ctx = sc.Context(max_n=n, max_W=W, max_segments=len(segs))
+    grads = []
+    for t in range(pool):
+        g = torch.empty(W, n, device=dev)
+        for ww in range(W):
+            g[ww] = wl.generate(w, ww + 1000 * rank, t, dev, sizes=sizes)
+        grads.append(g)
+    res = {s: torch.zeros(W, n, device=dev) for s in schemes}
+    vals = torch.empty(W, max(K, 1), device=dev)
+    idx = torch.empty(W, max(K, 1), device=dev, dtype=torch.int32)
+    out = torch.empty(n, device=dev)
+
+    def seeds(t):
+        return [wl.step_seed(w.base_seed, t)] * W          # shared coordinates (the paper's allReduce mode)
+
+    def one_step(t, marks=None):
+        for s, code in zip(schemes, codes):
+            ctx.sc_step(code, grads[t % pool], res[s], seg_t, seeds(t), vals, idx, out)
+            if marks is not None:
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record()
+                marks.append(ev)
+
+    for t in range(args.warmup):
+        one_step(t)
+    status = ctx.sc_sync_status()
+    if status != 0:
+        raise RuntimeError(f"device status after warm-up: {sc.strerror(status)}")
+
+    sampler = ClockSampler(str(torch.cuda.get_device_properties(dev).uuid))
+    if not sampler.uuid.startswith("GPU-"):
+        sampler.uuid = "GPU-" + sampler.uuid
+    barrier()
+    if rank == 0:
+        sampler.start()
+    ctx.sc_profile(True)
+    launches0 = ctx.launch_count
+    marks = []
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for t in range(args.steps):
+        one_step(args.warmup + t, marks)
+    end.record()
+    barrier()
+    elapsed_ms = start.elapsed_time(end)
+    launches = ctx.launch_count - launches0
+    prof = ctx.sc_profile_read()
+    ctx.sc_profile(False)
+    clocks = sampler.stop() if rank == 0 else {}
+    status = ctx.sc_sync_status()
+    if status != 0:
+        raise RuntimeError(f"device status after the timed region: {sc.strerror(status)}")
+    if dist is not None:
+        tmax = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tmax.item())
+
+    # per-scheme device time from the marks
+    per_scheme_ms = {s: 0.0 for s in schemes}
+    prev = start
+    for i, ev in enumerate(marks):
+        per_scheme_ms[schemes[i % len(schemes)]] += prev.elapsed_time(ev)
+        prev = ev
+
+    peak, peak_src = measured_peak()
+    elems_per_step = W * n * len(schemes)
+    value = world * elems_per_step * args.steps / (elapsed_ms * 1e-3)
+
+    kernels = {}
+    for kind, (ms, cnt) in prof.items():
+        if cnt:
+            b = algorithmic_bytes(kind, n, W, K, shared=True)
+            kernels[kind] = {"launches": int(cnt), "ms_total": round(ms, 4), "ms_avg": round(ms / cnt, 5),
+                             "share": round(ms / max(elapsed_ms, 1e-9), 4),
+                             "alg_GBps": round(b / (ms / cnt * 1e-3) / 1e9, 1) if ms > 0 else None}
+    dom = max(kernels, key=lambda k_: kernels[k_]["ms_total"]) if kernels else None
+    roofline = None
+    if dom:
+        ach = kernels[dom]["alg_GBps"]
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s",
+                    "frac": round(ach / peak, 4), "peak_source": peak_src, "traffic": None}
+        tfile = os.path.join(ROOT, "profiles", "traffic.json")     # per-launch DRAM bytes from an ncu capture, if recorded
+        try:
+            tr = json.load(open(tfile)).get(dom)
+            if tr:
+                roofline["traffic"] = tr["bytes_per_element"] * n * W
+                roofline["traffic_note"] = tr.get("note")
+        except Exception:
+            pass
+    step_roof = {}
+    for s in schemes:
+        t_s = per_scheme_ms[s] / args.steps * 1e-3
+        bmin = step_min_bytes(s, n, W, K, shared=True)
+        step_roof[s] = {"ms": round(t_s * 1e3, 4), "elements_per_s": W * n / t_s, "min_GB": round(bmin / 1e9, 3),
+                        "GBps_min_bytes": round(bmin / t_s / 1e9, 1),
+                        "frac_of_8000": round(bmin / t_s / 1e9 / CONTRACT_PEAK_GBS, 4),
+                        "frac_of_measured": round(bmin / t_s / 1e9 / peak, 4)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: flat n={n} x W={W} simulated workers per GPU, {w.values} values, "
+                               f"density {num}/{den} (k={K}), schemes {','.join(schemes)}, shared seed per step, "
+                               f"error feedback on, {pool} gradient sets cycled",
+                   "segments": len(segs), "l2": "inputs (%.1f GB per scheme pass) far larger than L2" % (8e-9 * n * W),
+                   "replicas": world},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "per_scheme": step_roof,
+        "kernels": kernels,
+    }
+
+    # ---- end to end through the C ABI with host buffers ------------------------------------
+    if not args.no_e2e and rank == 0:
+        line["e2e"] = run_e2e(args, ctx, sc, wl, w, sizes, W, schemes, codes, seg_t, res, n, dev)
+    elif rank == 0:
+        line["e2e"] = None
+
+    # ---- CPU oracle on a bounded sample -----------------------------------------------------
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        line["cpu_baseline"] = run_cpu_baseline(args, wl, w, sizes, schemes, num, den, grads[0])
+
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+def run_e2e(args, ctx, sc, wl, w, sizes, W, schemes, codes, seg_t, res, n, dev):
+    import psutil
+    import torch
+    need = 4 * n * (W + 1)
+    if psutil.virtual_memory().available < 2 * need + (8 << 30):
+        return {"value": None, "unit": UNIT, "note": "not enough host memory for pinned staging"}
+    h_grads = torch.empty(W, n, dtype=torch.float32).pin_memory()
+    h_out = torch.empty(n, dtype=torch.float32).pin_memory()
+    for ww in range(W):
+        h_grads[ww].copy_(wl.generate(w, ww, 7, dev, sizes=sizes))
+    torch.cuda.synchronize()
+    steps = max(1, args.e2e_steps)
+
+    def one(t):
+        for s, code in zip(schemes, codes):
+            ctx.sc_step_host(code, h_grads, res[s], seg_t, [wl.step_seed(w.base_seed, 1000 + t)] * W, h_out)
+
+    one(0)                                                # warm-up (allocates the device staging)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for t in range(steps):
+        one(1 + t)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    status = ctx.sc_sync_status()
+    if status != 0:
+        raise RuntimeError(f"device status after the end-to-end run: {sc.strerror(status)}")
+    return {"value": W * n * len(schemes) * steps / dt, "unit": UNIT, "steps": steps,
+            "ms_per_step": 1e3 * dt / steps,
+            "h2d_bytes_per_step": 4 * n * W * len(schemes), "d2h_bytes_per_step": 4 * n * len(schemes),
+            "note": "sc_step_host: pinned host gradients copied per worker, overlapped with compression; "
+                    "dense average copied back"}
+
+
+def run_cpu_baseline(args, wl, w, sizes, schemes, num, den, grads0):
+    import numpy as np
+    from oracle import sparsify_oracle as O
+    n_full = sum(sizes)
+    if len(sizes) == 1 and n_full > 50_000_000:
+        sizes_s = [n_full // args.cpu_sample_div]
+    else:
+        sizes_s = sizes
+    n = sum(sizes_s)
+    segs = [(s.offset, s.n, s.k) for s in wl.segment_table(sizes_s, num, den)]
+    g = grads0[0, :n].cpu().numpy()
+    e = np.zeros(n, np.float32)
+    t0 = time.perf_counter()
+    for s in schemes:
+        v, i, _ = O.compress_segments(O.SCHEMES[s], g, e, segs, wl.step_seed(w.base_seed, 0))
+        O.aggregate([v], [i], n)
+    dt = time.perf_counter() - t0
+    return {"value": n * len(schemes) / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 2),
+            "sample": f"worker 0, first {n} of {n_full} elements, schemes {','.join(schemes)}, density {num}/{den}, "
+                      f"compress + aggregate of that one message"}
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world == 1 and args.gpus > 1:
+        sys.stderr.write("bench.py: --gpus > 1 expects to be launched by torch.distributed.run; running 1 GPU\n")
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -72,6 +72,17 @@ int sc_sync_status(sc_ctx* ctx, void* stream);
 size_t sc_scratch_bytes(const sc_ctx* ctx);
 uint64_t sc_launch_count(const sc_ctx* ctx);
 
+/* Instrumentation (no counterpart in the paper).  sc_profile(ctx, 1) makes every
+ * later kernel launch of this context be bracketed by two CUDA events on the
+ * launching stream and forgets earlier records; sc_profile(ctx, 0) stops it.
+ * sc_profile_read waits for the recorded launches and fills, for each of
+ * sc_profile_kinds() kernel kinds (named by sc_profile_name), the summed device
+ * time in milliseconds and the number of launches (HOST arrays of that length). */
+int sc_profile(sc_ctx* ctx, int enable);
+int sc_profile_kinds(void);
+const char* sc_profile_name(int kind);
+int sc_profile_read(sc_ctx* ctx, double* h_ms, uint64_t* h_launches);
+
 /* Algorithm 1, accumulate + compress + residual lines, one worker, global scope.
  * grad[n] read-only; residual[n] in/out (reads e, writes e'); out_vals[k],
  * out_idx[k] written.  k == 0 is allowed (residual <- g + e). */

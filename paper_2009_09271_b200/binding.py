@@ -19,6 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsparsecomm.so")
 
 EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_scratch_bytes", "sc_launch_count",
+           "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
            "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_step", "sc_step_host"]
 
 
@@ -57,6 +58,14 @@ def load_library() -> ctypes.CDLL:
     lib.sc_scratch_bytes.restype = sz
     lib.sc_launch_count.argtypes = [vp]
     lib.sc_launch_count.restype = u64
+    lib.sc_profile.argtypes = [vp, ci]
+    lib.sc_profile.restype = ci
+    lib.sc_profile_kinds.argtypes = []
+    lib.sc_profile_kinds.restype = ci
+    lib.sc_profile_name.argtypes = [ci]
+    lib.sc_profile_name.restype = ctypes.c_char_p
+    lib.sc_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(u64)]
+    lib.sc_profile_read.restype = ci
     lib.sc_compress.argtypes = [vp, ci, vp, vp, sz, sz, u64, vp, vp, vp]
     lib.sc_compress.restype = ci
     lib.sc_compress_batch.argtypes = [vp, ci, ci, vp, vp, sz, ctypes.POINTER(ScSegment), ci,
@@ -143,6 +152,17 @@ class Context:
     @property
     def launch_count(self) -> int:
         return self._lib.sc_launch_count(self._h)
+
+    def sc_profile(self, enable: bool) -> None:
+        _check(self._lib.sc_profile(self._h, 1 if enable else 0), "sc_profile")
+
+    def sc_profile_read(self) -> dict:
+        """{kernel kind: (milliseconds, launches)} since sc_profile(True)."""
+        kinds = self._lib.sc_profile_kinds()
+        ms = (ctypes.c_double * kinds)()
+        cnt = (ctypes.c_uint64 * kinds)()
+        _check(self._lib.sc_profile_read(self._h, ms, cnt), "sc_profile_read")
+        return {self._lib.sc_profile_name(i).decode(): (ms[i], cnt[i]) for i in range(kinds)}
 
     # -- the C ABI, one method per entry point ---------------------------------
     def sc_sync_status(self, stream=None) -> int:

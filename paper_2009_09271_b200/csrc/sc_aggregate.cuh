@@ -34,43 +34,79 @@ agg_bounds_kernel(const uint32_t* __restrict__ idx, uint32_t rows, uint32_t K, u
     bounds[gid] = lo;
 }
 
-// rows_idx: number of coordinate rows (W, or 1 when all workers share them).
+constexpr uint32_t AGG_STAGE = 2048;     // message entries staged in shared memory per round
+
+// One CTA per tile of ATILE coordinates.  The slices of all W messages that fall into the
+// tile are first fetched together into shared memory (one wave of independent loads), then
+// applied to the accumulator worker by worker, so the per-coordinate sum runs in worker
+// order without one global-memory round trip per worker.  With shared coordinates every
+// slot j carries W values, summed in registers in worker order.
 __global__ void __launch_bounds__(THREADS)
 agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
                  const uint32_t* __restrict__ bounds, uint32_t W, uint32_t shared_idx, uint32_t K,
                  uint32_t n, uint32_t ntiles, float* __restrict__ out, int* __restrict__ status) {
     __shared__ __align__(16) float acc[ATILE];
-    __shared__ uint32_t s_lo[64], s_hi[64];
-    __shared__ uint32_t s_any;
+    __shared__ uint32_t st_loc[AGG_STAGE];
+    __shared__ float st_val[AGG_STAGE];
+    __shared__ uint32_t s_lo[64], s_off[65];
     const float fW = (float)W;
     for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
         const uint32_t tile_lo = t * ATILE;
         const uint32_t tile_n = min(ATILE, n - tile_lo);
         for (uint32_t i = threadIdx.x; i < ATILE; i += THREADS) acc[i] = 0.0f;
-        if (threadIdx.x == 0) s_any = 0;
-        __syncthreads();
-        for (uint32_t w0 = 0; w0 < W; w0 += 64) {
-            const uint32_t wn = min(64u, W - w0);
-            if (threadIdx.x < wn) {
-                const uint32_t r = shared_idx ? 0u : (w0 + threadIdx.x);
-                const uint32_t* b = bounds + (size_t)r * (ntiles + 1) + t;
-                const uint32_t lo = b[0], hi = b[1];
-                s_lo[threadIdx.x] = lo; s_hi[threadIdx.x] = hi;
-                if (hi > lo) s_any = 1;
+        if (shared_idx) {
+            const uint32_t lo = bounds[t], hi = bounds[t + 1];
+            __syncthreads();
+            for (uint32_t j = lo + threadIdx.x; j < hi; j += THREADS) {
+                const uint32_t loc = idx[j] - tile_lo;
+                float sum = 0.0f;
+                for (uint32_t w = 0; w < W; ++w) sum = sum + vals[(size_t)w * K + j];
+                if (loc < tile_n) acc[loc] = sum;
+                else atomicMin(status, ST_DEVICE_CHECK);
             }
             __syncthreads();
-            if (s_any) {
-                for (uint32_t ww = 0; ww < wn; ++ww) {
-                    const uint32_t w = w0 + ww;
-                    const uint32_t lo = s_lo[ww], hi = s_hi[ww];
-                    const float* v = vals + (size_t)w * K;
-                    const uint32_t* ix = idx + (shared_idx ? 0 : (size_t)w * K);
-                    for (uint32_t j = lo + threadIdx.x; j < hi; j += THREADS) {
-                        const uint32_t loc = ix[j] - tile_lo;
-                        if (loc < tile_n) acc[loc] = acc[loc] + v[j];
-                        else atomicMin(status, ST_DEVICE_CHECK);
+        } else {
+            for (uint32_t w0 = 0; w0 < W; w0 += 64) {
+                const uint32_t wn = min(64u, W - w0);
+                __syncthreads();
+                if (threadIdx.x < wn) {
+                    const uint32_t* b = bounds + (size_t)(w0 + threadIdx.x) * (ntiles + 1) + t;
+                    const uint32_t lo = b[0], hi = b[1];
+                    s_lo[threadIdx.x] = lo;
+                    s_off[threadIdx.x + 1] = hi - lo;
+                }
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    uint32_t run = 0;
+                    s_off[0] = 0;
+                    for (uint32_t i = 0; i < wn; ++i) { run += s_off[i + 1]; s_off[i + 1] = run; }
+                }
+                __syncthreads();
+                const uint32_t total = s_off[wn];
+                for (uint32_t cs = 0; cs < total; cs += AGG_STAGE) {
+                    const uint32_t ce = min(total, cs + AGG_STAGE);
+                    for (uint32_t q = cs + threadIdx.x; q < ce; q += THREADS) {
+                        uint32_t lo = 0, hi = wn;               // last i with s_off[i] <= q
+                        while (hi - lo > 1) {
+                            const uint32_t mid = (lo + hi) >> 1;
+                            if (s_off[mid] <= q) lo = mid; else hi = mid;
+                        }
+                        const size_t j = (size_t)(w0 + lo) * K + s_lo[lo] + (q - s_off[lo]);
+                        st_loc[q - cs] = idx[j] - tile_lo;
+                        st_val[q - cs] = vals[j];
                     }
                     __syncthreads();
+                    for (uint32_t i = 0; i < wn; ++i) {
+                        const uint32_t a = max(s_off[i], cs), b = min(s_off[i + 1], ce);
+                        if (a < b) {                             // uniform over the CTA
+                            for (uint32_t q = a + threadIdx.x; q < b; q += THREADS) {
+                                const uint32_t loc = st_loc[q - cs];
+                                if (loc < tile_n) acc[loc] = acc[loc] + st_val[q - cs];
+                                else atomicMin(status, ST_DEVICE_CHECK);
+                            }
+                            __syncthreads();
+                        }
+                    }
                 }
             }
             __syncthreads();

@@ -32,6 +32,7 @@ struct sc_ctx {
     unsigned long long* d_ticket = nullptr;
     uint32_t* d_mask = nullptr;
     uint32_t* d_bounds = nullptr;
+    uint32_t* d_offsets = nullptr;   // per seed group: exclusive kept-count prefix over tiles
     uint64_t* d_seeds = nullptr;
     int* d_status = nullptr;
 
@@ -45,6 +46,12 @@ struct sc_ctx {
     uint64_t launches = 0;
 
     int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1;
+
+    // optional per-kernel timing (sc_profile)
+    bool prof_on = false;
+    struct ProfRec { int kind; cudaEvent_t a, b; };
+    std::vector<ProfRec> prof_recs;
+    std::vector<cudaEvent_t> prof_free;
 
     // host-buffer entry point
     float* d_stage_grads = nullptr;
@@ -84,13 +91,47 @@ class DeviceGuard {
     bool set_ = false;
 };
 
+enum { KIND_HIST0 = 0, KIND_RESOLVE, KIND_REFINE, KIND_PACK_TOPK, KIND_SCATTER, KIND_MASK_COUNT, KIND_ROW_SCAN,
+       KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES, KIND_COUNT };
+const char* const kKindNames[KIND_COUNT] = {"topk_hist0", "topk_resolve", "topk_refine", "pack_topk", "randk_scatter",
+                                            "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
+                                            "agg_tiles"};
+
+// Counts a kernel launch and, when profiling is on, brackets it with two events.
+class Launch {
+  public:
+    Launch(sc_ctx* c, int kind, cudaStream_t st) : c_(c), st_(st) {
+        ++c->launches;
+        if (!c->prof_on) return;
+        rec_.kind = kind;
+        rec_.a = take(); rec_.b = take();
+        if (rec_.a && rec_.b) { cudaEventRecord(rec_.a, st_); on_ = true; }
+    }
+    ~Launch() {
+        if (!on_) return;
+        cudaEventRecord(rec_.b, st_);
+        c_->prof_recs.push_back(rec_);
+    }
+  private:
+    cudaEvent_t take() {
+        if (!c_->prof_free.empty()) { cudaEvent_t e = c_->prof_free.back(); c_->prof_free.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+        return e;
+    }
+    sc_ctx* c_;
+    cudaStream_t st_;
+    sc_ctx::ProfRec rec_{};
+    bool on_ = false;
+};
+
 // Validates the segment table and (re)builds the device copy when it changed.
 int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaStream_t stream) {
     if (c->layout_valid && c->cached_n == n && (int)c->cached_segs.size() == nseg &&
         std::memcmp(c->cached_segs.data(), segs, sizeof(sc_segment) * nseg) == 0)
         return SC_OK;
     std::vector<SegEntry> h(nseg + 1);
-    uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0;
+    uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0;
     for (int s = 0; s < nseg; ++s) {
         const sc_segment& g = segs[s];
         if (g.offset < end_prev || g.offset > n || g.n > n - g.offset) return SC_ERR_INVALID;
@@ -99,9 +140,11 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         SegEntry e{};
         e.offset = g.offset; e.n = (uint32_t)g.n; e.k = (uint32_t)g.k;
         e.msg_off = (uint32_t)msg; e.tile_begin = (uint32_t)tiles; e.scat_begin = (uint32_t)scat;
-        e.mask_word_begin = maskw;
+        e.mask_word_begin = maskw; e.grp_begin = (uint32_t)groups;
         h[s] = e;
-        tiles += (g.n + 3 + TILE - 1) / TILE;
+        const uint64_t seg_tiles = (g.n + 3 + TILE - 1) / TILE;
+        tiles += seg_tiles;
+        groups += (seg_tiles + PACK_GROUP - 1) / PACK_GROUP;
         scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
         maskw += (g.n + 31) / 32;
         msg += g.k;
@@ -109,11 +152,11 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
     SegEntry sentinel{};
     sentinel.offset = n; sentinel.msg_off = (uint32_t)msg; sentinel.tile_begin = (uint32_t)tiles;
-    sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw;
+    sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw; sentinel.grp_begin = (uint32_t)groups;
     h[nseg] = sentinel;
     SC_CUDA(cudaMemcpyAsync(c->d_segs, h.data(), sizeof(SegEntry) * (nseg + 1), cudaMemcpyHostToDevice, stream));
     Layout L{};
-    L.segs = c->d_segs; L.nseg = (uint32_t)nseg; L.tiles_per_worker = (uint32_t)tiles;
+    L.segs = c->d_segs; L.nseg = (uint32_t)nseg; L.tiles_per_worker = (uint32_t)tiles; L.groups_per_worker = (uint32_t)groups;
     L.scat_per_group = (uint32_t)scat; L.K_total = (uint32_t)msg; L.n_total = n; L.mask_words_per_group = maskw;
     c->layout = L;
     c->cached_segs.assign(segs, segs + nseg);
@@ -160,59 +203,73 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
 
     if (scheme == SC_TOPK) {
         SC_CUDA(cudaMemsetAsync(c->d_hist, 0, (size_t)P * HIST_WORDS * sizeof(uint32_t), stream));
-        topk_hist0_kernel<true><<<persistent_grid(c, c->occ_hist, items), THREADS, 0, stream>>>(
-            L, grads, residuals, c->d_hist, items);
-        topk_resolve_kernel<0><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status);
-        topk_refine_kernel<1><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
-            L, residuals, c->d_hist, c->d_state, items);
-        topk_resolve_kernel<1><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status);
-        topk_refine_kernel<2><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
-            L, residuals, c->d_hist, c->d_state, items);
-        topk_resolve_kernel<2><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status);
-        c->launches += 6;
+        { Launch l(c, KIND_HIST0, stream);
+          topk_hist0_kernel<true><<<persistent_grid(c, c->occ_hist, items), THREADS, 0, stream>>>(
+              L, grads, residuals, c->d_hist, items); }
+        { Launch l(c, KIND_RESOLVE, stream);
+          topk_resolve_kernel<0><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status); }
+        { Launch l(c, KIND_REFINE, stream);
+          topk_refine_kernel<1><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
+              L, residuals, c->d_hist, c->d_state, items); }
+        { Launch l(c, KIND_RESOLVE, stream);
+          topk_resolve_kernel<1><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status); }
+        { Launch l(c, KIND_REFINE, stream);
+          topk_refine_kernel<2><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
+              L, residuals, c->d_hist, c->d_state, items); }
+        { Launch l(c, KIND_RESOLVE, stream);
+          topk_resolve_kernel<2><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status); }
     } else {
         SC_CUDA(cudaMemcpyAsync(c->d_seeds, h_seeds, sizeof(uint64_t) * W, cudaMemcpyHostToDevice, stream));
     }
 
     if (scheme == SC_RANDBLOCK) {
-        randblock_kernel<<<persistent_grid(c, c->occ_block, items), THREADS, 0, stream>>>(
-            L, grads, residuals, c->d_seeds, out_vals, out_idx, items);
-        c->launches += 1;
+        { Launch l(c, KIND_RANDBLOCK, stream);
+          randblock_kernel<<<persistent_grid(c, c->occ_block, items), THREADS, 0, stream>>>(
+              L, grads, residuals, c->d_seeds, out_vals, out_idx, items); }
         SC_CUDA(cudaGetLastError());
         return SC_OK;
     }
 
-    if (scheme == SC_RANDK && !mask_ready) {
+    if (scheme == SC_RANDK) {
         const uint32_t groups = shared_seeds ? 1u : (uint32_t)W;
-        SC_CUDA(cudaMemsetAsync(c->d_mask, 0, (size_t)groups * L.mask_words_per_group * sizeof(uint32_t), stream));
-        const uint64_t blocks = (uint64_t)groups * L.scat_per_group;
-        if (blocks > 0x7FFFFFFFull) return SC_ERR_RANGE;
-        if (blocks > 0) {
-            randk_scatter_kernel<<<(uint32_t)blocks, THREADS, 0, stream>>>(L, c->d_seeds, c->d_mask, c->d_status);
-            c->launches += 1;
+        if (!mask_ready) {
+            SC_CUDA(cudaMemsetAsync(c->d_mask, 0, (size_t)groups * L.mask_words_per_group * sizeof(uint32_t), stream));
+            const uint64_t blocks = (uint64_t)groups * L.scat_per_group;
+            if (blocks > 0x7FFFFFFFull) return SC_ERR_RANGE;
+            if (blocks > 0) {
+                Launch l(c, KIND_SCATTER, stream);
+                randk_scatter_kernel<<<(uint32_t)blocks, THREADS, 0, stream>>>(L, c->d_seeds, c->d_mask, c->d_status);
+            }
+            const uint64_t warps = (uint64_t)groups * L.tiles_per_worker;
+            { Launch l(c, KIND_MASK_COUNT, stream);
+              mask_count_kernel<<<(uint32_t)((warps + WARPS - 1) / WARPS), THREADS, 0, stream>>>(
+                  L, c->d_mask, groups, c->d_offsets); }
+            { Launch l(c, KIND_ROW_SCAN, stream);
+              row_scan_kernel<<<groups, THREADS, 0, stream>>>(c->d_offsets, L.tiles_per_worker); }
         }
+        { Launch l(c, KIND_RANDK_PACK, stream);
+          randk_pack_kernel<<<persistent_grid(c, c->occ_pack_mask, items), THREADS, 0, stream>>>(
+              L, grads, residuals, c->d_mask, c->d_offsets, shared_seeds ? 0u : 1u, out_vals, out_idx, items,
+              c->d_status); }
+        SC_CUDA(cudaGetLastError());
+        return SC_OK;
     }
 
     PackParams pp{};
     pp.L = L; pp.grads = grads; pp.residuals = residuals; pp.out_vals = out_vals; pp.out_idx = out_idx;
-    pp.state = c->d_state; pp.mask = c->d_mask; pp.mask_per_worker = shared_seeds ? 0u : 1u;
+    pp.state = c->d_state; pp.mask = c->d_mask; pp.mask_per_worker = 0u;
     if (++c->epoch >= (1u << 28)) {            // tags wrapped: forget every old word
         SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), stream));
         c->epoch = 1;
     }
-    pp.epoch = c->epoch; pp.total_items = items;
+    const uint32_t gitems = (uint32_t)W * L.groups_per_worker;
+    pp.epoch = c->epoch; pp.total_items = gitems;
     pp.ticket = c->d_ticket; pp.ticket_base = c->ticket_base;
     pp.desc = c->d_desc; pp.status = c->d_status;
-    uint32_t grid;
-    if (scheme == SC_TOPK) {
-        grid = persistent_grid(c, c->occ_pack_topk, items);
-        pack_kernel<PACK_TOPK><<<grid, THREADS, 0, stream>>>(pp);
-    } else {
-        grid = persistent_grid(c, c->occ_pack_mask, items);
-        pack_kernel<PACK_MASK><<<grid, THREADS, 0, stream>>>(pp);
-    }
-    c->ticket_base += (unsigned long long)items + grid;   // every CTA draws exactly one ticket past the end
-    c->launches += 1;
+    const uint32_t grid = persistent_grid(c, c->occ_pack_topk, gitems);
+    { Launch l(c, KIND_PACK_TOPK, stream);
+      pack_kernel<PACK_TOPK><<<grid, THREADS, 0, stream>>>(pp); }
+    c->ticket_base += (unsigned long long)gitems + grid;   // every CTA draws exactly one ticket past the end
     SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
@@ -223,11 +280,12 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
     const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
     const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
     const uint64_t threads = (uint64_t)rows * (ntiles + 1ull);
-    agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
-        idx, rows, (uint32_t)k, ntiles, c->d_bounds);
-    agg_tiles_kernel<<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, stream>>>(
-        vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
-    c->launches += 2;
+    { Launch l(c, KIND_AGG_BOUNDS, stream);
+      agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
+          idx, rows, (uint32_t)k, ntiles, c->d_bounds); }
+    { Launch l(c, KIND_AGG_TILES, stream);
+      agg_tiles_kernel<<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, stream>>>(
+          vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status); }
     SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
@@ -289,6 +347,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_ticket, 1)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_mask, (size_t)max_W * c->max_mask_words)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_bounds, (size_t)max_W * (c->max_atiles + 1))) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_offsets, (size_t)max_W * (c->max_tiles_per_worker + 1))) == SC_OK &&
         (rc = dev_alloc(c, &c->d_seeds, (size_t)max_W)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_status, 1)) == SC_OK) {
         bool ok = cudaMemset(c->d_desc, 0, (size_t)max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long)) == cudaSuccess &&
@@ -301,7 +360,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel<true>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_refine, topk_refine_kernel<1>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_topk, pack_kernel<PACK_TOPK>, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_mask, pack_kernel<PACK_MASK>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_mask, randk_pack_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_block, randblock_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel, THREADS, 0);
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
@@ -315,9 +374,11 @@ void sc_destroy(sc_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
     cudaFree(c->d_segs); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
-    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_seeds); cudaFree(c->d_status);
+    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_seeds); cudaFree(c->d_status);
     cudaFree(c->d_stage_grads); cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); cudaFree(c->d_stage_out);
     for (cudaEvent_t e : c->ev_worker) cudaEventDestroy(e);
+    for (auto& r : c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (cudaEvent_t e : c->prof_free) cudaEventDestroy(e);
     if (c->ev_start) cudaEventDestroy(c->ev_start);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     delete c;
@@ -336,6 +397,32 @@ int sc_sync_status(sc_ctx* c, void* stream) {
         SC_CUDA(cudaStreamSynchronize(st));
     }
     return h;
+}
+
+int sc_profile(sc_ctx* c, int enable) {
+    if (!c) return SC_ERR_INVALID;
+    for (auto& r : c->prof_recs) { c->prof_free.push_back(r.a); c->prof_free.push_back(r.b); }
+    c->prof_recs.clear();
+    c->prof_on = enable != 0;
+    return SC_OK;
+}
+
+int sc_profile_kinds(void) { return KIND_COUNT; }
+
+const char* sc_profile_name(int kind) { return (kind >= 0 && kind < KIND_COUNT) ? kKindNames[kind] : "?"; }
+
+int sc_profile_read(sc_ctx* c, double* ms, uint64_t* launches) {
+    if (!c || !ms || !launches) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    for (int k = 0; k < KIND_COUNT; ++k) { ms[k] = 0.0; launches[k] = 0; }
+    for (auto& r : c->prof_recs) {
+        SC_CUDA(cudaEventSynchronize(r.b));
+        float t = 0.f;
+        SC_CUDA(cudaEventElapsedTime(&t, r.a, r.b));
+        ms[r.kind] += t;
+        launches[r.kind] += 1;
+    }
+    return SC_OK;
 }
 
 size_t sc_scratch_bytes(const sc_ctx* c) { return c ? c->scratch_bytes : 0; }

@@ -9,6 +9,7 @@ constexpr int THREADS = 256;            // threads per CTA in every tile kernel
 constexpr int QUADS = 4;                // float4 per thread per tile
 constexpr int TILE = THREADS * QUADS * 4;   // 4096 elements = 16 KB per operand per tile
 constexpr int WARPS = THREADS / 32;
+constexpr int PACK_GROUP = 8;           // tiles handled per chained-scan step of the pack kernel
 
 constexpr uint32_t HIST0_BINS = 2048;   // key bits 30..20
 constexpr uint32_t HIST1_BINS = 1024;   // key bits 19..10
@@ -27,13 +28,14 @@ struct SegEntry {
     uint32_t msg_off;         // K_s: first message slot of the segment
     uint32_t tile_begin;      // first tile of the segment inside a worker
     uint32_t scat_begin;      // first scatter chunk of the segment inside a seed group
-    uint32_t pad;
+    uint32_t grp_begin;       // first pack group (PACK_GROUP tiles) of the segment inside a worker
 };
 
 struct Layout {
     const SegEntry* segs;     // device array, nseg + 1 entries (last = sentinel with the totals)
     uint32_t nseg;
     uint32_t tiles_per_worker;
+    uint32_t groups_per_worker;
     uint32_t scat_per_group;
     uint32_t K_total;         // message entries per worker
     uint64_t n_total;         // elements per worker row
@@ -119,6 +121,14 @@ __device__ inline uint32_t find_by_tile(const Layout& L, uint32_t lt) {
     }
     return lo;
 }
+__device__ inline uint32_t find_by_group(const Layout& L, uint32_t lg) {
+    uint32_t lo = 0, hi = L.nseg;
+    while (hi - lo > 1) {
+        uint32_t mid = (lo + hi) >> 1;
+        if (L.segs[mid].grp_begin <= lg) lo = mid; else hi = mid;
+    }
+    return lo;
+}
 __device__ inline uint32_t find_by_scat(const Layout& L, uint32_t ls) {
     uint32_t lo = 0, hi = L.nseg;
     while (hi - lo > 1) {
@@ -131,7 +141,7 @@ __device__ inline uint32_t find_by_scat(const Layout& L, uint32_t ls) {
 // A quad is four consecutive elements starting at segment-local element `base`
 // (which may be negative or reach past n for the ragged first/last quad).  The
 // address seg + base is 16-byte aligned by construction.
-__device__ inline uint32_t load_quad(const float* __restrict__ seg, long long base, uint32_t n, float v[4]) {
+__device__ inline uint32_t load_quad(const float* seg, long long base, uint32_t n, float v[4]) {
     if (base >= 0 && base + 3 < (long long)n) {
         float4 q = *reinterpret_cast<const float4*>(seg + base);
         v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
@@ -145,7 +155,7 @@ __device__ inline uint32_t load_quad(const float* __restrict__ seg, long long ba
     }
     return m;
 }
-__device__ inline uint32_t load_quad_stream(const float* __restrict__ seg, long long base, uint32_t n, float v[4]) {
+__device__ inline uint32_t load_quad_stream(const float* seg, long long base, uint32_t n, float v[4]) {
     if (base >= 0 && base + 3 < (long long)n) {
         float4 q = __ldcs(reinterpret_cast<const float4*>(seg + base));
         v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
@@ -159,7 +169,7 @@ __device__ inline uint32_t load_quad_stream(const float* __restrict__ seg, long 
     }
     return m;
 }
-__device__ inline void store_quad(float* __restrict__ seg, long long base, uint32_t valid, const float v[4]) {
+__device__ inline void store_quad(float* seg, long long base, uint32_t valid, const float v[4]) {
     if (valid == 0xFu) {
         *reinterpret_cast<float4*>(seg + base) = make_float4(v[0], v[1], v[2], v[3]);
         return;

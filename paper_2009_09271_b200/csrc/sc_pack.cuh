@@ -1,16 +1,23 @@
 // Stream-compaction pack + residual writeback (Algorithm 1: q^w = C(p), e' = p - q^w).
 //
-// One persistent kernel walks all (worker, segment, tile) items in order, handing
-// out tiles through an atomic ticket so that every tile's predecessors are already
-// owned by running CTAs.  Inside a tile the rank of each kept element comes from
-// warp ballots and population counts; across tiles from a single-pass chained scan
-// (each tile publishes its count, then looks back over its predecessors' words).
-// Every wait on a predecessor is bounded; when it runs out the kernel records
-// ST_TIMEOUT in the status word and carries on with a zero prefix.
+// One persistent kernel walks all (worker, segment, tile group) items in order, handing
+// out groups of PACK_GROUP tiles through an atomic ticket so that every group's
+// predecessors are already owned by running CTAs.
+//   phase 1  streams the group's tiles: forms or reads p, classifies every element, keeps
+//            only the 4-bit "kept" masks per quad (shared memory) and the per-warp counts;
+//   scan     block scan of the counts, then ONE chained-scan look-back per group (each
+//            group publishes its count, then sums its predecessors' words);
+//   phase 2  re-reads only the quads that hold kept elements (they are still in L2),
+//            writes values and coordinates at their ranks and zeroes them in the residual.
+// Grouping matters because a chained scan advances by at most 32 descriptors per L2 round
+// trip: with single 16 KB tiles that caps the pass near 1 TB/s, far below HBM.
+// Every wait on a predecessor is bounded; when it runs out the kernel records ST_TIMEOUT
+// in the status word and carries on with a zero prefix.
 //
-// PACK_TOPK: p is read from the residual buffer (parked there by the histogram
-//            pass); kept = key > T, plus the first r coordinates with key == T.
-// PACK_MASK: p = g + e is formed here; kept = membership bit of the coordinate.
+// PACK_TOPK: p is read from the residual buffer (parked there by the histogram pass);
+//            kept = key > T, plus the first r coordinates with key == T.
+// PACK_MASK: p = g + e is formed here and written to the residual buffer in phase 1;
+//            kept = membership bit of the coordinate.
 #pragma once
 #include "sc_common.cuh"
 
@@ -27,12 +34,12 @@ struct PackParams {
     const TopkState* state;          // PACK_TOPK
     const uint32_t* mask;            // PACK_MASK
     uint32_t mask_per_worker;        // 1: worker w uses mask group w, 0: all use group 0
-    uint32_t epoch;                  // tag of this launch inside the tile words
-    uint32_t total_items;
+    uint32_t epoch;                  // tag of this launch inside the descriptor words
+    uint32_t total_items;            // groups over all workers
     uint32_t pad;
     unsigned long long* ticket;
     unsigned long long ticket_base;
-    unsigned long long* desc;        // two words per item
+    unsigned long long* desc;        // two words per group
     int* status;
 };
 
@@ -59,7 +66,11 @@ __device__ inline uint32_t warp_sum(uint32_t v) {
 }
 
 // Chained-scan look-back executed by warp 0.  Returns the exclusive prefixes of
-// the two counters over tiles [first, item) of the same problem.
+// the two counters over items [first, item) of the same problem.  Each round
+// inspects 32 * LB_DEPTH predecessors (LB_DEPTH consecutive words per lane), so
+// the scan front moves that many groups per L2 round trip.
+constexpr int LB_DEPTH = 4;
+
 __device__ inline void lookback(const PackParams& P, uint32_t item, uint32_t first, bool dual,
                                 uint32_t& ex0, uint32_t& ex1) {
     const uint32_t lane = threadIdx.x & 31u;
@@ -68,19 +79,23 @@ __device__ inline void lookback(const PackParams& P, uint32_t item, uint32_t fir
     uint32_t polls = 0;
     bool done = false;
     while (!done) {
-        const long long my = pos - lane;
-        const bool inrange = my >= (long long)first;
-        unsigned long long w0 = 0, w1 = 0;
-        uint32_t st = 0;
+        const long long mine = pos - (long long)lane * LB_DEPTH;      // nearest of this lane's words
+        unsigned long long w0[LB_DEPTH], w1[LB_DEPTH];
+        uint32_t st[LB_DEPTH];
         while (true) {
             bool ready = true;
-            if (inrange) {
-                w0 = desc_load(P.desc + 2 * my);
-                st = desc_status(w0, P.epoch);
-                ready = st != 0;
-                if (dual) {
-                    w1 = desc_load(P.desc + 2 * my + 1);
-                    ready = ready && desc_status(w1, P.epoch) == st;
+#pragma unroll
+            for (int d = 0; d < LB_DEPTH; ++d) {
+                const long long at = mine - d;
+                st[d] = DESC_INC; w0[d] = 0; w1[d] = 0;               // out of range counts as "done, zero"
+                if (at >= (long long)first) {
+                    w0[d] = desc_load(P.desc + 2 * at);
+                    st[d] = desc_status(w0[d], P.epoch);
+                    if (dual) {
+                        w1[d] = desc_load(P.desc + 2 * at + 1);
+                        if (desc_status(w1[d], P.epoch) != st[d]) st[d] = 0;
+                    }
+                    ready = ready && st[d] != 0;
                 }
             }
             if (__all_sync(0xFFFFFFFFu, ready)) break;
@@ -89,29 +104,51 @@ __device__ inline void lookback(const PackParams& P, uint32_t item, uint32_t fir
                 ex0 = 0; ex1 = 0;
                 return;
             }
-            __nanosleep(40);
+            __nanosleep(20);
         }
-        const uint32_t inc_mask = __ballot_sync(0xFFFFFFFFu, inrange && st == DESC_INC);
+        // sum this lane's words up to and including its first inclusive one
+        uint32_t s0 = 0, s1 = 0;
+        bool found = false;
+#pragma unroll
+        for (int d = 0; d < LB_DEPTH; ++d) {
+            if (!found) {
+                s0 += (uint32_t)(w0[d] & DESC_VAL_MASK);
+                s1 += (uint32_t)(w1[d] & DESC_VAL_MASK);
+                found = st[d] == DESC_INC;
+            }
+        }
+        const uint32_t inc_mask = __ballot_sync(0xFFFFFFFFu, found);
         const uint32_t upto = inc_mask ? (uint32_t)(__ffs((int)inc_mask) - 1) : 31u;
-        const bool use = inrange && lane <= upto;
-        acc0 += warp_sum(use ? (uint32_t)(w0 & DESC_VAL_MASK) : 0u);
-        if (dual) acc1 += warp_sum(use ? (uint32_t)(w1 & DESC_VAL_MASK) : 0u);
-        if (inc_mask) done = true; else pos -= 32;
+        acc0 += warp_sum(lane <= upto ? s0 : 0u);
+        if (dual) acc1 += warp_sum(lane <= upto ? s1 : 0u);
+        if (inc_mask) done = true; else pos -= 32 * LB_DEPTH;
     }
     ex0 = (uint32_t)acc0;
     ex1 = (uint32_t)acc1;
 }
 
+// Element-to-thread mapping inside a tile: thread t owns the 16 consecutive elements
+// [16 t, 16 t + 16) (four float4 loads of one 64-byte run), so that the rank of a kept
+// element is (kept in lower lanes, one warp scan per tile) + (kept bits below it in the
+// thread's own 16-bit mask).
 template <int MODE>
 __global__ void __launch_bounds__(THREADS)
 pack_kernel(PackParams P) {
-    static_assert(QUADS * WARPS == 32, "one warp scans the per-(quad, warp) counts");
-    __shared__ uint32_t s_dec[4];
-    __shared__ uint32_t s_cnt[2][32];
-    __shared__ uint32_t s_excl[2][32];
-    __shared__ uint32_t s_tile_excl[2];
+    constexpr int G = PACK_GROUP;
+    constexpr int NCNT = G * WARPS;                // one count per (tile, warp)
+    constexpr int EPL = NCNT / 32;                 // count entries per lane in the warp scan
+    constexpr int BATCH = 4;                       // quads re-read together in phase 2
+    constexpr int EPT = QUADS * 4;                 // elements per thread per tile
+    static_assert(NCNT % 32 == 0 && G * QUADS <= 32 && EPT == 16, "table layout");
+    constexpr bool TOPK = MODE == PACK_TOPK;
+    __shared__ uint32_t s_dec[5];
+    __shared__ uint16_t s_abits[G][THREADS];                   // kept / above-threshold bits of 16 elements
+    __shared__ uint16_t s_tbits[TOPK ? G : 1][THREADS];        // tie bits
+    __shared__ uint16_t s_arank[G][THREADS];                   // kept elements in lower lanes, same tile
+    __shared__ uint16_t s_trank[TOPK ? G : 1][THREADS];
+    __shared__ uint32_t s_cnt[2][NCNT];
+    __shared__ uint32_t s_grp_excl[2];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const uint32_t lt_mask = (1u << lane) - 1u;
     const Layout& L = P.L;
 
     while (true) {
@@ -120,112 +157,173 @@ pack_kernel(PackParams P) {
             uint32_t item = tk < (unsigned long long)P.total_items ? (uint32_t)tk : 0xFFFFFFFFu;
             s_dec[0] = item;
             if (item != 0xFFFFFFFFu) {
-                uint32_t w = item / L.tiles_per_worker;
-                uint32_t lt = item - w * L.tiles_per_worker;
-                uint32_t s = find_by_tile(L, lt);
-                s_dec[1] = w; s_dec[2] = s; s_dec[3] = lt - L.segs[s].tile_begin;
+                uint32_t w = item / L.groups_per_worker;
+                uint32_t lg = item - w * L.groups_per_worker;
+                uint32_t s = find_by_group(L, lg);
+                const SegEntry sg = L.segs[s];
+                uint32_t gi = lg - sg.grp_begin;                              // group inside the segment
+                uint32_t ntiles = L.segs[s + 1].tile_begin - sg.tile_begin;
+                s_dec[1] = w; s_dec[2] = s; s_dec[3] = gi;
+                s_dec[4] = min((uint32_t)G, ntiles - gi * G);
             }
         }
         __syncthreads();
         const uint32_t item = s_dec[0];
         if (item == 0xFFFFFFFFu) break;
-        const uint32_t w = s_dec[1], s = s_dec[2], t = s_dec[3];
+        const uint32_t w = s_dec[1], s = s_dec[2], gi = s_dec[3], ntl = s_dec[4];
         const SegEntry seg = L.segs[s];
         const size_t row = (size_t)w * L.n_total + seg.offset;
         float* e = P.residuals + row;
+        const float* g = P.grads + row;
         const uint32_t mis = misalign_of(e);
+        const long long t0 = (long long)gi * G;
 
         uint32_t T = 0, r = 0;
         bool dual = false;
         const uint32_t* mask = nullptr;
-        if (MODE == PACK_TOPK) {
+        if (TOPK) {
             const TopkState st = P.state[(size_t)w * L.nseg + s];
             T = st.T; r = st.r; dual = st.dual != 0;
         } else {
             mask = P.mask + (P.mask_per_worker ? (size_t)w * L.mask_words_per_group : 0) + seg.mask_word_begin;
         }
 
-        float p[QUADS][4];
-        uint32_t valid[QUADS], abits[QUADS], tbits[QUADS];
-        uint32_t arank[QUADS], trank[QUADS];
+        // ---- phase 1: stream, classify, rank inside the warp, count -------------------------
+        uint32_t pend = 0;                       // bit gl*QUADS+j: this thread's quad holds a candidate
+#pragma unroll 2
+        for (uint32_t gl = 0; gl < (uint32_t)G; ++gl) {
+            uint32_t ab16 = 0, tb16 = 0;
+            if (gl < ntl) {
+                const long long first = (t0 + gl) * TILE - mis;          // local index of the tile's first element
+                const long long mine = first + (long long)threadIdx.x * EPT;
+                if (first >= 0 && first + TILE <= (long long)seg.n) {   // whole tile inside the segment
+                    float4 q[QUADS];
+                    const float4* pe = reinterpret_cast<const float4*>(e + mine);
 #pragma unroll
-        for (int j = 0; j < QUADS; ++j) {
-            const long long base = (long long)t * TILE + (long long)(j * THREADS + threadIdx.x) * 4 - mis;
-            valid[j] = load_quad(e, base, seg.n, p[j]);
-            abits[j] = 0; tbits[j] = 0;
-            if (MODE == PACK_MASK) {
-                float gv[4];
-                load_quad_stream(P.grads + row, base, seg.n, gv);
+                    for (int j = 0; j < QUADS; ++j) q[j] = pe[j];
+                    if (!TOPK) {
+                        const float4* pg = reinterpret_cast<const float4*>(g + mine);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) p[j][c] = gv[c] + p[j][c];
-                if (valid[j] == 0xFu) {
-                    const uint32_t a = (uint32_t)(base >> 5), b = (uint32_t)((base + 3) >> 5);
-                    const uint32_t lo = __ldg(mask + a);
-                    const uint32_t hi = (b != a) ? __ldg(mask + b) : lo;
-                    abits[j] = __funnelshift_r(lo, hi, (uint32_t)(base & 31)) & 0xFu;
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if ((valid[j] >> c) & 1u) {
-                            const long long i = base + c;
-                            abits[j] |= ((__ldg(mask + (i >> 5)) >> (uint32_t)(i & 31)) & 1u) << c;
+                        for (int j = 0; j < QUADS; ++j) {
+                            const float4 gv = __ldcs(pg + j);
+                            q[j].x = gv.x + q[j].x; q[j].y = gv.y + q[j].y;
+                            q[j].z = gv.z + q[j].z; q[j].w = gv.w + q[j].w;
                         }
-                }
-            } else {
+                        float4* po = reinterpret_cast<float4*>(e + mine);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t key = key_of(p[j][c]);
-                    const uint32_t v = (valid[j] >> c) & 1u;
-                    if (dual) {
-                        abits[j] |= (v & (uint32_t)(key > T)) << c;
-                        tbits[j] |= (v & (uint32_t)(key == T)) << c;
+                        for (int j = 0; j < QUADS; ++j) po[j] = q[j];
+                        const uint32_t pos = (uint32_t)mine, a = pos >> 5, sh = pos & 31u;
+                        const uint32_t lo = __ldg(mask + a);
+                        const uint32_t hi = (sh > 16u) ? __ldg(mask + a + 1) : lo;
+                        ab16 = __funnelshift_r(lo, hi, sh) & 0xFFFFu;
                     } else {
-                        abits[j] |= (v & (uint32_t)(key >= T)) << c;
+#pragma unroll
+                        for (int j = 0; j < QUADS; ++j) {
+                            const float v[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const uint32_t key = key_of(v[c]);
+                                if (dual) {
+                                    ab16 |= (uint32_t)(key > T) << (4 * j + c);
+                                    tb16 |= (uint32_t)(key == T) << (4 * j + c);
+                                } else {
+                                    ab16 |= (uint32_t)(key >= T) << (4 * j + c);
+                                }
+                            }
+                        }
+                    }
+                } else {                                                   // ragged first / last tile
+#pragma unroll
+                    for (int j = 0; j < QUADS; ++j) {
+                        const long long base = mine + 4 * j;
+                        float p[4];
+                        const uint32_t valid = load_quad(e, base, seg.n, p);
+                        if (!TOPK) {
+                            float gv[4];
+                            load_quad_stream(g, base, seg.n, gv);
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) p[c] = gv[c] + p[c];
+                            if (valid) store_quad(e, base, valid, p);
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                if ((valid >> c) & 1u) {
+                                    const long long i = base + c;
+                                    ab16 |= ((__ldg(mask + (i >> 5)) >> (uint32_t)(i & 31)) & 1u) << (4 * j + c);
+                                }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const uint32_t key = key_of(p[c]);
+                                const uint32_t v = (valid >> c) & 1u;
+                                if (dual) {
+                                    ab16 |= (v & (uint32_t)(key > T)) << (4 * j + c);
+                                    tb16 |= (v & (uint32_t)(key == T)) << (4 * j + c);
+                                } else {
+                                    ab16 |= (v & (uint32_t)(key >= T)) << (4 * j + c);
+                                }
+                            }
+                        }
                     }
                 }
-            }
-            // rank of this thread's quad inside the warp's 128 consecutive elements
-            uint32_t below = 0, wtot = 0;
+                const uint32_t any16 = ab16 | tb16;
+                if (any16) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, (abits[j] >> c) & 1u);
-                below += __popc(bal & lt_mask);
-                wtot += __popc(bal);
-            }
-            arank[j] = below;
-            if (lane == 0) s_cnt[0][j * WARPS + warp] = wtot;
-            trank[j] = 0;
-            if (dual) {
-                below = 0; wtot = 0;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, (tbits[j] >> c) & 1u);
-                    below += __popc(bal & lt_mask);
-                    wtot += __popc(bal);
+                    for (int j = 0; j < QUADS; ++j)
+                        if ((any16 >> (4 * j)) & 0xFu) pend |= 1u << (gl * QUADS + j);
                 }
-                trank[j] = below;
-                if (lane == 0) s_cnt[1][j * WARPS + warp] = wtot;
+                uint32_t inc = __popc(ab16);
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                    if (lane >= (uint32_t)d) inc += t;
+                }
+                s_arank[gl][threadIdx.x] = (uint16_t)(inc - __popc(ab16));
+                if (lane == 31u) s_cnt[0][gl * WARPS + warp] = inc;
+                if (TOPK && dual) {
+                    uint32_t tinc = __popc(tb16);
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, tinc, d);
+                        if (lane >= (uint32_t)d) tinc += t;
+                    }
+                    s_trank[TOPK ? gl : 0][threadIdx.x] = (uint16_t)(tinc - __popc(tb16));
+                    if (lane == 31u) s_cnt[1][gl * WARPS + warp] = tinc;
+                }
+            } else if (lane == 0) {
+                s_cnt[0][gl * WARPS + warp] = 0;
+                s_cnt[1][gl * WARPS + warp] = 0;
             }
+            s_abits[gl][threadIdx.x] = (uint16_t)ab16;
+            if (TOPK) s_tbits[gl][threadIdx.x] = (uint16_t)tb16;
         }
         __syncthreads();
 
+        // ---- scan of the per-(tile, warp) counts + one look-back for the group (warp 0) -------
         if (warp == 0) {
-            const uint32_t v0 = s_cnt[0][lane];
-            const uint32_t v1 = dual ? s_cnt[1][lane] : 0u;
-            uint32_t i0 = v0, i1 = v1;
+            uint32_t v0[EPL], v1[EPL], sum0 = 0, sum1 = 0;
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) {
+                v0[i] = s_cnt[0][lane * EPL + i];
+                v1[i] = dual ? s_cnt[1][lane * EPL + i] : 0u;
+                sum0 += v0[i]; sum1 += v1[i];
+            }
+            uint32_t i0 = sum0, i1 = sum1;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                uint32_t a = __shfl_up_sync(0xFFFFFFFFu, i0, d);
-                uint32_t b = __shfl_up_sync(0xFFFFFFFFu, i1, d);
+                const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, i0, d);
+                const uint32_t b = __shfl_up_sync(0xFFFFFFFFu, i1, d);
                 if (lane >= (uint32_t)d) { i0 += a; i1 += b; }
             }
-            s_excl[0][lane] = i0 - v0;
-            s_excl[1][lane] = i1 - v1;
-            const uint32_t tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31);
-            const uint32_t tot1 = __shfl_sync(0xFFFFFFFFu, i1, 31);
+            const uint32_t tot0 = __shfl_sync(0xFFFFFFFFu, i0, 31), tot1 = __shfl_sync(0xFFFFFFFFu, i1, 31);
+            uint32_t ex0 = i0 - sum0, ex1 = i1 - sum1;
+#pragma unroll
+            for (int i = 0; i < EPL; ++i) {
+                s_cnt[0][lane * EPL + i] = ex0; ex0 += v0[i];
+                s_cnt[1][lane * EPL + i] = ex1; ex1 += v1[i];
+            }
             unsigned long long* my = P.desc + 2 * (size_t)item;
-            uint32_t ex0 = 0, ex1 = 0;
-            if (t == 0) {
+            uint32_t gex0 = 0, gex1 = 0;
+            if (gi == 0) {
                 if (lane == 0) {
                     desc_store(my, P.epoch, DESC_INC, tot0);
                     if (dual) desc_store(my + 1, P.epoch, DESC_INC, tot1);
@@ -235,60 +333,78 @@ pack_kernel(PackParams P) {
                     desc_store(my, P.epoch, DESC_AGG, tot0);
                     if (dual) desc_store(my + 1, P.epoch, DESC_AGG, tot1);
                 }
-                lookback(P, item, item - t, dual, ex0, ex1);
+                lookback(P, item, item - gi, dual, gex0, gex1);
                 if (lane == 0) {
-                    desc_store(my, P.epoch, DESC_INC, (unsigned long long)ex0 + tot0);
-                    if (dual) desc_store(my + 1, P.epoch, DESC_INC, (unsigned long long)ex1 + tot1);
+                    desc_store(my, P.epoch, DESC_INC, (unsigned long long)gex0 + tot0);
+                    if (dual) desc_store(my + 1, P.epoch, DESC_INC, (unsigned long long)gex1 + tot1);
                 }
             }
-            if (lane == 0) { s_tile_excl[0] = ex0; s_tile_excl[1] = ex1; }
+            if (lane == 0) { s_grp_excl[0] = gex0; s_grp_excl[1] = gex1; }
         }
         __syncthreads();
 
+        // ---- phase 2: each thread walks its own pending quads, BATCH re-reads in flight -------
         float* ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
         uint32_t* oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
-        const uint32_t tex0 = s_tile_excl[0], tex1 = s_tile_excl[1];
+        const uint32_t gex0 = s_grp_excl[0], gex1 = s_grp_excl[1];
+        const uint32_t idx0 = (uint32_t)seg.offset;
+        while (pend) {
+            int sl[BATCH];
+            float q[BATCH][4];
+            uint32_t valid[BATCH];
+            long long base[BATCH];
 #pragma unroll
-        for (int j = 0; j < QUADS; ++j) {
-            const long long base = (long long)t * TILE + (long long)(j * THREADS + threadIdx.x) * 4 - mis;
-            uint32_t a_before = tex0 + s_excl[0][j * WARPS + warp] + arank[j];
-            uint32_t t_before = dual ? tex1 + s_excl[1][j * WARPS + warp] + trank[j] : 0u;
-            uint32_t kept = 0;
-            if (abits[j] | tbits[j]) {
+            for (int b = 0; b < BATCH; ++b) {
+                sl[b] = pend ? (__ffs((int)pend) - 1) : -1;
+                if (pend) pend &= pend - 1u;
+            }
+#pragma unroll
+            for (int b = 0; b < BATCH; ++b) {
+                valid[b] = 0; base[b] = 0;
+                if (sl[b] >= 0) {
+                    const uint32_t gl = (uint32_t)sl[b] / QUADS, j = (uint32_t)sl[b] % QUADS;
+                    base[b] = (t0 + gl) * TILE - mis + (long long)threadIdx.x * EPT + 4 * j;
+                    valid[b] = load_quad(e, base[b], seg.n, q[b]);
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < BATCH; ++b) {
+                if (sl[b] < 0) continue;
+                const uint32_t gl = (uint32_t)sl[b] / QUADS, j = (uint32_t)sl[b] % QUADS;
+                const uint32_t ab16 = s_abits[gl][threadIdx.x];
+                const uint32_t tb16 = (TOPK && dual) ? s_tbits[gl][threadIdx.x] : 0u;
+                const uint32_t below = (1u << (4 * j)) - 1u;
+                uint32_t a_before = gex0 + s_cnt[0][gl * WARPS + warp] + s_arank[gl][threadIdx.x] + __popc(ab16 & below);
+                uint32_t t_before = 0;
+                if (TOPK && dual)
+                    t_before = gex1 + s_cnt[1][gl * WARPS + warp] + s_trank[TOPK ? gl : 0][threadIdx.x] + __popc(tb16 & below);
+                const uint32_t ab = (ab16 >> (4 * j)) & 0xFu, tb = (tb16 >> (4 * j)) & 0xFu;
+                uint32_t kept = 0;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint32_t ab = (abits[j] >> c) & 1u, tb = (tbits[j] >> c) & 1u;
-                    if (ab | tb) {
+                    const uint32_t abc = (ab >> c) & 1u, tbc = (tb >> c) & 1u;
+                    if (abc | tbc) {
                         uint32_t slot = 0xFFFFFFFFu;
-                        if (ab) slot = a_before + (dual ? min(t_before, r) : 0u);
+                        if (abc) slot = a_before + (dual ? min(t_before, r) : 0u);
                         else if (t_before < r) slot = a_before + t_before;
                         if (slot != 0xFFFFFFFFu) {
                             if (slot < seg.k) {
-                                ovals[slot] = p[j][c];
-                                oidx[slot] = (uint32_t)(seg.offset + (uint64_t)(base + c));
+                                ovals[slot] = q[b][c];
+                                oidx[slot] = idx0 + (uint32_t)(base[b] + c);
                             } else {
                                 atomicMin(P.status, ST_DEVICE_CHECK);
                             }
                             kept |= 1u << c;
+                            q[b][c] = 0.0f;
                         }
-                        a_before += ab;
-                        t_before += tb;
+                        a_before += abc;
+                        t_before += tbc;
                     }
                 }
-            }
-            if (MODE == PACK_MASK) {
-                if (valid[j]) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) if ((kept >> c) & 1u) p[j][c] = 0.0f;
-                    store_quad(e, base, valid[j], p[j]);
-                }
-            } else if (kept) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) if ((kept >> c) & 1u) p[j][c] = 0.0f;
-                store_quad(e, base, valid[j], p[j]);
+                if (kept) store_quad(e, base[b], valid[b], q[b]);
             }
         }
-        __syncthreads();    // s_dec, s_cnt, s_excl are reused by the next tile
+        __syncthreads();    // shared tables are reused by the next group
     }
 }
 
