@@ -125,6 +125,8 @@ def algorithmic_bytes(kind: str, n: int, W: int, K: int, shared: bool) -> float:
         "agg_tiles": 4.0 * n + (4.0 * K * W + 4.0 * K if shared else 8.0 * K * W),
         "agg_bounds": 4.0 * (n / 4096.0) * (1 if shared else W),
         "topk_resolve": 0.0,
+        "topk_main": 12.0 * n * W + 8.0 * K * W,          # read g, e; write e' and the flagged (value, coordinate) list
+        "topk_emit": 16.0 * K * W,                        # read the flagged list, write vals and idx
     }.get(kind, 0.0)
 
 

@@ -83,6 +83,15 @@ int sc_profile_kinds(void);
 const char* sc_profile_name(int kind);
 int sc_profile_read(sc_ctx* ctx, double* h_ms, uint64_t* h_launches);
 
+/* Instrumentation (no counterpart in the paper).  Top-k of a segment of 2^20 or
+ * more elements first tries a one-pass path whose work depends on a sampled
+ * bracket of the threshold; if the exact counts show the bracket missed, it redoes
+ * the selection with a multi-pass radix select.  Both give the same bits.  After
+ * synchronising `stream` this fills h_counts[3] for the most recent top-k call:
+ * (worker, segment) pairs served by [0] the radix select because the segment is
+ * small, [1] the one-pass path, [2] the radix select after a missed bracket. */
+int sc_topk_path_counts(sc_ctx* ctx, void* stream, uint32_t* h_counts);
+
 /* Algorithm 1, accumulate + compress + residual lines, one worker, global scope.
  * grad[n] read-only; residual[n] in/out (reads e, writes e'); out_vals[k],
  * out_idx[k] written.  k == 0 is allowed (residual <- g + e). */

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsparsecomm.so")
 
 EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_scratch_bytes", "sc_launch_count",
-           "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
+           "sc_topk_path_counts", "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
            "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_step", "sc_step_host"]
 
 
@@ -58,6 +58,8 @@ def load_library() -> ctypes.CDLL:
     lib.sc_scratch_bytes.restype = sz
     lib.sc_launch_count.argtypes = [vp]
     lib.sc_launch_count.restype = u64
+    lib.sc_topk_path_counts.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.sc_topk_path_counts.restype = ci
     lib.sc_profile.argtypes = [vp, ci]
     lib.sc_profile.restype = ci
     lib.sc_profile_kinds.argtypes = []
@@ -152,6 +154,12 @@ class Context:
     @property
     def launch_count(self) -> int:
         return self._lib.sc_launch_count(self._h)
+
+    def sc_topk_path_counts(self, stream=None) -> tuple:
+        """(small-segment radix select, one-pass path, radix select after a missed bracket)."""
+        out = (ctypes.c_uint32 * 3)()
+        _check(self._lib.sc_topk_path_counts(self._h, _stream(stream), out), "sc_topk_path_counts")
+        return tuple(out)
 
     def sc_profile(self, enable: bool) -> None:
         _check(self._lib.sc_profile(self._h, 1 if enable else 0), "sc_profile")

@@ -12,6 +12,7 @@
 #include "sc_pack.cuh"
 #include "sc_random.cuh"
 #include "sc_topk.cuh"
+#include "sc_topk_fast.cuh"
 
 using namespace sc;
 
@@ -32,7 +33,28 @@ struct sc_ctx {
     unsigned long long* d_ticket = nullptr;
     uint32_t* d_mask = nullptr;
     uint32_t* d_bounds = nullptr;
-    uint32_t* d_offsets = nullptr;   // per seed group: exclusive kept-count prefix over tiles
+    uint32_t* d_offsets = nullptr;   // per seed group / worker: exclusive kept-count prefix over tiles
+    // sampled-bracket top-k path
+    FastState* d_fstate = nullptr;
+    uint32_t* d_sample = nullptr;
+    uint32_t* d_cand_hist = nullptr;
+    uint2* d_cand = nullptr;
+    uint2* d_list2 = nullptr;
+    uint32_t* d_tile_sure = nullptr;
+    uint32_t* d_tile_cbase = nullptr;
+    uint32_t* d_tile_ccnt = nullptr;
+    uint32_t* d_tile_fbase = nullptr;
+    uint32_t* d_tile_fcnt = nullptr;
+    unsigned long long* d_reserve = nullptr;
+    uint2* d_flagged = nullptr;      // grown on demand: its size depends on k
+    size_t flagged_slots = 0;
+    uint32_t* d_nslow = nullptr;     // [0]: segments for the radix select, [1]: segments whose bracket missed
+    size_t max_fast_per_worker = 0, max_cand_per_worker = 0;
+    uint32_t last_topk_problems = 0; // (worker, segment) pairs of the most recent top-k call
+    uint32_t slow_segments = 0;      // segments of the cached table that take the radix-select path
+    uint32_t max_sample_m = 0;
+    uint32_t max_flag_cap = 0;
+    int occ_main = 1, occ_emit = 1;
     uint64_t* d_seeds = nullptr;
     int* d_status = nullptr;
 
@@ -41,7 +63,6 @@ struct sc_ctx {
     bool layout_valid = false;
     Layout layout{};
 
-    unsigned long long ticket_base = 0;
     uint32_t epoch = 0;
     uint64_t launches = 0;
 
@@ -92,10 +113,12 @@ class DeviceGuard {
 };
 
 enum { KIND_HIST0 = 0, KIND_RESOLVE, KIND_REFINE, KIND_PACK_TOPK, KIND_SCATTER, KIND_MASK_COUNT, KIND_ROW_SCAN,
-       KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES, KIND_COUNT };
+       KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES, KIND_SAMPLE, KIND_BRACKET, KIND_MAIN,
+       KIND_CANDBIN, KIND_CANDFILTER, KIND_FINAL, KIND_TILECOUNT, KIND_EMIT, KIND_RESTORE, KIND_COUNT };
 const char* const kKindNames[KIND_COUNT] = {"topk_hist0", "topk_resolve", "topk_refine", "pack_topk", "randk_scatter",
                                             "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
-                                            "agg_tiles"};
+                                            "agg_tiles", "topk_sample", "topk_bracket", "topk_main", "topk_candbin",
+                                            "topk_candfilter", "topk_final", "topk_tilecount", "topk_emit", "topk_restore"};
 
 // Counts a kernel launch and, when profiling is on, brackets it with two events.
 class Launch {
@@ -131,7 +154,8 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         std::memcmp(c->cached_segs.data(), segs, sizeof(sc_segment) * nseg) == 0)
         return SC_OK;
     std::vector<SegEntry> h(nseg + 1);
-    uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0;
+    uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0, cand = 0, flag = 0;
+    uint32_t fast_count = 0, slow_count = 0, max_m = 0, max_cap = 0;
     for (int s = 0; s < nseg; ++s) {
         const sc_segment& g = segs[s];
         if (g.offset < end_prev || g.offset > n || g.n > n - g.offset) return SC_ERR_INVALID;
@@ -141,6 +165,21 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         e.offset = g.offset; e.n = (uint32_t)g.n; e.k = (uint32_t)g.k;
         e.msg_off = (uint32_t)msg; e.tile_begin = (uint32_t)tiles; e.scat_begin = (uint32_t)scat;
         e.mask_word_begin = maskw; e.grp_begin = (uint32_t)groups;
+        if (g.n >= FAST_MIN_N) {
+            uint64_t m = (g.n / 16) & ~7ull;
+            m = std::min<uint64_t>(std::max<uint64_t>(m, SAMPLE_MIN), SAMPLE_MAX);
+            e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
+            e.cand_cap = (uint32_t)(g.n / 32 + 16384);
+            e.cand_begin = cand;
+            cand += e.cand_cap;
+            e.flag_cap = (uint32_t)std::min<uint64_t>(g.n, g.k + e.cand_cap);
+            e.flag_begin = flag;
+            flag += e.flag_cap;
+            max_cap = std::max(max_cap, e.flag_cap);
+            max_m = std::max(max_m, e.sample_m);
+        } else {
+            ++slow_count;
+        }
         h[s] = e;
         const uint64_t seg_tiles = (g.n + 3 + TILE - 1) / TILE;
         tiles += seg_tiles;
@@ -150,6 +189,17 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         msg += g.k;
     }
     if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
+    if (fast_count > c->max_fast_per_worker || cand > c->max_cand_per_worker) return SC_ERR_RANGE;
+    if ((size_t)c->max_W * flag > c->flagged_slots) {      // the flagged list follows k: grow it (synchronous, rare)
+        SC_CUDA(cudaStreamSynchronize(stream));
+        cudaFree(c->d_flagged); c->d_flagged = nullptr;
+        c->scratch_bytes -= c->flagged_slots * sizeof(uint2);
+        c->flagged_slots = 0;
+        const size_t want = (size_t)c->max_W * flag;
+        if (cudaMalloc(reinterpret_cast<void**>(&c->d_flagged), want * sizeof(uint2)) != cudaSuccess) return SC_ERR_WORKSPACE;
+        c->flagged_slots = want;
+        c->scratch_bytes += want * sizeof(uint2);
+    }
     SegEntry sentinel{};
     sentinel.offset = n; sentinel.msg_off = (uint32_t)msg; sentinel.tile_begin = (uint32_t)tiles;
     sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw; sentinel.grp_begin = (uint32_t)groups;
@@ -158,7 +208,9 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     Layout L{};
     L.segs = c->d_segs; L.nseg = (uint32_t)nseg; L.tiles_per_worker = (uint32_t)tiles; L.groups_per_worker = (uint32_t)groups;
     L.scat_per_group = (uint32_t)scat; L.K_total = (uint32_t)msg; L.n_total = n; L.mask_words_per_group = maskw;
+    L.cand_per_worker = cand; L.flag_per_worker = flag; L.fast_per_worker = fast_count;
     c->layout = L;
+    c->slow_segments = slow_count; c->max_sample_m = max_m; c->max_flag_cap = max_cap;
     c->cached_segs.assign(segs, segs + nseg);
     c->cached_n = n;
     c->layout_valid = true;
@@ -203,21 +255,59 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
 
     if (scheme == SC_TOPK) {
         SC_CUDA(cudaMemsetAsync(c->d_hist, 0, (size_t)P * HIST_WORDS * sizeof(uint32_t), stream));
+        SC_CUDA(cudaMemsetAsync(c->d_fstate, 0, (size_t)P * sizeof(FastState), stream));
+        c->last_topk_problems = P;
+        const uint32_t n_slow0 = (uint32_t)W * c->slow_segments;
+        const uint32_t counters[2] = {n_slow0, 0u};
+        SC_CUDA(cudaMemcpyAsync(c->d_nslow, counters, sizeof(counters), cudaMemcpyHostToDevice, stream));
+        if (L.fast_per_worker) {
+            FastParams fp{};
+            fp.L = L; fp.grads = grads; fp.residuals = residuals; fp.out_vals = out_vals; fp.out_idx = out_idx;
+            fp.state = c->d_fstate; fp.sample = c->d_sample; fp.cand_hist = c->d_cand_hist;
+            fp.list2 = c->d_list2; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
+            fp.flagged = c->d_flagged; fp.reserve = c->d_reserve; fp.offsets = c->d_offsets;
+            fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
+            SC_CUDA(cudaMemsetAsync(c->d_reserve, 0, (size_t)P * sizeof(unsigned long long), stream));
+            SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
+            { Launch l(c, KIND_SAMPLE, stream);
+              topk_sample_kernel<<<dim3((c->max_sample_m / 8 + THREADS - 1) / THREADS, P), THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_BRACKET, stream);
+              topk_bracket_kernel<<<P, THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_MAIN, stream);
+              topk_main_kernel<<<persistent_grid(c, c->occ_main, items), THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_CANDBIN, stream);
+              topk_candbin_kernel<<<P, THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_CANDFILTER, stream);
+              const uint32_t gx = std::min<uint32_t>((c->max_flag_cap + THREADS * 4 - 1) / (THREADS * 4), 2048u);
+              topk_candfilter_kernel<<<dim3(std::max(gx, 1u), P), THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_FINAL, stream);
+              topk_final_kernel<<<P, THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_RESTORE, stream);
+              const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
+              topk_restore_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_TILECOUNT, stream);
+              topk_tilecount_kernel<<<(items + WARPS - 1) / WARPS, THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_ROW_SCAN, stream);
+              row_scan_kernel<<<W, THREADS, 0, stream>>>(c->d_offsets, L.tiles_per_worker); }
+            { Launch l(c, KIND_EMIT, stream);
+              const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
+              topk_emit_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
+        }
         { Launch l(c, KIND_HIST0, stream);
-          topk_hist0_kernel<true><<<persistent_grid(c, c->occ_hist, items), THREADS, 0, stream>>>(
-              L, grads, residuals, c->d_hist, items); }
+          topk_hist0_kernel<<<persistent_grid(c, c->occ_hist, items), THREADS, 0, stream>>>(
+              L, grads, residuals, c->d_hist, c->d_fstate, c->d_nslow, items); }
         { Launch l(c, KIND_RESOLVE, stream);
-          topk_resolve_kernel<0><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status); }
+          topk_resolve_kernel<0><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
         { Launch l(c, KIND_REFINE, stream);
           topk_refine_kernel<1><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
-              L, residuals, c->d_hist, c->d_state, items); }
+              L, residuals, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, items); }
         { Launch l(c, KIND_RESOLVE, stream);
-          topk_resolve_kernel<1><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status); }
+          topk_resolve_kernel<1><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
         { Launch l(c, KIND_REFINE, stream);
           topk_refine_kernel<2><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
-              L, residuals, c->d_hist, c->d_state, items); }
+              L, residuals, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, items); }
         { Launch l(c, KIND_RESOLVE, stream);
-          topk_resolve_kernel<2><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_status); }
+          topk_resolve_kernel<2><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
     } else {
         SC_CUDA(cudaMemcpyAsync(c->d_seeds, h_seeds, sizeof(uint64_t) * W, cudaMemcpyHostToDevice, stream));
     }
@@ -258,18 +348,19 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
     PackParams pp{};
     pp.L = L; pp.grads = grads; pp.residuals = residuals; pp.out_vals = out_vals; pp.out_idx = out_idx;
     pp.state = c->d_state; pp.mask = c->d_mask; pp.mask_per_worker = 0u;
+    pp.fstate = c->d_fstate; pp.n_slow = c->d_nslow;
+    SC_CUDA(cudaMemsetAsync(c->d_ticket, 0, sizeof(unsigned long long), stream));
     if (++c->epoch >= (1u << 28)) {            // tags wrapped: forget every old word
         SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), stream));
         c->epoch = 1;
     }
     const uint32_t gitems = (uint32_t)W * L.groups_per_worker;
     pp.epoch = c->epoch; pp.total_items = gitems;
-    pp.ticket = c->d_ticket; pp.ticket_base = c->ticket_base;
+    pp.ticket = c->d_ticket;
     pp.desc = c->d_desc; pp.status = c->d_status;
     const uint32_t grid = persistent_grid(c, c->occ_pack_topk, gitems);
     { Launch l(c, KIND_PACK_TOPK, stream);
       pack_kernel<PACK_TOPK><<<grid, THREADS, 0, stream>>>(pp); }
-    c->ticket_base += (unsigned long long)gitems + grid;   // every CTA draws exactly one ticket past the end
     SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
@@ -339,6 +430,10 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     c->max_mask_words = (max_n + 31) / 32 + (size_t)max_segments;
     c->max_atiles = (max_n + ATILE - 1) / ATILE;
     const size_t P = (size_t)max_W * max_segments;
+    c->max_fast_per_worker = std::min<size_t>((size_t)max_segments, std::max<size_t>(1, max_n >> 20));
+    c->max_cand_per_worker = max_n / 32 + c->max_fast_per_worker * 16384;
+    const size_t items_max = (size_t)max_W * c->max_tiles_per_worker;
+    const size_t fastP = (size_t)max_W * c->max_fast_per_worker;
     int rc = SC_OK;
     if ((rc = dev_alloc(c, &c->d_segs, (size_t)max_segments + 1)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_hist, P * HIST_WORDS)) == SC_OK &&
@@ -348,6 +443,14 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_mask, (size_t)max_W * c->max_mask_words)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_bounds, (size_t)max_W * (c->max_atiles + 1))) == SC_OK &&
         (rc = dev_alloc(c, &c->d_offsets, (size_t)max_W * (c->max_tiles_per_worker + 1))) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_fstate, P)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_sample, fastP * SAMPLE_MAX)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_cand_hist, fastP * CAND_BINS)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_list2, fastP * LIST2_CAP)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tile_fbase, items_max)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tile_fcnt, items_max)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_reserve, P)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_nslow, 2)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_seeds, (size_t)max_W)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_status, 1)) == SC_OK) {
         bool ok = cudaMemset(c->d_desc, 0, (size_t)max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long)) == cudaSuccess &&
@@ -357,7 +460,9 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         if (!ok) rc = SC_ERR_CUDA;
     }
     if (rc == SC_OK) {
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel<true>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main, topk_main_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit, topk_emit_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_refine, topk_refine_kernel<1>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_topk, pack_kernel<PACK_TOPK>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_mask, randk_pack_kernel, THREADS, 0);
@@ -374,7 +479,10 @@ void sc_destroy(sc_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
     cudaFree(c->d_segs); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
-    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_seeds); cudaFree(c->d_status);
+    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate); cudaFree(c->d_sample);
+    cudaFree(c->d_cand_hist); cudaFree(c->d_cand); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_cbase);
+    cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt); cudaFree(c->d_reserve);
+    cudaFree(c->d_flagged); cudaFree(c->d_nslow); cudaFree(c->d_seeds); cudaFree(c->d_status);
     cudaFree(c->d_stage_grads); cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); cudaFree(c->d_stage_out);
     for (cudaEvent_t e : c->ev_worker) cudaEventDestroy(e);
     for (auto& r : c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -422,6 +530,19 @@ int sc_profile_read(sc_ctx* c, double* ms, uint64_t* launches) {
         ms[r.kind] += t;
         launches[r.kind] += 1;
     }
+    return SC_OK;
+}
+
+int sc_topk_path_counts(sc_ctx* c, void* stream, uint32_t* h_counts) {
+    if (!c || !h_counts) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::vector<FastState> h(c->last_topk_problems);
+    h_counts[0] = h_counts[1] = h_counts[2] = 0;
+    if (h.empty()) return SC_OK;
+    SC_CUDA(cudaMemcpyAsync(h.data(), c->d_fstate, h.size() * sizeof(FastState), cudaMemcpyDeviceToHost, st));
+    SC_CUDA(cudaStreamSynchronize(st));
+    for (const FastState& f : h) if (f.path < 3) ++h_counts[f.path];
     return SC_OK;
 }
 

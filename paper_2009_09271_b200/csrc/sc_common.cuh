@@ -29,6 +29,14 @@ struct SegEntry {
     uint32_t tile_begin;      // first tile of the segment inside a worker
     uint32_t scat_begin;      // first scatter chunk of the segment inside a seed group
     uint32_t grp_begin;       // first pack group (PACK_GROUP tiles) of the segment inside a worker
+    uint32_t fast;            // 1: large segment, top-k goes through the sampled-bracket path
+    uint32_t sample_m;        // sample size of that path (multiple of 8)
+    uint32_t cand_cap;        // capacity of the segment's candidate list
+    uint32_t fast_index;      // index among the fast segments of a worker
+    uint64_t cand_begin;      // first candidate slot of the segment inside a worker
+    uint64_t flag_begin;      // first flagged-list slot of the segment inside a worker
+    uint32_t flag_cap;        // capacity of the segment's flagged list (k + candidate capacity)
+    uint32_t pad;
 };
 
 struct Layout {
@@ -40,6 +48,10 @@ struct Layout {
     uint32_t K_total;         // message entries per worker
     uint64_t n_total;         // elements per worker row
     uint64_t mask_words_per_group;
+    uint64_t cand_per_worker; // candidate slots per worker (all fast segments)
+    uint64_t flag_per_worker; // flagged-list slots per worker
+    uint32_t fast_per_worker; // fast segments per worker
+    uint32_t pad;
 };
 
 // Per (worker, segment) result of the radix select.
@@ -52,6 +64,28 @@ struct TopkState {
     uint32_t dual;     // 1 if only some of the ties are kept (r < number of ties)
     uint32_t pad0, pad1;
 };
+
+// Top-k of a large segment: state of the sampled-bracket path.
+enum { PATH_SLOW = 0,     // small segment: multi-pass radix select
+       PATH_FAST = 1,     // bracket holds: single streaming pass + sparse emit
+       PATH_FAILED = 2 }; // bracket missed or a list overflowed: radix select on the parked p
+struct FastState {
+    uint32_t path;
+    uint32_t lo, hi;       // bracket: key > hi is surely kept, key < lo surely dropped
+    uint32_t shift;        // candidate histogram bin = (key - lo) >> shift
+    uint32_t sure_total;   // elements with key > hi
+    uint32_t cand_total;   // candidate slots reserved (may exceed the capacity)
+    uint32_t lo2, hi2;     // key range of the candidate-histogram bin that holds the threshold
+    uint32_t need2;        // 1-based rank of the threshold inside that bin (0: no candidate is kept)
+    uint32_t cnt2;         // candidates copied into the short list
+    uint32_t T, icut;      // kept <=> key > T, or key == T and coordinate < icut
+    uint32_t pad[4];
+};
+
+constexpr uint32_t FAST_MIN_N = 1u << 20;
+constexpr uint32_t SAMPLE_MIN = 1u << 14, SAMPLE_MAX = 1u << 18;
+constexpr uint32_t CAND_BINS = 2048;
+constexpr uint32_t LIST2_CAP = 4096;
 
 // ---------------------------------------------------------------------------
 // integer hashing (the generator specification; integer-only, so host, device

@@ -32,13 +32,14 @@ struct PackParams {
     float* out_vals;
     uint32_t* out_idx;
     const TopkState* state;          // PACK_TOPK
+    const FastState* fstate;         // segments already served by the sampled-bracket path are skipped
+    const uint32_t* n_slow;          // 0: nothing to do for this launch
     const uint32_t* mask;            // PACK_MASK
     uint32_t mask_per_worker;        // 1: worker w uses mask group w, 0: all use group 0
     uint32_t epoch;                  // tag of this launch inside the descriptor words
     uint32_t total_items;            // groups over all workers
     uint32_t pad;
-    unsigned long long* ticket;
-    unsigned long long ticket_base;
+    unsigned long long* ticket;      // zeroed before the launch
     unsigned long long* desc;        // two words per group
     int* status;
 };
@@ -150,10 +151,11 @@ pack_kernel(PackParams P) {
     __shared__ uint32_t s_grp_excl[2];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const Layout& L = P.L;
+    if (*P.n_slow == 0u) return;
 
     while (true) {
         if (threadIdx.x == 0) {
-            unsigned long long tk = atomicAdd(P.ticket, 1ull) - P.ticket_base;
+            unsigned long long tk = atomicAdd(P.ticket, 1ull);
             uint32_t item = tk < (unsigned long long)P.total_items ? (uint32_t)tk : 0xFFFFFFFFu;
             s_dec[0] = item;
             if (item != 0xFFFFFFFFu) {
@@ -171,6 +173,7 @@ pack_kernel(PackParams P) {
         const uint32_t item = s_dec[0];
         if (item == 0xFFFFFFFFu) break;
         const uint32_t w = s_dec[1], s = s_dec[2], gi = s_dec[3], ntl = s_dec[4];
+        if (P.fstate[(size_t)w * L.nseg + s].path == PATH_FAST) { __syncthreads(); continue; }
         const SegEntry seg = L.segs[s];
         const size_t row = (size_t)w * L.n_total + seg.offset;
         float* e = P.residuals + row;

@@ -24,14 +24,17 @@ __device__ inline void flush_hist(uint32_t* sh, uint32_t* __restrict__ gh) {
     __syncthreads();
 }
 
-// Level 0.  FUSE_ADD: read g and e, write p = g + e into the residual buffer.
-// Otherwise the residual buffer already holds p.
-template <bool FUSE_ADD>
+// Level 0.  For a segment on the plain radix-select path (PATH_SLOW) this pass reads g and e
+// and writes p = g + e into the residual buffer; for a segment whose sampled bracket failed
+// (PATH_FAILED) the residual buffer already holds p.  Segments served by the fast path are
+// skipped, and the whole launch returns at once when no segment needs it.
 __global__ void __launch_bounds__(THREADS)
 topk_hist0_kernel(Layout L, const float* __restrict__ grads, float* __restrict__ residuals,
-                  uint32_t* __restrict__ hist, uint32_t total_items) {
+                  uint32_t* __restrict__ hist, const FastState* __restrict__ fstate,
+                  const uint32_t* __restrict__ n_slow, uint32_t total_items) {
     __shared__ uint32_t sh[HIST0_BINS];
-    __shared__ uint32_t s_dec[3];
+    __shared__ uint32_t s_dec[4];
+    if (*n_slow == 0u) return;
     for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) sh[b] = 0;
     __syncthreads();
     long long cur_prob = -1;
@@ -41,9 +44,12 @@ topk_hist0_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
             uint32_t lt = item - w * L.tiles_per_worker;
             uint32_t s = find_by_tile(L, lt);
             s_dec[0] = w; s_dec[1] = s; s_dec[2] = lt - L.segs[s].tile_begin;
+            s_dec[3] = fstate[(size_t)w * L.nseg + s].path;
         }
         __syncthreads();
-        const uint32_t w = s_dec[0], s = s_dec[1], t = s_dec[2];
+        const uint32_t w = s_dec[0], s = s_dec[1], t = s_dec[2], path = s_dec[3];
+        if (path == PATH_FAST) { __syncthreads(); continue; }
+        const bool FUSE_ADD = path == PATH_SLOW;
         const long long prob = (long long)w * L.nseg + s;
         if (prob != cur_prob) {
             if (cur_prob >= 0) flush_hist<HIST0_BINS>(sh, hist + (size_t)cur_prob * HIST_WORDS);
@@ -89,11 +95,13 @@ topk_hist0_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
 template <int LEVEL>
 __global__ void __launch_bounds__(THREADS)
 topk_refine_kernel(Layout L, const float* __restrict__ residuals, uint32_t* __restrict__ hist,
-                   const TopkState* __restrict__ state, uint32_t total_items) {
+                   const TopkState* __restrict__ state, const FastState* __restrict__ fstate,
+                   const uint32_t* __restrict__ n_slow, uint32_t total_items) {
     constexpr uint32_t SHIFT = (LEVEL == 1) ? 10u : 0u;
     constexpr uint32_t HOFF = (LEVEL == 1) ? HIST0_BINS : HIST0_BINS + HIST1_BINS;
     __shared__ uint32_t sh[1024];
     __shared__ uint32_t s_dec[3];
+    if (*n_slow == 0u) return;
     for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) sh[b] = 0;
     __syncthreads();
     long long cur_prob = -1;
@@ -108,7 +116,7 @@ topk_refine_kernel(Layout L, const float* __restrict__ residuals, uint32_t* __re
         const uint32_t w = s_dec[0], s = s_dec[1], t = s_dec[2];
         const long long prob = (long long)w * L.nseg + s;
         const TopkState st = state[prob];
-        if (st.active) {                                   // uniform over the CTA
+        if (st.active && fstate[prob].path != PATH_FAST) {   // uniform over the CTA
             if (prob != cur_prob) {
                 if (cur_prob >= 0) flush_hist<1024>(sh, hist + (size_t)cur_prob * HIST_WORDS + HOFF);
                 cur_prob = prob;
@@ -148,6 +156,7 @@ topk_refine_kernel(Layout L, const float* __restrict__ residuals, uint32_t* __re
 template <int LEVEL>
 __global__ void __launch_bounds__(THREADS)
 topk_resolve_kernel(Layout L, const uint32_t* __restrict__ hist, TopkState* __restrict__ state,
+                    const FastState* __restrict__ fstate, const uint32_t* __restrict__ n_slow,
                     int* __restrict__ status) {
     constexpr uint32_t BINS = (LEVEL == 0) ? HIST0_BINS : 1024u;
     constexpr uint32_t SHIFT = (LEVEL == 0) ? 20u : (LEVEL == 1) ? 10u : 0u;
@@ -157,6 +166,7 @@ topk_resolve_kernel(Layout L, const uint32_t* __restrict__ hist, TopkState* __re
     __shared__ uint32_t s_found;
     const uint32_t prob = blockIdx.x;
     const uint32_t s = prob % L.nseg;
+    if (*n_slow == 0u || fstate[prob].path == PATH_FAST) return;
     uint32_t need, prefix;
     if (LEVEL == 0) {
         need = L.segs[s].k;

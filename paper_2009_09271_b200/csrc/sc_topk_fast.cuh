@@ -1,0 +1,571 @@
+// Top-k of a large segment in ONE pass over g and e (Methodology, "Top-k Sparsification";
+// Algorithm 1 accumulate / compress / residual lines).
+//
+// A radix select has to see every key before it knows the threshold, which costs extra
+// passes over HBM.  Here a small systematic sample of |g + e| brackets the threshold first:
+//   sample   m keys per (worker, segment); two order statistics of the sample, six standard
+//            deviations either side of rank k m / n, give [lo, hi] with
+//            count(key > hi) <= k <= count(key >= lo) except with negligible probability;
+//   main     the streaming pass forms p = g + e and writes the residual at once: 0 for the
+//            "sure" elements (key > hi), p for the rest.  Every element with key >= lo is
+//            appended, in coordinate order inside its tile, to a "flagged" list (value,
+//            coordinate); the few candidates (lo <= key <= hi) also go to a candidate list
+//            and into a 2048-bin histogram;
+//   resolve  the candidate histogram pins the bin of the k-th key, the candidates of that
+//            bin are sorted in shared memory: exact threshold T and the coordinate cut for
+//            ties.  Every count is exact, so the result equals the plain definition; the
+//            sample only decides how much work that takes.  If the bracket is wrong (counts
+//            prove it) or a list overflows, the segment falls back to the radix select on
+//            the parked p;
+//   emit     per-tile kept counts -> exclusive scan -> a pass over the flagged list only:
+//            kept entries go to the message in ascending coordinate order, kept candidates
+//            are zeroed in the residual.  On a fall-back the sure values are first written
+//            back from the flagged list.
+// No CTA waits on another anywhere on this path.
+#pragma once
+#include "sc_common.cuh"
+
+namespace sc {
+
+struct FastParams {
+    Layout L;
+    const float* grads;
+    float* residuals;
+    float* out_vals;
+    uint32_t* out_idx;
+    FastState* state;          // [W * nseg]
+    uint32_t* sample;          // [W * fast_per_worker][SAMPLE_MAX]
+    uint32_t* cand_hist;       // [W * fast_per_worker][CAND_BINS]
+    uint2* list2;              // [W * fast_per_worker][LIST2_CAP]
+    uint2* flagged;            // [W][flag_per_worker] (value bits, coordinate inside the segment)
+    uint32_t* tile_fbase;      // first flagged slot of the tile (0xFFFFFFFF: the list was full, nothing written)
+    uint32_t* tile_fcnt;       // flagged elements of the tile
+    unsigned long long* reserve;   // [W * nseg]: candidates reserved << 32 | flagged reserved
+    uint32_t* n_failed;        // segments whose bracket missed
+    uint32_t* offsets;         // [W][tiles_per_worker + 1]
+    uint32_t* n_slow;          // segments that need the radix-select path
+    int* status;
+    uint32_t total_items;
+};
+
+// ---- shared helper: walk a histogram from its highest bin down to the bin that holds the
+// need-th largest element.  All THREADS threads call it; results are uniform.
+template <uint32_t BINS, typename HistPtr>
+__device__ inline bool find_from_top(HistPtr h, uint32_t need, uint32_t* s_tmp /*WARPS+4*/, uint32_t& bin,
+                                     uint32_t& need_in, uint32_t& cnt) {
+    constexpr uint32_t BPT = BINS / THREADS;
+    uint32_t local[BPT], sum = 0;
+#pragma unroll
+    for (uint32_t c = 0; c < BPT; ++c) {
+        local[c] = h[BINS - 1u - (threadIdx.x * BPT + c)];
+        sum += local[c];
+    }
+    if (threadIdx.x == 0) s_tmp[WARPS + 1] = 0xFFFFFFFFu;
+    uint32_t total;
+    const uint32_t before = block_exclusive_scan(sum, s_tmp, &total);
+    if (need >= 1 && before < need && need <= before + sum) {
+        uint32_t acc = before;
+#pragma unroll
+        for (uint32_t c = 0; c < BPT; ++c) {
+            if (need <= acc + local[c]) {
+                s_tmp[WARPS + 1] = BINS - 1u - (threadIdx.x * BPT + c);
+                s_tmp[WARPS + 2] = need - acc;
+                s_tmp[WARPS + 3] = local[c];
+                break;
+            }
+            acc += local[c];
+        }
+    }
+    __syncthreads();
+    bin = s_tmp[WARPS + 1]; need_in = s_tmp[WARPS + 2]; cnt = s_tmp[WARPS + 3];
+    __syncthreads();
+    return bin != 0xFFFFFFFFu;
+}
+
+// ---- sample: one 32-byte sector (8 elements) of g and e per thread ----------------------
+__global__ void __launch_bounds__(THREADS)
+topk_sample_kernel(FastParams P) {
+    const Layout& L = P.L;
+    const uint32_t prob = blockIdx.y;
+    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    const SegEntry seg = L.segs[s];
+    if (!seg.fast) return;
+    const uint32_t c = blockIdx.x * THREADS + threadIdx.x;            // sector of the sample
+    if (c >= seg.sample_m / 8u) return;
+    const size_t row = (size_t)w * L.n_total + seg.offset;
+    const float* g = P.grads + row;
+    const float* e = P.residuals + row;
+    const uint32_t a0 = (8u - (uint32_t)((reinterpret_cast<uintptr_t>(e) >> 2) & 7u)) & 7u;   // first 32B-aligned element
+    const uint32_t sectors = (seg.n - a0) / 8u;
+    const uint32_t sidx = (uint32_t)(((uint64_t)c * sectors) / (seg.sample_m / 8u));
+    const size_t at = (size_t)a0 + (size_t)sidx * 8u;
+    const float4 e0 = *reinterpret_cast<const float4*>(e + at), e1 = *reinterpret_cast<const float4*>(e + at + 4);
+    const float4 g0 = *reinterpret_cast<const float4*>(g + at), g1 = *reinterpret_cast<const float4*>(g + at + 4);
+    uint4 k0, k1;
+    k0.x = key_of(g0.x + e0.x); k0.y = key_of(g0.y + e0.y); k0.z = key_of(g0.z + e0.z); k0.w = key_of(g0.w + e0.w);
+    k1.x = key_of(g1.x + e1.x); k1.y = key_of(g1.y + e1.y); k1.z = key_of(g1.z + e1.z); k1.w = key_of(g1.w + e1.w);
+    uint4* out = reinterpret_cast<uint4*>(P.sample + ((size_t)w * L.fast_per_worker + seg.fast_index) * SAMPLE_MAX + (size_t)c * 8u);
+    out[0] = k0; out[1] = k1;
+}
+
+// ---- bracket: two order statistics of the sample, to 21 bits (one CTA per problem) ------
+__global__ void __launch_bounds__(THREADS)
+topk_bracket_kernel(FastParams P) {
+    __shared__ uint32_t h0[HIST0_BINS];
+    __shared__ uint32_t hA[1024], hB[1024];
+    __shared__ uint32_t s_tmp[WARPS + 4];
+    const Layout& L = P.L;
+    const uint32_t prob = blockIdx.x;
+    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    const SegEntry seg = L.segs[s];
+    if (!seg.fast) return;
+    const uint32_t m = seg.sample_m;
+    const uint4* smp = reinterpret_cast<const uint4*>(P.sample + ((size_t)w * L.fast_per_worker + seg.fast_index) * SAMPLE_MAX);
+    // ranks (from the top) that bracket the k-th largest of the segment
+    const double q = (double)seg.k / (double)seg.n;
+    const double centre = q * (double)m;
+    const double delta = 6.0 * sqrt((double)m * q * (1.0 - q)) + 2.0;
+    const long long j_hi = (long long)floor(centre - delta);          // keys above this rank: surely kept
+    const long long j_lo = (long long)ceil(centre + delta);           // keys below this rank: surely dropped
+    const bool have_hi = j_hi >= 1, have_lo = j_lo <= (long long)m;
+
+    for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) h0[b] = 0;
+    for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) { hA[b] = 0; hB[b] = 0; }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < m / 4u; i += THREADS) {
+        const uint4 k = smp[i];
+        atomicAdd(&h0[k.x >> 20], 1u); atomicAdd(&h0[k.y >> 20], 1u);
+        atomicAdd(&h0[k.z >> 20], 1u); atomicAdd(&h0[k.w >> 20], 1u);
+    }
+    __syncthreads();
+    uint32_t binA = 0, needA = 0, binB = 0, needB = 0, cnt = 0;
+    if (have_hi) find_from_top<HIST0_BINS>(h0, (uint32_t)j_hi, s_tmp, binA, needA, cnt);
+    if (have_lo) find_from_top<HIST0_BINS>(h0, (uint32_t)j_lo, s_tmp, binB, needB, cnt);
+    for (uint32_t i = threadIdx.x; i < m / 4u; i += THREADS) {
+        const uint4 k = smp[i];
+        const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (have_hi && (kk[c] >> 20) == binA) atomicAdd(&hA[(kk[c] >> 10) & 1023u], 1u);
+            if (have_lo && (kk[c] >> 20) == binB) atomicAdd(&hB[(kk[c] >> 10) & 1023u], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t hi = 0x7FFFFFFFu, lo = 0u, bin1 = 0, need1 = 0;
+    if (have_hi && find_from_top<1024>(hA, needA, s_tmp, bin1, need1, cnt)) hi = (binA << 20) | (bin1 << 10) | 1023u;
+    if (have_lo && find_from_top<1024>(hB, needB, s_tmp, bin1, need1, cnt)) lo = (binB << 20) | (bin1 << 10);
+    if (lo > hi) lo = hi;                                              // (cannot happen; keeps the bracket sane)
+    if (threadIdx.x == 0) {
+        const uint32_t width_m1 = hi - lo;
+        const uint32_t bits = width_m1 ? 32u - (uint32_t)__clz((int)width_m1) : 0u;
+        FastState st = {};
+        st.path = PATH_FAST; st.lo = lo; st.hi = hi; st.shift = bits > 11u ? bits - 11u : 0u;
+        P.state[prob] = st;
+    }
+}
+
+// ---- main streaming pass ---------------------------------------------------------------
+// Mapping: warp w of a tile owns 512 consecutive elements as four rows of 128; lane l holds
+// the quad at 128 j + 4 l of row j (coalesced 512-byte accesses).  Four per-row counts ride
+// in the bytes of one word, so one 5-step warp scan ranks all rows.
+__device__ inline uint32_t pack_counts(uint32_t bits16) {
+    return __popc(bits16 & 0xFu) | (__popc(bits16 & 0xF0u) << 8) | (__popc(bits16 & 0xF00u) << 16) |
+           (__popc(bits16 & 0xF000u) << 24);
+}
+__device__ inline uint32_t warp_inclusive_scan(uint32_t v, uint32_t lane) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= (uint32_t)d) v += t;
+    }
+    return v;
+}
+__device__ inline uint32_t bytes_sum(uint32_t v) { return (v & 0xFFu) + ((v >> 8) & 0xFFu) + ((v >> 16) & 0xFFu) + (v >> 24); }
+
+__global__ void __launch_bounds__(THREADS, 4)
+topk_main_kernel(FastParams P) {
+    __shared__ uint32_t sh[CAND_BINS];
+    __shared__ uint32_t s_wsure[2][WARPS], s_wcand[2][WARPS], s_wflag[2][WARPS];
+    __shared__ unsigned long long s_base[2];
+    const Layout& L = P.L;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) sh[b] = 0;
+    __syncthreads();
+    long long cur_prob = -1;
+    size_t cur_fidx = 0;
+    uint32_t lo = 0, hi = 0, shift = 0, parity = 0;
+    for (uint32_t item = blockIdx.x; item < P.total_items; item += gridDim.x) {
+        const uint32_t w = item / L.tiles_per_worker;
+        const uint32_t lt = item - w * L.tiles_per_worker;
+        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+        const SegEntry seg = L.segs[s];
+        if (!seg.fast) continue;                                       // uniform over the CTA
+        const long long prob = (long long)w * L.nseg + s;
+        if (prob != cur_prob) {
+            if (cur_prob >= 0) {
+                __syncthreads();
+                for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
+                    const uint32_t c = sh[b];
+                    if (c) { atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c); sh[b] = 0; }
+                }
+                __syncthreads();
+            }
+            cur_prob = prob;
+            cur_fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
+            const FastState st = P.state[prob];
+            lo = st.lo; hi = st.hi; shift = st.shift;
+        }
+        parity ^= 1u;
+        const uint32_t t = lt - seg.tile_begin;
+        const size_t row = (size_t)w * L.n_total + seg.offset;
+        const float* g = P.grads + row;
+        float* e = P.residuals + row;
+        const uint32_t mis = misalign_of(e);
+        const long long first = (long long)t * TILE - mis;
+        const long long mine = first + warp * 512 + lane * 4;            // quad of row 0; row j at + 128 j
+        const bool full = first >= 0 && first + TILE <= (long long)seg.n;
+
+        float p[QUADS][4];
+        uint32_t valid16 = 0;
+        if (full) {
+            float4 ev[QUADS], gv[QUADS];
+#pragma unroll
+            for (int j = 0; j < QUADS; ++j) {
+                ev[j] = __ldcs(reinterpret_cast<const float4*>(e + mine + 128 * j));
+                gv[j] = __ldcs(reinterpret_cast<const float4*>(g + mine + 128 * j));
+            }
+#pragma unroll
+            for (int j = 0; j < QUADS; ++j) {
+                p[j][0] = gv[j].x + ev[j].x; p[j][1] = gv[j].y + ev[j].y;
+                p[j][2] = gv[j].z + ev[j].z; p[j][3] = gv[j].w + ev[j].w;
+            }
+            valid16 = 0xFFFFu;
+        } else {
+#pragma unroll
+            for (int j = 0; j < QUADS; ++j) {
+                const long long base = mine + 128 * j;
+                float gq[4];
+                const uint32_t valid = load_quad(e, base, seg.n, p[j]);
+                load_quad_stream(g, base, seg.n, gq);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) p[j][c] = gq[c] + p[j][c];
+                valid16 |= valid << (4 * j);
+            }
+        }
+        // classify
+        uint32_t flag16 = 0, sure16 = 0;
+#pragma unroll
+        for (int j = 0; j < QUADS; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t key = key_of(p[j][c]);
+                flag16 |= (uint32_t)(key >= lo) << (4 * j + c);
+                sure16 |= (uint32_t)(key > hi) << (4 * j + c);
+            }
+        flag16 &= valid16; sure16 &= valid16;
+        const uint32_t cand16 = flag16 & ~sure16;
+        // ranks of the flagged elements inside the warp, in coordinate order
+        const uint32_t fcnt4 = pack_counts(flag16);
+        const uint32_t finc4 = warp_inclusive_scan(fcnt4, lane);
+        const uint32_t ftot4 = __shfl_sync(0xFFFFFFFFu, finc4, 31);
+        const uint32_t wcand = __reduce_add_sync(0xFFFFFFFFu, __popc(cand16));
+        const uint32_t wsure = __reduce_add_sync(0xFFFFFFFFu, __popc(sure16));
+        if (lane == 0) { s_wsure[parity][warp] = wsure; s_wcand[parity][warp] = wcand; s_wflag[parity][warp] = bytes_sum(ftot4); }
+        __syncthreads();
+        uint32_t tsure = 0, tcand = 0, tflag = 0, fwbase = 0;
+#pragma unroll
+        for (int i = 0; i < WARPS; ++i) {
+            tsure += s_wsure[parity][i];
+            const uint32_t f = s_wflag[parity][i];
+            fwbase += (i < (int)warp) ? f : 0u;
+            tcand += s_wcand[parity][i]; tflag += f;
+        }
+        if (threadIdx.x == 0) {
+            unsigned long long base = 0;
+            if (tflag) base = atomicAdd(P.reserve + prob, ((unsigned long long)tcand << 32) | tflag);
+            const uint32_t fbase = (uint32_t)base;
+            const bool fits = (unsigned long long)fbase + tflag <= seg.flag_cap;
+            if (tsure && fits) atomicAdd(&P.state[prob].sure_total, tsure);
+            P.tile_fbase[item] = fits ? fbase : 0xFFFFFFFFu; P.tile_fcnt[item] = tflag;
+            s_base[parity] = fits ? base : ~0ull;
+        }
+        bool fits = true;
+        if (tflag) {                                                   // uniform over the CTA
+            __syncthreads();
+            const unsigned long long base = s_base[parity];
+            fits = base != ~0ull;
+            if (fits && flag16) {
+                uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
+                uint32_t rowbase = (uint32_t)base + fwbase;
+#pragma unroll
+                for (int j = 0; j < QUADS; ++j) {
+                    uint32_t slot = rowbase + ((finc4 - fcnt4) >> (8 * j) & 0xFFu);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if ((flag16 >> (4 * j + c)) & 1u)
+                            flist[slot++] = make_uint2(__float_as_uint(p[j][c]), (uint32_t)(mine + 128 * j + c));
+                    rowbase += (ftot4 >> (8 * j)) & 0xFFu;
+                }
+            }
+            if (fits && cand16) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if ((cand16 >> i) & 1u)
+                        atomicAdd(&sh[min((key_of(p[i >> 2][i & 3]) - lo) >> shift, CAND_BINS - 1u)], 1u);
+            }
+        }
+        // residual: sure elements are certainly kept, so they become zero right here (only if
+        // their values made it into the flagged list, from where a fall-back can restore them)
+        if (fits && sure16) {
+#pragma unroll
+            for (int j = 0; j < QUADS; ++j)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if ((sure16 >> (4 * j + c)) & 1u) p[j][c] = 0.0f;
+        }
+        if (full) {
+#pragma unroll
+            for (int j = 0; j < QUADS; ++j)
+                *reinterpret_cast<float4*>(e + mine + 128 * j) = make_float4(p[j][0], p[j][1], p[j][2], p[j][3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < QUADS; ++j) {
+                const uint32_t valid = (valid16 >> (4 * j)) & 0xFu;
+                if (valid) store_quad(e, mine + 128 * j, valid, p[j]);
+            }
+        }
+    }
+    if (cur_prob >= 0) {
+        __syncthreads();
+        for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
+            const uint32_t c = sh[b];
+            if (c) atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c);
+        }
+    }
+}
+
+// ---- resolve 1: validity of the bracket, bin of the threshold (one CTA per problem) ------
+__global__ void __launch_bounds__(THREADS)
+topk_candbin_kernel(FastParams P) {
+    __shared__ uint32_t s_tmp[WARPS + 4];
+    const Layout& L = P.L;
+    const uint32_t prob = blockIdx.x;
+    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    const SegEntry seg = L.segs[s];
+    if (!seg.fast) return;
+    FastState st = P.state[prob];
+    if (st.path != PATH_FAST) return;
+    const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
+    const unsigned long long rsv = P.reserve[prob];
+    st.cand_total = (uint32_t)(rsv >> 32);
+    const uint32_t flag_total = (uint32_t)rsv;
+    bool ok = flag_total <= seg.flag_cap && st.sure_total <= seg.k &&
+              (uint64_t)seg.k <= (uint64_t)st.sure_total + st.cand_total;
+    uint32_t bin = 0, need_in = 0, cnt = 0;
+    const uint32_t need = ok ? seg.k - st.sure_total : 0u;
+    if (ok && need) {
+        ok = find_from_top<CAND_BINS>(P.cand_hist + fidx * CAND_BINS, need, s_tmp, bin, need_in, cnt);
+        ok = ok && cnt <= LIST2_CAP;
+    }
+    if (threadIdx.x == 0) {
+        if (!ok) {
+            st.path = PATH_FAILED;
+            atomicAdd(P.n_slow, 1u);
+            atomicAdd(P.n_failed, 1u);
+        } else if (need == 0) {
+            st.need2 = 0; st.T = st.hi; st.icut = 0;                   // exactly the sure elements are kept
+        } else {
+            st.lo2 = st.lo + (bin << st.shift);
+            const uint64_t top = (uint64_t)st.lo2 + (1ull << st.shift) - 1ull;
+            st.hi2 = bin == CAND_BINS - 1u ? st.hi : (uint32_t)min(top, (uint64_t)st.hi);
+            st.need2 = need_in;
+            st.T = cnt;                                                // expected length of the short list (checked later)
+        }
+        st.cnt2 = 0;
+        P.state[prob] = st;
+    }
+}
+
+// ---- filter: copy the flagged entries of the threshold's bin into the short list -------------
+__global__ void __launch_bounds__(THREADS)
+topk_candfilter_kernel(FastParams P) {
+    const Layout& L = P.L;
+    const uint32_t prob = blockIdx.y;
+    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    const SegEntry seg = L.segs[s];
+    if (!seg.fast) return;
+    const FastState* stp = P.state + prob;
+    if (stp->path != PATH_FAST || stp->need2 == 0) return;
+    const uint32_t total = (uint32_t)P.reserve[prob];                 // flagged entries (<= flag_cap on this path)
+    const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
+    const uint2* list = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
+    uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
+    for (uint32_t i = blockIdx.x * THREADS + threadIdx.x; i < total; i += gridDim.x * THREADS) {
+        const uint2 c = list[i];
+        const uint32_t key = c.x & 0x7FFFFFFFu;
+        if (key >= lo2 && key <= hi2) {
+            const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
+            if (pos < LIST2_CAP) out[pos] = make_uint2(key, c.y);
+        }
+    }
+}
+
+// ---- resolve 2: sort the short list, read off the threshold and the tie cut -------------------
+__global__ void __launch_bounds__(THREADS)
+topk_final_kernel(FastParams P) {
+    __shared__ unsigned long long srt[LIST2_CAP];
+    const Layout& L = P.L;
+    const uint32_t prob = blockIdx.x;
+    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    if (!L.segs[s].fast) return;
+    FastState st = P.state[prob];
+    if (st.path != PATH_FAST || st.need2 == 0) return;
+    const uint32_t cnt = st.cnt2;
+    if (cnt != st.T || cnt > LIST2_CAP || st.need2 > cnt) {            // short list disagrees with the histogram
+        if (threadIdx.x == 0) { P.state[prob].path = PATH_FAILED; atomicAdd(P.n_slow, 1u); atomicAdd(P.n_failed, 1u); }
+        return;
+    }
+    uint32_t size = 1;
+    while (size < cnt) size <<= 1;
+    const uint2* in = P.list2 + ((size_t)w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
+    for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
+        unsigned long long v = 0;                                       // padding sorts last
+        if (i < cnt) { const uint2 c = in[i]; v = ((unsigned long long)c.x << 32) | (0xFFFFFFFFu - c.y); }
+        srt[i] = v;
+    }
+    __syncthreads();
+    // bitonic sort, descending: larger key first, equal keys: lower coordinate first
+    for (uint32_t k2 = 2; k2 <= size; k2 <<= 1) {
+        for (uint32_t j = k2 >> 1; j > 0; j >>= 1) {
+            for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
+                const uint32_t ixj = i ^ j;
+                if (ixj > i) {
+                    const unsigned long long a = srt[i], b = srt[ixj];
+                    const bool desc = (i & k2) == 0;
+                    if (desc ? (a < b) : (a > b)) { srt[i] = b; srt[ixj] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) {
+        const unsigned long long v = srt[st.need2 - 1u];
+        st.T = (uint32_t)(v >> 32);
+        st.icut = (0xFFFFFFFFu - (uint32_t)v) + 1u;                  // coordinates below this are kept among the ties
+        if (st.icut == 0) st.icut = 0xFFFFFFFFu;                      // (coordinate 2^32-1 cannot occur: n < 2^32)
+        P.state[prob] = st;
+    }
+}
+
+__device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint32_t icut) {
+    return key > T || (key == T && coord < icut);
+}
+
+// ---- kept count per tile: one warp per tile counts over the tile's flagged slice -------------
+__global__ void __launch_bounds__(THREADS)
+topk_tilecount_kernel(FastParams P) {
+    const Layout& L = P.L;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t item = blockIdx.x * WARPS + (threadIdx.x >> 5);
+    if (item >= P.total_items) return;
+    const uint32_t w = item / L.tiles_per_worker;
+    const uint32_t lt = item - w * L.tiles_per_worker;
+    const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+    const SegEntry seg = L.segs[s];
+    uint32_t kept = 0;
+    if (seg.fast) {
+        const FastState* st = P.state + (size_t)w * L.nseg + s;
+        if (st->path == PATH_FAST) {
+            const uint32_t T = st->T, icut = st->icut;
+            const uint32_t base = P.tile_fbase[item], cnt = P.tile_fcnt[item];
+            const uint2* list = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + base;
+            for (uint32_t i = lane; i < cnt; i += 32) {
+                const uint2 c = list[i];
+                kept += fast_kept(c.x & 0x7FFFFFFFu, c.y, T, icut) ? 1u : 0u;
+            }
+            kept = __reduce_add_sync(0xFFFFFFFFu, kept);
+        }
+    }
+    if (lane == 0) P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
+}
+
+// ---- emit: one warp per tile walks the tile's slice of the flagged list -------------------------
+__global__ void __launch_bounds__(THREADS)
+topk_emit_kernel(FastParams P) {
+    const Layout& L = P.L;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const uint32_t warps_total = gridDim.x * WARPS;
+    for (uint32_t item = blockIdx.x * WARPS + (threadIdx.x >> 5); item < P.total_items; item += warps_total) {
+        const uint32_t cnt = P.tile_fcnt[item];
+        if (cnt == 0u) continue;
+        const uint32_t w = item / L.tiles_per_worker;
+        const uint32_t lt = item - w * L.tiles_per_worker;
+        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+        const SegEntry seg = L.segs[s];
+        if (!seg.fast) continue;
+        const FastState* st = P.state + (size_t)w * L.nseg + s;
+        if (st->path != PATH_FAST) continue;
+        const uint32_t T = st->T, icut = st->icut, hi = st->hi;
+        const uint32_t base = P.tile_fbase[item];
+        const uint32_t* off = P.offsets + (size_t)w * (L.tiles_per_worker + 1);
+        uint32_t running = off[lt] - off[seg.tile_begin];               // kept coordinates of the segment before this tile
+        const uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + base;
+        float* e = P.residuals + (size_t)w * L.n_total + seg.offset;
+        float* ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
+        uint32_t* oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
+        const uint32_t idx0 = (uint32_t)seg.offset;
+        for (uint32_t b = 0; b < cnt; b += 64) {                        // two independent loads in flight per lane
+            const uint32_t i0 = b + lane, i1 = b + 32 + lane;
+            uint2 a0 = make_uint2(0, 0), a1 = make_uint2(0, 0);
+            if (i0 < cnt) a0 = flist[i0];
+            if (i1 < cnt) a1 = flist[i1];
+            const uint32_t k0 = a0.x & 0x7FFFFFFFu, k1 = a1.x & 0x7FFFFFFFu;
+            const bool s0 = i0 < cnt && fast_kept(k0, a0.y, T, icut);
+            const bool s1 = i1 < cnt && fast_kept(k1, a1.y, T, icut);
+            const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, s0), b1 = __ballot_sync(0xFFFFFFFFu, s1);
+            if (s0) {
+                const uint32_t rank = running + __popc(b0 & lt_mask);
+                if (rank < seg.k) { ovals[rank] = __uint_as_float(a0.x); oidx[rank] = idx0 + a0.y; }
+                else atomicMin(P.status, ST_DEVICE_CHECK);
+                if (k0 <= hi) e[a0.y] = 0.0f;                           // a kept candidate: the main pass left p there
+            }
+            running += __popc(b0);
+            if (s1) {
+                const uint32_t rank = running + __popc(b1 & lt_mask);
+                if (rank < seg.k) { ovals[rank] = __uint_as_float(a1.x); oidx[rank] = idx0 + a1.y; }
+                else atomicMin(P.status, ST_DEVICE_CHECK);
+                if (k1 <= hi) e[a1.y] = 0.0f;
+            }
+            running += __popc(b1);
+        }
+    }
+}
+
+// ---- restore: a segment fell back; put the sure values back so that the residual holds p ------
+__global__ void __launch_bounds__(THREADS)
+topk_restore_kernel(FastParams P) {
+    const Layout& L = P.L;
+    if (*P.n_failed == 0u) return;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warps_total = gridDim.x * WARPS;
+    for (uint32_t item = blockIdx.x * WARPS + (threadIdx.x >> 5); item < P.total_items; item += warps_total) {
+        const uint32_t w = item / L.tiles_per_worker;
+        const uint32_t lt = item - w * L.tiles_per_worker;
+        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+        const SegEntry seg = L.segs[s];
+        if (!seg.fast) continue;
+        const FastState* st = P.state + (size_t)w * L.nseg + s;
+        if (st->path != PATH_FAILED) continue;
+        const uint32_t base = P.tile_fbase[item], cnt = P.tile_fcnt[item], hi = st->hi;
+        if (base == 0xFFFFFFFFu || cnt == 0u) continue;                 // nothing was written, nothing was zeroed
+        const uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + base;
+        float* e = P.residuals + (size_t)w * L.n_total + seg.offset;
+        for (uint32_t i = lane; i < cnt; i += 32) {
+            const uint2 a = flist[i];
+            if ((a.x & 0x7FFFFFFFu) > hi) e[a.y] = __uint_as_float(a.x);
+        }
+    }
+}
+
+}  // namespace sc

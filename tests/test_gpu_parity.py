@@ -16,7 +16,7 @@ TILE = 4096
 
 @pytest.fixture(scope="module")
 def ctx():
-    c = sc.Context(max_n=1 << 21, max_W=8, max_segments=64)
+    c = sc.Context(max_n=(1 << 22) + 64, max_W=8, max_segments=64)
     yield c
     c.close()
 
@@ -153,6 +153,57 @@ def test_lstm_like_zero_rows(ctx):
                     e = run_step_both(ctx, scheme, g, e, segs, [wl.step_seed(3, t)] * W)
 
 
+BIG = 1 << 20          # segments of at least this many elements take the sampled-bracket top-k path
+
+
+@pytest.mark.parametrize("n", [BIG, BIG + 5, 3 * BIG + 4099])
+def test_topk_large_segment_all_densities(ctx, n):
+    g = rand(n, 11).view(1, n)
+    e = rand(n, 12).view(1, n)
+    for k in (0, 1, 7, n // 10000, n // 100, n // 10, n // 2, n - 1, n):
+        run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, k)], [0])
+        assert ctx.sc_topk_path_counts() == (0, 1, 0), k       # continuous values: the one-pass path serves it
+
+
+def test_topk_large_segment_misaligned_rows_and_mixed_table(ctx):
+    W, n = 3, BIG + 4099                       # odd row length: rows 1, 2 start misaligned
+    g = torch.stack([rand(n, 900 + w) for w in range(W)])
+    e = torch.stack([rand(n, 950 + w) for w in range(W)])
+    run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, n // 100)], [0] * W)
+    # a table that mixes tiny, medium and large tensors, unaligned starts
+    sizes = [7, BIG + 1, 64, 5000, BIG + BIG // 2 + 3, 33]
+    segs = wl.segment_table(sizes, 1, 100)
+    n2 = sum(sizes)
+    g2 = torch.stack([rand(n2, 960 + w) * (1 + w) for w in range(2)])
+    e2 = torch.stack([rand(n2, 970 + w) for w in range(2)])
+    e2 = run_step_both(ctx, sc.SC_TOPK, g2, e2, segs, [0, 0])
+    assert ctx.sc_topk_path_counts() == (8, 4, 0)
+    run_step_both(ctx, sc.SC_TOPK, g2, e2, segs, [0, 0], use="host")
+
+
+def test_topk_large_segment_degenerate_values_fall_back(ctx):
+    """Inputs on which a sampled bracket cannot isolate the threshold (all equal, mostly
+    zero, few distinct values): the exact result must not depend on that."""
+    n = BIG + 77
+    e = torch.zeros(1, n)
+    eq = torch.full((1, n), -0.5)
+    for k in (1, n // 100, n - 3):
+        run_step_both(ctx, sc.SC_TOPK, eq, e, [(0, n, k)], [0])
+        assert ctx.sc_topk_path_counts() == (0, 0, 1)           # every element ties: the bracket cannot hold
+    z = torch.zeros(1, n)
+    nz = torch.randperm(n, generator=torch.Generator().manual_seed(1))[: n // 20]
+    z[0, nz] = rand(n // 20, 13)
+    for k in (n // 100, n // 20 - 1, n // 20, n // 20 + 1, n // 10):
+        run_step_both(ctx, sc.SC_TOPK, z, e, [(0, n, k)], [0])
+    ints = torch.randint(-3, 4, (1, n), generator=torch.Generator().manual_seed(2)).float()
+    for k in (10, n // 100, n // 3):
+        run_step_both(ctx, sc.SC_TOPK, ints, e, [(0, n, k)], [0])
+    heavy = wl.gen_student_t(n, torch.Generator().manual_seed(3), "cpu").view(1, n)
+    heavy[0, 17] = float("inf"); heavy[0, 4242] = float("nan")
+    for k in (1, 2, 3, n // 1000):
+        run_step_both(ctx, sc.SC_TOPK, heavy, e, [(0, n, k)], [0])
+
+
 def test_aggregate_generic_shared_and_collisions(ctx):
     rng = np.random.default_rng(0)
     W, n, k = 7, 50_001, 5000
@@ -217,7 +268,7 @@ def test_argument_errors_leave_buffers_untouched(ctx):
     assert lib.sc_compress(h, 0, g.data_ptr(), e.data_ptr(), n, n + 1, 0, vals.data_ptr(), idx.data_ptr(), None) == -2
     assert lib.sc_compress(h, 0, None, e.data_ptr(), n, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -1
     assert lib.sc_compress(h, 0, g.data_ptr() + 4, e.data_ptr(), n - 1, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -1
-    assert lib.sc_compress(h, 0, g.data_ptr(), e.data_ptr(), (1 << 21) + 1, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -2
+    assert lib.sc_compress(h, 0, g.data_ptr(), e.data_ptr(), (1 << 22) + 65, k, 0, vals.data_ptr(), idx.data_ptr(), None) == -2
     assert lib.sc_aggregate(h, 0, vals.data_ptr(), idx.data_ptr(), k, n, e.data_ptr(), None) == -2
     assert lib.sc_aggregate(h, 1, vals.data_ptr(), idx.data_ptr(), n + 1, n, e.data_ptr(), None) == -2
     torch.cuda.synchronize()
