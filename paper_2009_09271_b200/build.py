@@ -10,8 +10,15 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparsecomm.so")
 SOURCES = ["sc_api.cu"]
-HEADERS = ["sc_common.cuh", "sc_topk.cuh", "sc_pack.cuh", "sc_random.cuh", "sc_aggregate.cuh",
-           os.path.join("..", "..", "include", "sparsecomm.h")]
+
+
+def _dependencies():
+    """Every file under csrc/ plus the public header."""
+    deps = [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC)) if f.endswith((".cu", ".cuh", ".h"))]
+    deps.append(os.path.join(HERE, "..", "include", "sparsecomm.h"))
+    deps.append(os.path.abspath(__file__))
+    return deps
+
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-lineinfo",
@@ -33,8 +40,7 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.abspath(__file__)]
-    return any(os.path.getmtime(d) > t for d in deps)
+    return any(os.path.getmtime(d) > t for d in _dependencies())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

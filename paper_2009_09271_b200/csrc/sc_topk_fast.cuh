@@ -138,25 +138,30 @@ topk_bracket_kernel(FastParams P) {
         atomicAdd(&h0[k.z >> 20], 1u); atomicAdd(&h0[k.w >> 20], 1u);
     }
     __syncthreads();
+    // when k is so small that no sample rank lies safely above the threshold there is no "sure"
+    // set (hi stays at the largest key); the candidate histogram then spans up to the largest
+    // sample key and everything above it shares the last bin
+    const uint32_t rankA = have_hi ? (uint32_t)j_hi : 1u;
     uint32_t binA = 0, needA = 0, binB = 0, needB = 0, cnt = 0;
-    if (have_hi) find_from_top<HIST0_BINS>(h0, (uint32_t)j_hi, s_tmp, binA, needA, cnt);
+    find_from_top<HIST0_BINS>(h0, rankA, s_tmp, binA, needA, cnt);
     if (have_lo) find_from_top<HIST0_BINS>(h0, (uint32_t)j_lo, s_tmp, binB, needB, cnt);
     for (uint32_t i = threadIdx.x; i < m / 4u; i += THREADS) {
         const uint4 k = smp[i];
         const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            if (have_hi && (kk[c] >> 20) == binA) atomicAdd(&hA[(kk[c] >> 10) & 1023u], 1u);
+            if ((kk[c] >> 20) == binA) atomicAdd(&hA[(kk[c] >> 10) & 1023u], 1u);
             if (have_lo && (kk[c] >> 20) == binB) atomicAdd(&hB[(kk[c] >> 10) & 1023u], 1u);
         }
     }
     __syncthreads();
-    uint32_t hi = 0x7FFFFFFFu, lo = 0u, bin1 = 0, need1 = 0;
-    if (have_hi && find_from_top<1024>(hA, needA, s_tmp, bin1, need1, cnt)) hi = (binA << 20) | (bin1 << 10) | 1023u;
+    uint32_t top = 0x7FFFFFFFu, lo = 0u, bin1 = 0, need1 = 0;
+    if (find_from_top<1024>(hA, needA, s_tmp, bin1, need1, cnt)) top = (binA << 20) | (bin1 << 10) | 1023u;
     if (have_lo && find_from_top<1024>(hB, needB, s_tmp, bin1, need1, cnt)) lo = (binB << 20) | (bin1 << 10);
-    if (lo > hi) lo = hi;                                              // (cannot happen; keeps the bracket sane)
+    const uint32_t hi = have_hi ? top : 0x7FFFFFFFu;
+    if (lo > top) lo = top;                                            // (cannot happen; keeps the bracket sane)
     if (threadIdx.x == 0) {
-        const uint32_t width_m1 = hi - lo;
+        const uint32_t width_m1 = top - lo;
         const uint32_t bits = width_m1 ? 32u - (uint32_t)__clz((int)width_m1) : 0u;
         FastState st = {};
         st.path = PATH_FAST; st.lo = lo; st.hi = hi; st.shift = bits > 11u ? bits - 11u : 0u;
