@@ -50,10 +50,15 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
     __shared__ float st_val[AGG_STAGE];
     __shared__ uint32_t s_lo[64], s_off[65];
     const float fW = (float)W;
+    // Dividing by a power of two equals multiplying by its (exact) reciprocal, bit for bit, and an
+    // IEEE division costs about ten instructions: take the product when W allows it.
+    const bool pow2 = (W & (W - 1u)) == 0u;
+    const float rW = 1.0f / fW;
     for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
         const uint32_t tile_lo = t * ATILE;
         const uint32_t tile_n = min(ATILE, n - tile_lo);
-        for (uint32_t i = threadIdx.x; i < ATILE; i += THREADS) acc[i] = 0.0f;
+        for (uint32_t i = threadIdx.x; i < ATILE / 4; i += THREADS)
+            reinterpret_cast<float4*>(acc)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         if (shared_idx) {
             const uint32_t lo = bounds[t], hi = bounds[t + 1];
             __syncthreads();
@@ -115,11 +120,12 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
         if (tile_n == ATILE) {
             for (uint32_t i = threadIdx.x; i < ATILE / 4; i += THREADS) {
                 float4 a = reinterpret_cast<const float4*>(acc)[i];
-                a.x = a.x / fW; a.y = a.y / fW; a.z = a.z / fW; a.w = a.w / fW;
+                if (pow2) { a.x *= rW; a.y *= rW; a.z *= rW; a.w *= rW; }
+                else { a.x = a.x / fW; a.y = a.y / fW; a.z = a.z / fW; a.w = a.w / fW; }
                 __stcs(reinterpret_cast<float4*>(o) + i, a);
             }
         } else {
-            for (uint32_t i = threadIdx.x; i < tile_n; i += THREADS) o[i] = acc[i] / fW;
+            for (uint32_t i = threadIdx.x; i < tile_n; i += THREADS) o[i] = pow2 ? acc[i] * rW : acc[i] / fW;
         }
         __syncthreads();
     }

@@ -187,34 +187,47 @@ __device__ inline uint32_t warp_inclusive_scan(uint32_t v, uint32_t lane) {
 }
 __device__ inline uint32_t bytes_sum(uint32_t v) { return (v & 0xFFu) + ((v >> 8) & 0xFFu) + ((v >> 16) & 0xFFu) + (v >> 24); }
 
-__global__ void __launch_bounds__(THREADS, 4)
+__global__ void __launch_bounds__(THREADS)
 topk_main_kernel(FastParams P) {
     __shared__ uint32_t sh[CAND_BINS];
-    __shared__ uint32_t s_wsure[2][WARPS], s_wcand[2][WARPS], s_wflag[2][WARPS];
+    __shared__ __align__(16) float s_p[QUADS][THREADS][4];           // the tile's p values, for the rare per-element work
+    __shared__ uint32_t s_wflag[2][WARPS], s_wcand[2][WARPS];
     __shared__ unsigned long long s_base[2];
+    __shared__ uint32_t s_red[WARPS + 1];
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) sh[b] = 0;
     __syncthreads();
     long long cur_prob = -1;
     size_t cur_fidx = 0;
-    uint32_t lo = 0, hi = 0, shift = 0, parity = 0;
-    for (uint32_t item = blockIdx.x; item < P.total_items; item += gridDim.x) {
-        const uint32_t w = item / L.tiles_per_worker;
-        const uint32_t lt = item - w * L.tiles_per_worker;
-        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-        const SegEntry seg = L.segs[s];
-        if (!seg.fast) continue;                                       // uniform over the CTA
-        const long long prob = (long long)w * L.nseg + s;
-        if (prob != cur_prob) {
-            if (cur_prob >= 0) {
-                __syncthreads();
-                for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
-                    const uint32_t c = sh[b];
-                    if (c) { atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c); sh[b] = 0; }
-                }
-                __syncthreads();
+    uint32_t lo = 0, hi = 0, shift = 0, parity = 0, my_sure = 0;
+    for (uint32_t item = blockIdx.x; ; item += gridDim.x) {
+        // ---- which tile; flush the per-segment accumulators when the segment changes -------------
+        bool have = item < P.total_items;
+        uint32_t w = 0, lt = 0, s = 0;
+        SegEntry seg{};
+        if (have) {
+            w = item / L.tiles_per_worker;
+            lt = item - w * L.tiles_per_worker;
+            s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+            seg = L.segs[s];
+        }
+        const long long prob = have ? (long long)w * L.nseg + s : -2;
+        if (prob != cur_prob && cur_prob >= 0) {                       // uniform over the CTA
+            uint32_t total;
+            block_exclusive_scan(my_sure, s_red, &total);              // (only the total is used)
+            if (threadIdx.x == 0 && total) atomicAdd(&P.state[cur_prob].sure_total, total);
+            for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
+                const uint32_t c = sh[b];
+                if (c) { atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c); sh[b] = 0; }
             }
+            __syncthreads();
+            my_sure = 0;
+            cur_prob = -1;
+        }
+        if (!have) break;
+        if (!seg.fast) continue;                                       // uniform over the CTA
+        if (prob != cur_prob) {
             cur_prob = prob;
             cur_fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
             const FastState st = P.state[prob];
@@ -230,8 +243,8 @@ topk_main_kernel(FastParams P) {
         const long long mine = first + warp * 512 + lane * 4;            // quad of row 0; row j at + 128 j
         const bool full = first >= 0 && first + TILE <= (long long)seg.n;
 
-        float p[QUADS][4];
-        uint32_t valid16 = 0;
+        // ---- stream: p = g + e goes straight back to the residual and into shared memory ------------
+        uint32_t flag16 = 0;                                           // bit 4 j + c: key >= lo
         if (full) {
             float4 ev[QUADS], gv[QUADS];
 #pragma unroll
@@ -241,46 +254,49 @@ topk_main_kernel(FastParams P) {
             }
 #pragma unroll
             for (int j = 0; j < QUADS; ++j) {
-                p[j][0] = gv[j].x + ev[j].x; p[j][1] = gv[j].y + ev[j].y;
-                p[j][2] = gv[j].z + ev[j].z; p[j][3] = gv[j].w + ev[j].w;
+                const float4 p = make_float4(gv[j].x + ev[j].x, gv[j].y + ev[j].y, gv[j].z + ev[j].z, gv[j].w + ev[j].w);
+                *reinterpret_cast<float4*>(e + mine + 128 * j) = p;
+                *reinterpret_cast<float4*>(&s_p[j][threadIdx.x][0]) = p;
+                flag16 |= (uint32_t)(key_of(p.x) >= lo) << (4 * j) | (uint32_t)(key_of(p.y) >= lo) << (4 * j + 1) |
+                          (uint32_t)(key_of(p.z) >= lo) << (4 * j + 2) | (uint32_t)(key_of(p.w) >= lo) << (4 * j + 3);
             }
-            valid16 = 0xFFFFu;
         } else {
 #pragma unroll
             for (int j = 0; j < QUADS; ++j) {
                 const long long base = mine + 128 * j;
-                float gq[4];
-                const uint32_t valid = load_quad(e, base, seg.n, p[j]);
+                float p[4], gq[4];
+                const uint32_t valid = load_quad(e, base, seg.n, p);
                 load_quad_stream(g, base, seg.n, gq);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) p[j][c] = gq[c] + p[j][c];
-                valid16 |= valid << (4 * j);
+                for (int c = 0; c < 4; ++c) {
+                    p[c] = gq[c] + p[c];
+                    flag16 |= (((valid >> c) & 1u) & (uint32_t)(key_of(p[c]) >= lo)) << (4 * j + c);
+                }
+                if (valid) store_quad(e, base, valid, p);
+                *reinterpret_cast<float4*>(&s_p[j][threadIdx.x][0]) = make_float4(p[0], p[1], p[2], p[3]);
             }
         }
-        // classify
-        uint32_t flag16 = 0, sure16 = 0;
-#pragma unroll
-        for (int j = 0; j < QUADS; ++j)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t key = key_of(p[j][c]);
-                flag16 |= (uint32_t)(key >= lo) << (4 * j + c);
-                sure16 |= (uint32_t)(key > hi) << (4 * j + c);
-            }
-        flag16 &= valid16; sure16 &= valid16;
-        const uint32_t cand16 = flag16 & ~sure16;
-        // ranks of the flagged elements inside the warp, in coordinate order
+        // ---- ranks of the flagged elements, in coordinate order ---------------------------------------
         const uint32_t fcnt4 = pack_counts(flag16);
         const uint32_t finc4 = warp_inclusive_scan(fcnt4, lane);
         const uint32_t ftot4 = __shfl_sync(0xFFFFFFFFu, finc4, 31);
-        const uint32_t wcand = __reduce_add_sync(0xFFFFFFFFu, __popc(cand16));
-        const uint32_t wsure = __reduce_add_sync(0xFFFFFFFFu, __popc(sure16));
-        if (lane == 0) { s_wsure[parity][warp] = wsure; s_wcand[parity][warp] = wcand; s_wflag[parity][warp] = bytes_sum(ftot4); }
+        const uint32_t ex4 = finc4 - fcnt4;
+        // candidates (lo <= key <= hi) are counted from shared memory, only by lanes that have a flag
+        uint32_t ccnt = 0;
+        {
+            uint32_t bits = flag16;
+            while (bits) {
+                const uint32_t i = (uint32_t)__ffs((int)bits) - 1u;
+                bits &= bits - 1u;
+                ccnt += key_of(s_p[i >> 2][threadIdx.x][i & 3u]) <= hi ? 1u : 0u;
+            }
+        }
+        const uint32_t wcand = __reduce_add_sync(0xFFFFFFFFu, ccnt);
+        if (lane == 0) { s_wflag[parity][warp] = bytes_sum(ftot4); s_wcand[parity][warp] = wcand; }
         __syncthreads();
-        uint32_t tsure = 0, tcand = 0, tflag = 0, fwbase = 0;
+        uint32_t tcand = 0, tflag = 0, fwbase = 0;
 #pragma unroll
         for (int i = 0; i < WARPS; ++i) {
-            tsure += s_wsure[parity][i];
             const uint32_t f = s_wflag[parity][i];
             fwbase += (i < (int)warp) ? f : 0u;
             tcand += s_wcand[parity][i]; tflag += f;
@@ -288,63 +304,33 @@ topk_main_kernel(FastParams P) {
         if (threadIdx.x == 0) {
             unsigned long long base = 0;
             if (tflag) base = atomicAdd(P.reserve + prob, ((unsigned long long)tcand << 32) | tflag);
-            const uint32_t fbase = (uint32_t)base;
-            const bool fits = (unsigned long long)fbase + tflag <= seg.flag_cap;
-            if (tsure && fits) atomicAdd(&P.state[prob].sure_total, tsure);
-            P.tile_fbase[item] = fits ? fbase : 0xFFFFFFFFu; P.tile_fcnt[item] = tflag;
+            const bool fits = (unsigned long long)(uint32_t)base + tflag <= seg.flag_cap;
+            P.tile_fbase[item] = fits ? (uint32_t)base : 0xFFFFFFFFu;
+            P.tile_fcnt[item] = tflag;
             s_base[parity] = fits ? base : ~0ull;
         }
-        bool fits = true;
         if (tflag) {                                                   // uniform over the CTA
             __syncthreads();
             const unsigned long long base = s_base[parity];
-            fits = base != ~0ull;
-            if (fits && flag16) {
-                uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
-                uint32_t rowbase = (uint32_t)base + fwbase;
-#pragma unroll
-                for (int j = 0; j < QUADS; ++j) {
-                    uint32_t slot = rowbase + ((finc4 - fcnt4) >> (8 * j) & 0xFFu);
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if ((flag16 >> (4 * j + c)) & 1u)
-                            flist[slot++] = make_uint2(__float_as_uint(p[j][c]), (uint32_t)(mine + 128 * j + c));
-                    rowbase += (ftot4 >> (8 * j)) & 0xFFu;
+            if (base != ~0ull && flag16) {
+                // the tile's entries fit: write them, zero the sure ones in the residual (their values
+                // stay in the list, from where a fall-back restores them), histogram the candidates
+                uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + (uint32_t)base + fwbase;
+                uint32_t bits = flag16;
+                while (bits) {
+                    const uint32_t i = (uint32_t)__ffs((int)bits) - 1u;
+                    bits &= bits - 1u;
+                    const uint32_t j = i >> 2;
+                    const float v = s_p[j][threadIdx.x][i & 3u];
+                    const uint32_t key = key_of(v);
+                    const uint32_t rowbase = bytes_sum(ftot4 & ((1u << (8u * j)) - 1u));
+                    const uint32_t slot = rowbase + ((ex4 >> (8u * j)) & 0xFFu) + __popc(flag16 & ((1u << i) - 1u) & (0xFu << (4u * j)));
+                    const uint32_t coord = (uint32_t)(mine + 128 * (long long)j + (i & 3u));
+                    flist[slot] = make_uint2(__float_as_uint(v), coord);
+                    if (key > hi) { e[coord] = 0.0f; ++my_sure; }
+                    else atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
                 }
             }
-            if (fits && cand16) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if ((cand16 >> i) & 1u)
-                        atomicAdd(&sh[min((key_of(p[i >> 2][i & 3]) - lo) >> shift, CAND_BINS - 1u)], 1u);
-            }
-        }
-        // residual: sure elements are certainly kept, so they become zero right here (only if
-        // their values made it into the flagged list, from where a fall-back can restore them)
-        if (fits && sure16) {
-#pragma unroll
-            for (int j = 0; j < QUADS; ++j)
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if ((sure16 >> (4 * j + c)) & 1u) p[j][c] = 0.0f;
-        }
-        if (full) {
-#pragma unroll
-            for (int j = 0; j < QUADS; ++j)
-                *reinterpret_cast<float4*>(e + mine + 128 * j) = make_float4(p[j][0], p[j][1], p[j][2], p[j][3]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < QUADS; ++j) {
-                const uint32_t valid = (valid16 >> (4 * j)) & 0xFu;
-                if (valid) store_quad(e, mine + 128 * j, valid, p[j]);
-            }
-        }
-    }
-    if (cur_prob >= 0) {
-        __syncthreads();
-        for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
-            const uint32_t c = sh[b];
-            if (c) atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c);
         }
     }
 }
