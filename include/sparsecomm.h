@@ -120,6 +120,27 @@ int sc_aggregate(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, siz
 int sc_aggregate_shared(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
                         float* out, void* stream);
 
+/* The paper has no counterpart for this entry point: it is sc_aggregate for callers that
+ * are not allowed to allocate device memory.  Every other entry point needs an sc_ctx, and
+ * sc_create calls cudaMalloc.  That rules the library out for code that runs after a
+ * framework has handed all free device memory to its own pool (a later cudaMalloc fails),
+ * and for code inside a latency-critical section, since cudaMalloc may synchronise the
+ * whole device.  sc_aggregate_static needs no context and calls no cudaMalloc, cudaFree or
+ * any other allocating routine: its scratch (the per-tile message bounds, about 1 MB) is a
+ * fixed __device__ array inside the library, present on every GPU that loads the library
+ * until the process exits.
+ *   - Same arguments and result as sc_aggregate, same bits, for W <= 64 and
+ *     n <= 16,777,216.  Anything larger returns SC_ERR_RANGE before touching a buffer.
+ *   - The first call on a device looks up the array's address on that device (the device
+ *     must be current) and remembers it; make that first call before any stream capture.
+ *   - All calls on one GPU share the one array, which keeps the previous call's contents
+ *     (what has to start at zero is cleared on `stream` by the call itself).  Two calls
+ *     whose kernels can overlap on the GPU (different streams, no ordering) race on it.
+ *   - A message that breaks the ascending-coordinate rule is skipped silently here: there
+ *     is no context whose status word could report it. */
+int sc_aggregate_static(int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                        float* out, void* stream);
+
 /* One whole step: sc_compress_batch followed by the aggregate over the W
  * messages it produced (the shared-coordinate form when all seeds are equal and
  * the scheme is not top-k).  out[n] receives the dense average. */

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libsparsecomm.so")
 
 EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_scratch_bytes", "sc_launch_count",
            "sc_topk_path_counts", "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
-           "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_step", "sc_step_host"]
+           "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_aggregate_static", "sc_step", "sc_step_host"]
 
 
 class ScSegment(ctypes.Structure):
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.sc_aggregate.restype = ci
     lib.sc_aggregate_shared.argtypes = [vp, ci, vp, vp, sz, sz, vp, vp]
     lib.sc_aggregate_shared.restype = ci
+    lib.sc_aggregate_static.argtypes = [ci, vp, vp, sz, sz, vp, vp]
+    lib.sc_aggregate_static.restype = ci
     lib.sc_step.argtypes = [vp, ci, ci, vp, vp, sz, ctypes.POINTER(ScSegment), ci, ctypes.POINTER(u64),
                             vp, vp, vp, vp]
     lib.sc_step.restype = ci
@@ -121,6 +123,22 @@ def _check(code: int, what: str) -> None:
 def _want(t: torch.Tensor, dtype, name: str, cuda: bool = True) -> None:
     if t.dtype != dtype or not t.is_contiguous() or (cuda and not t.is_cuda):
         raise TypeError(f"{name}: expected a contiguous {'CUDA ' if cuda else ''}{dtype} tensor")
+
+
+STATIC_MAX_N, STATIC_MAX_W = 1 << 24, 64
+
+
+def sc_aggregate_static(W: int, vals, idx, k: int, n: int, out, stream=None) -> None:
+    """sc_aggregate without a Context, for callers that may not allocate device memory (the
+    library's own scratch for it is a fixed device array).  Limits: W <= 64, n <= 2**24.
+    All calls on one GPU share that scratch, so calls that may overlap on the GPU race."""
+    lib = load_library()
+    _want(vals, torch.float32, "vals"), _want(idx, torch.int32, "idx"), _want(out, torch.float32, "out")
+    if vals.numel() < W * k or idx.numel() < W * k or out.numel() < n:
+        raise ValueError("buffer sizes do not match W, k and n")
+    code = lib.sc_aggregate_static(W, _ptr(vals), _ptr(idx), k, n, _ptr(out), _stream(stream))
+    if code != 0:
+        raise SparseCommError(code, f"sc_aggregate_static (limits: W <= {STATIC_MAX_W}, n <= {STATIC_MAX_N})")
 
 
 class Context:

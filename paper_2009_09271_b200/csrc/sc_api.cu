@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -668,6 +669,73 @@ int sc_step_host(sc_ctx* c, int scheme, int W, const float* h_grads, float* resi
     if (rc != SC_OK) return rc;
     SC_CUDA(cudaMemcpyAsync(h_out, c->d_stage_out, n * sizeof(float), cudaMemcpyDeviceToHost, st));
     SC_CUDA(cudaStreamSynchronize(st));
+    return SC_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// sc_aggregate_static: the aggregate without a context, for callers that must not allocate.
+// Its scratch (the per-tile message bounds and a status word) lives in the fixed array below,
+// which every GPU that loads this library holds until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticMaxN = (size_t)1 << 24;                 // coordinates of the dense output
+constexpr int kStaticMaxW = 64;                                   // workers
+constexpr size_t kStaticTiles = kStaticMaxN / ATILE;
+constexpr size_t kStaticBoundsWords = (size_t)kStaticMaxW * (kStaticTiles + 1);
+constexpr size_t kStaticBytes = kStaticBoundsWords * sizeof(uint32_t) + 256;   // bounds, then the status word
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticDevice { unsigned char* base = nullptr; int sm_count = 0; };
+StaticDevice g_static_dev[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Looks up, once per device and with that device current, where the array lives on it.
+int static_scratch_for_current_device(StaticDevice* out) {
+    int dev = -1;
+    SC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDevice& d = g_static_dev[dev];
+    if (!d.base) {
+        void* ptr = nullptr;
+        SC_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        int sms = 0;
+        SC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        if (!ptr || sms <= 0) return SC_ERR_CUDA;
+        d.sm_count = sms;
+        d.base = static_cast<unsigned char*>(ptr);
+    }
+    *out = d;
+    return SC_OK;
+}
+
+}  // namespace
+
+int sc_aggregate_static(int W, const float* vals, const uint32_t* idx, size_t k, size_t n, float* out, void* stream) {
+    if (W < 1 || W > kStaticMaxW || n > kStaticMaxN || k > n) return SC_ERR_RANGE;
+    if ((n > 0 && !out) || (k > 0 && (!vals || !idx)) || !aligned16(out)) return SC_ERR_INVALID;
+    if (n == 0) return SC_OK;
+    StaticDevice d;
+    int rc = static_scratch_for_current_device(&d);
+    if (rc != SC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t* bounds = reinterpret_cast<uint32_t*>(d.base);
+    int* status = reinterpret_cast<int*>(d.base + kStaticBoundsWords * sizeof(uint32_t));
+    // the array keeps whatever the previous call left: the bounds in use are rewritten below,
+    // the status word has to start at zero
+    SC_CUDA(cudaMemsetAsync(status, 0, sizeof(int), st));
+    const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
+    const uint64_t threads = (uint64_t)W * (ntiles + 1ull);
+    agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, st>>>(
+        idx, (uint32_t)W, (uint32_t)k, ntiles, bounds);
+    const uint32_t grid = std::max(1u, std::min<uint32_t>(ntiles, (uint32_t)d.sm_count * 4u));
+    agg_tiles_kernel<<<grid, THREADS, 0, st>>>(vals, idx, bounds, (uint32_t)W, 0u, (uint32_t)k, (uint32_t)n, ntiles,
+                                               out, status);
+    SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
 
