@@ -47,7 +47,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-div", type=int, default=4, help="oracle sample = n / this of one worker")
+    ap.add_argument("--cpu-sample-div", type=int, default=1, help="oracle sample = n / this of one worker")
+    ap.add_argument("--selftest-dist", action="store_true",
+                    help="CPU-only check of the multi-rank plumbing (gloo): barrier, max over ranks, aggregate value")
     return ap.parse_args()
 
 
@@ -138,6 +140,52 @@ def step_min_bytes(scheme: str, n: int, W: int, K: int, shared: bool) -> float:
     return 12.0 * n * W + 8.0 * K * W + 8.0 * K + 4.0 * n
 
 
+class Ranks:
+    """Process-group plumbing of the benchmark: one process per GPU, no data-path collective.
+    Only the timing is reduced (max over ranks) and the per-rank work summed."""
+
+    def __init__(self, world: int, backend: str, device=None):
+        self.world, self.dist, self.device = world, None, device
+        if world > 1:
+            import torch.distributed as dist
+            kwargs = {"device_id": device} if backend == "nccl" and device is not None else {}
+            dist.init_process_group(backend, **kwargs)
+            self.dist = dist
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+
+    def max_ms(self, ms: float) -> float:
+        if self.dist is None:
+            return ms
+        import torch
+        t = torch.tensor([ms], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def whole_job_value(self, units_per_rank_per_step: float, steps: int, ms: float) -> float:
+        """Units all ranks processed divided by the slowest rank's time."""
+        return self.world * units_per_rank_per_step * steps / (self.max_ms(ms) * 1e-3)
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.barrier()
+            self.dist.destroy_process_group()
+
+
+def run_selftest_dist(args, rank: int, world: int):
+    """No GPU: every rank pretends to have timed `steps` steps in (10 + 5 rank) ms."""
+    ranks = Ranks(world, "gloo")
+    ranks.barrier()
+    value = ranks.whole_job_value(1000.0, args.steps, 10.0 + 5.0 * rank)
+    ranks.barrier()
+    if rank == 0:
+        print(json.dumps({"selftest": "dist", "n_gpus": world, "value": value,
+                          "max_ms": 10.0 + 5.0 * (world - 1)}), flush=True)
+    ranks.close()
+
+
 def build_problem(args):
     import workloads as wl
     w = wl.workload(args.workload)
@@ -202,16 +250,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
+    ranks = Ranks(world, "nccl", dev)
 
     def barrier():
         torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
+        ranks.barrier()
         torch.cuda.synchronize()
 
     w, sizes, W, schemes, segs, (num, den) = build_problem(args)
@@ -274,10 +317,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     status = ctx.sc_sync_status()
     if status != 0:
         raise RuntimeError(f"device status after the timed region: {sc.strerror(status)}")
-    if dist is not None:
-        tmax = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
+    elapsed_ms = ranks.max_ms(elapsed_ms)
 
     # per-scheme device time from the marks
     per_scheme_ms = {s: 0.0 for s in schemes}
@@ -346,9 +386,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         line["cpu_baseline"] = run_cpu_baseline(args, wl, w, sizes, schemes, num, den, grads[0])
 
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    ranks.close()
     if rank == 0:
         print(json.dumps(line), flush=True)
 
@@ -414,6 +452,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.selftest_dist:
+        run_selftest_dist(args, rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, rank)
         return

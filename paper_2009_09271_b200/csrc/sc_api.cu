@@ -547,16 +547,6 @@ int sc_topk_path_counts(sc_ctx* c, void* stream, uint32_t* h_counts) {
     return SC_OK;
 }
 
-int sc_debug_fast_state(sc_ctx* c, void* stream, uint32_t problem, uint32_t* h_words) {
-    if (!c || !h_words || problem >= c->last_topk_problems) return SC_ERR_INVALID;
-    DeviceGuard guard(c->device);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    SC_CUDA(cudaMemcpyAsync(h_words, c->d_fstate + problem, sizeof(FastState), cudaMemcpyDeviceToHost, st));
-    SC_CUDA(cudaMemcpyAsync(h_words + 16, c->d_reserve + problem, 8, cudaMemcpyDeviceToHost, st));
-    SC_CUDA(cudaStreamSynchronize(st));
-    return SC_OK;
-}
-
 size_t sc_scratch_bytes(const sc_ctx* c) { return c ? c->scratch_bytes : 0; }
 uint64_t sc_launch_count(const sc_ctx* c) { return c ? c->launches : 0; }
 
