@@ -54,7 +54,7 @@ struct sc_ctx {
     uint32_t last_topk_problems = 0; // (worker, segment) pairs of the most recent top-k call
     uint32_t slow_segments = 0;      // segments of the cached table that take the radix-select path
     uint32_t max_sample_m = 0;
-    uint32_t max_flag_cap = 0;
+    uint32_t max_flag_cap = 0, max_cand_cap = 0;
     int occ_main = 1, occ_emit = 1;
     uint64_t* d_seeds = nullptr;
     int* d_status = nullptr;
@@ -177,6 +177,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             e.flag_begin = flag;
             flag += e.flag_cap;
             max_cap = std::max(max_cap, e.flag_cap);
+            c->max_cand_cap = std::max(c->max_cand_cap, e.cand_cap);
             max_m = std::max(max_m, e.sample_m);
         } else {
             ++slow_count;
@@ -265,10 +266,12 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             FastParams fp{};
             fp.L = L; fp.grads = grads; fp.residuals = residuals; fp.out_vals = out_vals; fp.out_idx = out_idx;
             fp.state = c->d_fstate; fp.sample = c->d_sample; fp.cand_hist = c->d_cand_hist;
-            fp.list2 = c->d_list2; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
+            fp.list2 = c->d_list2; fp.cand = c->d_cand; fp.tile_sure = c->d_tile_sure; fp.tile_cbase = c->d_tile_cbase;
+            fp.tile_ccnt = c->d_tile_ccnt; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
             fp.flagged = c->d_flagged; fp.reserve = c->d_reserve; fp.offsets = c->d_offsets;
             fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
             SC_CUDA(cudaMemsetAsync(c->d_reserve, 0, (size_t)P * sizeof(unsigned long long), stream));
+            SC_CUDA(cudaMemsetAsync(c->d_tile_sure, 0, (size_t)items * sizeof(uint32_t), stream));
             SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
             { Launch l(c, KIND_SAMPLE, stream);
               topk_sample_kernel<<<dim3((c->max_sample_m / 8 + THREADS - 1) / THREADS, P), THREADS, 0, stream>>>(fp); }
@@ -279,7 +282,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             { Launch l(c, KIND_CANDBIN, stream);
               topk_candbin_kernel<<<P, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDFILTER, stream);
-              const uint32_t gx = std::min<uint32_t>((c->max_flag_cap + THREADS * 4 - 1) / (THREADS * 4), 2048u);
+              const uint32_t gx = std::min<uint32_t>((c->max_cand_cap + THREADS * 4 - 1) / (THREADS * 4), 1024u);
               topk_candfilter_kernel<<<dim3(std::max(gx, 1u), P), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_FINAL, stream);
               topk_final_kernel<<<P, THREADS, 0, stream>>>(fp); }
@@ -287,7 +290,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
               topk_restore_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_TILECOUNT, stream);
-              topk_tilecount_kernel<<<(items + WARPS - 1) / WARPS, THREADS, 0, stream>>>(fp); }
+              topk_tilecount_kernel<<<(uint32_t)(((uint64_t)items * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_ROW_SCAN, stream);
               row_scan_kernel<<<W, THREADS, 0, stream>>>(c->d_offsets, L.tiles_per_worker); }
             { Launch l(c, KIND_EMIT, stream);
@@ -448,6 +451,10 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_sample, fastP * SAMPLE_MAX)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_cand_hist, fastP * CAND_BINS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_list2, fastP * LIST2_CAP)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_cand, (size_t)max_W * c->max_cand_per_worker)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tile_sure, items_max)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tile_cbase, items_max)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tile_ccnt, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_fbase, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_fcnt, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_reserve, P)) == SC_OK &&

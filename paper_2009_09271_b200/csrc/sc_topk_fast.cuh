@@ -38,6 +38,10 @@ struct FastParams {
     uint32_t* cand_hist;       // [W * fast_per_worker][CAND_BINS]
     uint2* list2;              // [W * fast_per_worker][LIST2_CAP]
     uint2* flagged;            // [W][flag_per_worker] (value bits, coordinate inside the segment)
+    uint2* cand;               // [W][cand_per_worker] (key, coordinate) of the candidates, any order inside a tile
+    uint32_t* tile_sure;       // [W * tiles_per_worker] sure elements of the tile (zeroed before the pass)
+    uint32_t* tile_cbase;      // first candidate slot of the tile
+    uint32_t* tile_ccnt;       // candidates of the tile
     uint32_t* tile_fbase;      // first flagged slot of the tile (0xFFFFFFFF: the list was full, nothing written)
     uint32_t* tile_fcnt;       // flagged elements of the tile
     unsigned long long* reserve;   // [W * nseg]: candidates reserved << 32 | flagged reserved
@@ -193,6 +197,7 @@ topk_main_kernel(FastParams P) {
     __shared__ __align__(16) float s_p[QUADS][THREADS][4];           // the tile's p values, for the rare per-element work
     __shared__ uint32_t s_wflag[2][WARPS], s_wcand[2][WARPS];
     __shared__ unsigned long long s_base[2];
+    __shared__ uint32_t s_crun[2];                                    // running candidate slot inside the tile
     __shared__ uint32_t s_red[WARPS + 1];
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -304,10 +309,14 @@ topk_main_kernel(FastParams P) {
         if (threadIdx.x == 0) {
             unsigned long long base = 0;
             if (tflag) base = atomicAdd(P.reserve + prob, ((unsigned long long)tcand << 32) | tflag);
-            const bool fits = (unsigned long long)(uint32_t)base + tflag <= seg.flag_cap;
+            const bool fits = (unsigned long long)(uint32_t)base + tflag <= seg.flag_cap &&
+                              (base >> 32) + tcand <= seg.cand_cap;
             P.tile_fbase[item] = fits ? (uint32_t)base : 0xFFFFFFFFu;
             P.tile_fcnt[item] = tflag;
+            P.tile_cbase[item] = (uint32_t)(base >> 32);
+            P.tile_ccnt[item] = fits ? tcand : 0u;
             s_base[parity] = fits ? base : ~0ull;
+            s_crun[parity] = (uint32_t)(base >> 32);
         }
         if (tflag) {                                                   // uniform over the CTA
             __syncthreads();
@@ -316,20 +325,30 @@ topk_main_kernel(FastParams P) {
                 // the tile's entries fit: write them, zero the sure ones in the residual (their values
                 // stay in the list, from where a fall-back restores them), histogram the candidates
                 uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + (uint32_t)base + fwbase;
-                uint32_t bits = flag16;
+                uint2* clist = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin;
+                uint32_t bits = flag16, sure_here = 0;
+                // first slot of this lane's quad in each row, relative to the warp's slice (< 512: 16 bits each)
+                const uint32_t r0 = ftot4 & 0xFFu, r1 = (ftot4 >> 8) & 0xFFu, r2 = (ftot4 >> 16) & 0xFFu;
+                const uint32_t q01 = (ex4 & 0xFFu) | ((r0 + ((ex4 >> 8) & 0xFFu)) << 16);
+                const uint32_t q23 = (r0 + r1 + ((ex4 >> 16) & 0xFFu)) | ((r0 + r1 + r2 + (ex4 >> 24)) << 16);
+                const uint32_t mine32 = (uint32_t)mine;
                 while (bits) {
                     const uint32_t i = (uint32_t)__ffs((int)bits) - 1u;
                     bits &= bits - 1u;
                     const uint32_t j = i >> 2;
                     const float v = s_p[j][threadIdx.x][i & 3u];
                     const uint32_t key = key_of(v);
-                    const uint32_t rowbase = bytes_sum(ftot4 & ((1u << (8u * j)) - 1u));
-                    const uint32_t slot = rowbase + ((ex4 >> (8u * j)) & 0xFFu) + __popc(flag16 & ((1u << i) - 1u) & (0xFu << (4u * j)));
-                    const uint32_t coord = (uint32_t)(mine + 128 * (long long)j + (i & 3u));
+                    const uint32_t slot = (((j & 2u) ? q23 : q01) >> (16u * (j & 1u)) & 0xFFFFu) +
+                                          __popc(flag16 & ((1u << i) - 1u) & (0xFu << (4u * j)));
+                    const uint32_t coord = mine32 + 128u * j + (i & 3u);
                     flist[slot] = make_uint2(__float_as_uint(v), coord);
-                    if (key > hi) { e[coord] = 0.0f; ++my_sure; }
-                    else atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
+                    if (key > hi) { e[coord] = 0.0f; ++sure_here; }
+                    else {
+                        clist[atomicAdd(&s_crun[parity], 1u)] = make_uint2(key, coord);
+                        atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
+                    }
                 }
+                if (sure_here) { atomicAdd(P.tile_sure + item, sure_here); my_sure += sure_here; }
             }
         }
     }
@@ -350,7 +369,7 @@ topk_candbin_kernel(FastParams P) {
     const unsigned long long rsv = P.reserve[prob];
     st.cand_total = (uint32_t)(rsv >> 32);
     const uint32_t flag_total = (uint32_t)rsv;
-    bool ok = flag_total <= seg.flag_cap && st.sure_total <= seg.k &&
+    bool ok = flag_total <= seg.flag_cap && st.cand_total <= seg.cand_cap && st.sure_total <= seg.k &&
               (uint64_t)seg.k <= (uint64_t)st.sure_total + st.cand_total;
     uint32_t bin = 0, need_in = 0, cnt = 0;
     const uint32_t need = ok ? seg.k - st.sure_total : 0u;
@@ -377,7 +396,7 @@ topk_candbin_kernel(FastParams P) {
     }
 }
 
-// ---- filter: copy the flagged entries of the threshold's bin into the short list -------------
+// ---- filter: copy the candidates of the threshold's bin into the short list --------------------
 __global__ void __launch_bounds__(THREADS)
 topk_candfilter_kernel(FastParams P) {
     const Layout& L = P.L;
@@ -387,16 +406,15 @@ topk_candfilter_kernel(FastParams P) {
     if (!seg.fast) return;
     const FastState* stp = P.state + prob;
     if (stp->path != PATH_FAST || stp->need2 == 0) return;
-    const uint32_t total = (uint32_t)P.reserve[prob];                 // flagged entries (<= flag_cap on this path)
+    const uint32_t total = (uint32_t)(P.reserve[prob] >> 32);         // candidates (<= cand_cap on this path)
     const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
-    const uint2* list = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
+    const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin;
     uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
     for (uint32_t i = blockIdx.x * THREADS + threadIdx.x; i < total; i += gridDim.x * THREADS) {
         const uint2 c = list[i];
-        const uint32_t key = c.x & 0x7FFFFFFFu;
-        if (key >= lo2 && key <= hi2) {
+        if (c.x >= lo2 && c.x <= hi2) {
             const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
-            if (pos < LIST2_CAP) out[pos] = make_uint2(key, c.y);
+            if (pos < LIST2_CAP) out[pos] = c;
         }
     }
 }
@@ -452,32 +470,37 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
     return key > T || (key == T && coord < icut);
 }
 
-// ---- kept count per tile: one warp per tile counts over the tile's flagged slice -------------
+// ---- kept count per tile = sure elements + chosen candidates (8 lanes per tile) -----------------
 __global__ void __launch_bounds__(THREADS)
 topk_tilecount_kernel(FastParams P) {
     const Layout& L = P.L;
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t item = blockIdx.x * WARPS + (threadIdx.x >> 5);
-    if (item >= P.total_items) return;
-    const uint32_t w = item / L.tiles_per_worker;
-    const uint32_t lt = item - w * L.tiles_per_worker;
-    const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-    const SegEntry seg = L.segs[s];
-    uint32_t kept = 0;
-    if (seg.fast) {
-        const FastState* st = P.state + (size_t)w * L.nseg + s;
-        if (st->path == PATH_FAST) {
-            const uint32_t T = st->T, icut = st->icut;
-            const uint32_t base = P.tile_fbase[item], cnt = P.tile_fcnt[item];
-            const uint2* list = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + base;
-            for (uint32_t i = lane; i < cnt; i += 32) {
-                const uint2 c = list[i];
-                kept += fast_kept(c.x & 0x7FFFFFFFu, c.y, T, icut) ? 1u : 0u;
+    const uint32_t sub = threadIdx.x & 7u;
+    const uint32_t item = (blockIdx.x * THREADS + threadIdx.x) >> 3;
+    const bool live = item < P.total_items;
+    uint32_t kept = 0, w = 0, lt = 0;
+    if (live) {
+        w = item / L.tiles_per_worker;
+        lt = item - w * L.tiles_per_worker;
+        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+        const SegEntry seg = L.segs[s];
+        if (seg.fast) {
+            const FastState* st = P.state + (size_t)w * L.nseg + s;
+            if (st->path == PATH_FAST) {
+                const uint32_t T = st->T, icut = st->icut;
+                const uint32_t base = P.tile_cbase[item], cnt = P.tile_ccnt[item];
+                const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + base;
+                for (uint32_t i = sub; i < cnt; i += 8) {
+                    const uint2 c = list[i];
+                    kept += fast_kept(c.x, c.y, T, icut) ? 1u : 0u;
+                }
+                if (sub == 0) kept += P.tile_sure[item];
             }
-            kept = __reduce_add_sync(0xFFFFFFFFu, kept);
         }
     }
-    if (lane == 0) P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
+    kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 1);
+    kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 2);
+    kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 4);
+    if (live && sub == 0) P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
 }
 
 // ---- emit: one warp per tile walks the tile's slice of the flagged list -------------------------
@@ -506,29 +529,27 @@ topk_emit_kernel(FastParams P) {
         float* ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
         uint32_t* oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
         const uint32_t idx0 = (uint32_t)seg.offset;
-        for (uint32_t b = 0; b < cnt; b += 64) {                        // two independent loads in flight per lane
-            const uint32_t i0 = b + lane, i1 = b + 32 + lane;
-            uint2 a0 = make_uint2(0, 0), a1 = make_uint2(0, 0);
-            if (i0 < cnt) a0 = flist[i0];
-            if (i1 < cnt) a1 = flist[i1];
-            const uint32_t k0 = a0.x & 0x7FFFFFFFu, k1 = a1.x & 0x7FFFFFFFu;
-            const bool s0 = i0 < cnt && fast_kept(k0, a0.y, T, icut);
-            const bool s1 = i1 < cnt && fast_kept(k1, a1.y, T, icut);
-            const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, s0), b1 = __ballot_sync(0xFFFFFFFFu, s1);
-            if (s0) {
-                const uint32_t rank = running + __popc(b0 & lt_mask);
-                if (rank < seg.k) { ovals[rank] = __uint_as_float(a0.x); oidx[rank] = idx0 + a0.y; }
-                else atomicMin(P.status, ST_DEVICE_CHECK);
-                if (k0 <= hi) e[a0.y] = 0.0f;                           // a kept candidate: the main pass left p there
+        for (uint32_t b = 0; b < cnt; b += 128) {                       // four independent loads in flight per lane
+            uint2 a[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = b + 32u * u + lane;
+                a[u] = i < cnt ? flist[i] : make_uint2(0u, 0u);
             }
-            running += __popc(b0);
-            if (s1) {
-                const uint32_t rank = running + __popc(b1 & lt_mask);
-                if (rank < seg.k) { ovals[rank] = __uint_as_float(a1.x); oidx[rank] = idx0 + a1.y; }
-                else atomicMin(P.status, ST_DEVICE_CHECK);
-                if (k1 <= hi) e[a1.y] = 0.0f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = b + 32u * u + lane;
+                const uint32_t key = a[u].x & 0x7FFFFFFFu;
+                const bool sel = i < cnt && fast_kept(key, a[u].y, T, icut);
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, sel);
+                if (sel) {
+                    const uint32_t rank = running + __popc(bal & lt_mask);
+                    if (rank < seg.k) { ovals[rank] = __uint_as_float(a[u].x); oidx[rank] = idx0 + a[u].y; }
+                    else atomicMin(P.status, ST_DEVICE_CHECK);
+                    if (key <= hi) e[a[u].y] = 0.0f;                    // a kept candidate: the main pass left p there
+                }
+                running += __popc(bal);
             }
-            running += __popc(b1);
         }
     }
 }
