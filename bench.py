@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-events", action="store_true",
+                    help="do not bracket every kernel with events in the timed region (no roofline object)")
     ap.add_argument("--cpu-sample-div", type=int, default=1, help="oracle sample = n / this of one worker")
     ap.add_argument("--selftest-dist", action="store_true",
                     help="CPU-only check of the multi-rank plumbing (gloo): barrier, max over ranks, aggregate value")
@@ -299,7 +301,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     barrier()
     if rank == 0:
         sampler.start()
-    ctx.sc_profile(True)
+    ctx.sc_profile(not args.no_kernel_events)
     launches0 = ctx.launch_count
     marks = []
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
