@@ -293,6 +293,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     for t in range(args.warmup):
         one_step(t)
+    topk_paths = None
+    if "topk" in schemes:                       # which top-k path served the segments (not timed)
+        ctx.sc_step(sc.SC_TOPK, grads[0], res["topk"], seg_t, seeds(0), vals, idx, out)
+        topk_paths = dict(zip(("radix_small", "one_pass", "radix_after_missed_bracket"), ctx.sc_topk_path_counts()))
     status = ctx.sc_sync_status()
     if status != 0:
         raise RuntimeError(f"device status after warm-up: {sc.strerror(status)}")
@@ -371,6 +375,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "segments": len(segs), "l2": "inputs (%.1f GB per scheme pass) far larger than L2" % (8e-9 * n * W),
                    "replicas": world},
         "gpu_launches": int(launches),
+        "topk_paths": topk_paths,
         "clocks": clocks,
         "roofline": roofline,
         "per_scheme": step_roof,

@@ -183,7 +183,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             ++slow_count;
         }
         h[s] = e;
-        const uint64_t seg_tiles = (g.n + 3 + TILE - 1) / TILE;
+        const uint64_t seg_tiles = (g.n + 31 + TILE - 1) / TILE;   // a tile grid shifted by up to 31 elements
         tiles += seg_tiles;
         groups += (seg_tiles + PACK_GROUP - 1) / PACK_GROUP;
         scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
@@ -430,7 +430,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         return SC_ERR_CUDA;
     }
     c->max_n = max_n; c->max_W = max_W; c->max_seg = max_segments;
-    c->max_tiles_per_worker = (max_n + 3 + TILE - 1) / TILE + (size_t)max_segments + 1;
+    c->max_tiles_per_worker = (max_n + 31 + TILE - 1) / TILE + (size_t)max_segments + 1;
     c->max_mask_words = (max_n + 31) / 32 + (size_t)max_segments;
     c->max_atiles = (max_n + ATILE - 1) / ATILE;
     const size_t P = (size_t)max_W * max_segments;

@@ -174,7 +174,8 @@ __device__ inline uint32_t find_by_scat(const Layout& L, uint32_t ls) {
 
 // A quad is four consecutive elements starting at segment-local element `base`
 // (which may be negative or reach past n for the ragged first/last quad).  The
-// address seg + base is 16-byte aligned by construction.
+// address seg + base is 16-byte aligned by construction (base pointers are, and
+// tiles start on the 128-byte grid).
 __device__ inline uint32_t load_quad(const float* seg, long long base, uint32_t n, float v[4]) {
     if (base >= 0 && base + 3 < (long long)n) {
         float4 q = *reinterpret_cast<const float4*>(seg + base);
@@ -215,7 +216,9 @@ __device__ inline void store_quad(float* seg, long long base, uint32_t valid, co
 
 __device__ inline uint32_t key_of(float p) { return __float_as_uint(p) & 0x7FFFFFFFu; }
 
-__device__ inline uint32_t misalign_of(const void* p) { return (uint32_t)((reinterpret_cast<uintptr_t>(p) >> 2) & 3u); }
+// Tiles are laid on the 128-byte grid of the row, so that a warp's 512-byte access covers four
+// whole cache lines: elements of the segment before its first 128-byte boundary (0..31).
+__device__ inline uint32_t misalign_of(const void* p) { return (uint32_t)((reinterpret_cast<uintptr_t>(p) >> 2) & 31u); }
 
 // block-wide exclusive scan of one value per thread (THREADS threads); returns
 // the exclusive prefix, *total receives the block sum.  smem: WARPS + 1 words.
