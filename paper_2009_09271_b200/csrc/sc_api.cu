@@ -46,7 +46,8 @@ struct sc_ctx {
     uint32_t* d_tile_ccnt = nullptr;
     uint32_t* d_tile_fbase = nullptr;
     uint32_t* d_tile_fcnt = nullptr;
-    unsigned long long* d_reserve = nullptr;
+    uint32_t* d_cand_cnt = nullptr;  // [W * fast_per_worker][main grid]
+    size_t max_main_grid = 0;
     uint2* d_flagged = nullptr;      // grown on demand: its size depends on k
     size_t flagged_slots = 0;
     uint32_t* d_nslow = nullptr;     // [0]: segments for the radix select, [1]: segments whose bracket missed
@@ -166,24 +167,31 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         e.offset = g.offset; e.n = (uint32_t)g.n; e.k = (uint32_t)g.k;
         e.msg_off = (uint32_t)msg; e.tile_begin = (uint32_t)tiles; e.scat_begin = (uint32_t)scat;
         e.mask_word_begin = maskw; e.grp_begin = (uint32_t)groups;
+        const uint64_t seg_tiles = (g.n + 31 + TILE - 1) / TILE;   // a tile grid shifted by up to 31 elements
         if (g.n >= FAST_MIN_N) {
             uint64_t m = (g.n / 16) & ~7ull;
             m = std::min<uint64_t>(std::max<uint64_t>(m, SAMPLE_MIN), SAMPLE_MAX);
             e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
-            e.cand_cap = (uint32_t)(g.n / 32 + 16384);
+            // The main pass gives each of its CTAs a private region of the segment's flagged and
+            // candidate lists.  A CTA sees at most ceil(tiles / CTAs) tiles of the segment; a region
+            // holds that many tiles' share of (k + slack) resp. slack entries, slack = n / 32 + 16384.
+            const uint64_t slack = g.n / 32 + 16384;
+            const uint64_t ctas = std::max<uint64_t>(1, std::min<uint64_t>(c->max_main_grid, seg_tiles));
+            const uint64_t tiles_per_cta = (seg_tiles + ctas - 1) / ctas;
+            const uint64_t cand_region = tiles_per_cta * ((slack + seg_tiles - 1) / seg_tiles + 16);
+            const uint64_t flag_region = tiles_per_cta * ((g.k + slack + seg_tiles - 1) / seg_tiles + 16);
+            if (flag_region * c->max_main_grid > 0xFFFFFFFFull) return SC_ERR_RANGE;
+            e.cand_cap = (uint32_t)cand_region;          // per CTA
+            e.flag_cap = (uint32_t)flag_region;          // per CTA
             e.cand_begin = cand;
-            cand += e.cand_cap;
-            e.flag_cap = (uint32_t)std::min<uint64_t>(g.n, g.k + e.cand_cap);
             e.flag_begin = flag;
-            flag += e.flag_cap;
-            max_cap = std::max(max_cap, e.flag_cap);
-            c->max_cand_cap = std::max(c->max_cand_cap, e.cand_cap);
+            cand += cand_region * c->max_main_grid;
+            flag += flag_region * c->max_main_grid;
             max_m = std::max(max_m, e.sample_m);
         } else {
             ++slow_count;
         }
         h[s] = e;
-        const uint64_t seg_tiles = (g.n + 31 + TILE - 1) / TILE;   // a tile grid shifted by up to 31 elements
         tiles += seg_tiles;
         groups += (seg_tiles + PACK_GROUP - 1) / PACK_GROUP;
         scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
@@ -191,17 +199,18 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         msg += g.k;
     }
     if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
-    if (fast_count > c->max_fast_per_worker || cand > c->max_cand_per_worker) return SC_ERR_RANGE;
-    if ((size_t)c->max_W * flag > c->flagged_slots) {      // the flagged list follows k: grow it (synchronous, rare)
+    if (fast_count > c->max_fast_per_worker) return SC_ERR_RANGE;
+    if ((size_t)c->max_W * (flag + cand) > c->flagged_slots) {   // the lists follow k: grow them (synchronous, rare)
         SC_CUDA(cudaStreamSynchronize(stream));
         cudaFree(c->d_flagged); c->d_flagged = nullptr;
         c->scratch_bytes -= c->flagged_slots * sizeof(uint2);
         c->flagged_slots = 0;
-        const size_t want = (size_t)c->max_W * flag;
+        const size_t want = (size_t)c->max_W * (flag + cand);
         if (cudaMalloc(reinterpret_cast<void**>(&c->d_flagged), want * sizeof(uint2)) != cudaSuccess) return SC_ERR_WORKSPACE;
         c->flagged_slots = want;
         c->scratch_bytes += want * sizeof(uint2);
     }
+    c->d_cand = c->d_flagged + (size_t)c->max_W * flag;         // candidate lists live behind the flagged lists
     SegEntry sentinel{};
     sentinel.offset = n; sentinel.msg_off = (uint32_t)msg; sentinel.tile_begin = (uint32_t)tiles;
     sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw; sentinel.grp_begin = (uint32_t)groups;
@@ -268,9 +277,10 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             fp.state = c->d_fstate; fp.sample = c->d_sample; fp.cand_hist = c->d_cand_hist;
             fp.list2 = c->d_list2; fp.cand = c->d_cand; fp.tile_sure = c->d_tile_sure; fp.tile_cbase = c->d_tile_cbase;
             fp.tile_ccnt = c->d_tile_ccnt; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
-            fp.flagged = c->d_flagged; fp.reserve = c->d_reserve; fp.offsets = c->d_offsets;
+            fp.flagged = c->d_flagged; fp.cand_cnt = c->d_cand_cnt; fp.offsets = c->d_offsets;
+            fp.grid_main = persistent_grid(c, c->occ_main, items);
             fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
-            SC_CUDA(cudaMemsetAsync(c->d_reserve, 0, (size_t)P * sizeof(unsigned long long), stream));
+            SC_CUDA(cudaMemsetAsync(c->d_cand_cnt, 0, (size_t)W * L.fast_per_worker * fp.grid_main * sizeof(uint32_t), stream));
             SC_CUDA(cudaMemsetAsync(c->d_tile_sure, 0, (size_t)items * sizeof(uint32_t), stream));
             SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
             { Launch l(c, KIND_SAMPLE, stream);
@@ -278,12 +288,11 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             { Launch l(c, KIND_BRACKET, stream);
               topk_bracket_kernel<<<P, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_MAIN, stream);
-              topk_main_kernel<<<persistent_grid(c, c->occ_main, items), THREADS, 0, stream>>>(fp); }
+              topk_main_kernel<<<fp.grid_main, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDBIN, stream);
               topk_candbin_kernel<<<P, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDFILTER, stream);
-              const uint32_t gx = std::min<uint32_t>((c->max_cand_cap + THREADS * 4 - 1) / (THREADS * 4), 1024u);
-              topk_candfilter_kernel<<<dim3(std::max(gx, 1u), P), THREADS, 0, stream>>>(fp); }
+              topk_candfilter_kernel<<<dim3(fp.grid_main, P), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_FINAL, stream);
               topk_final_kernel<<<P, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_RESTORE, stream);
@@ -451,13 +460,11 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_sample, fastP * SAMPLE_MAX)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_cand_hist, fastP * CAND_BINS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_list2, fastP * LIST2_CAP)) == SC_OK &&
-        (rc = dev_alloc(c, &c->d_cand, (size_t)max_W * c->max_cand_per_worker)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_sure, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_cbase, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_ccnt, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_fbase, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_fcnt, items_max)) == SC_OK &&
-        (rc = dev_alloc(c, &c->d_reserve, P)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_nslow, 2)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_seeds, (size_t)max_W)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_status, 1)) == SC_OK) {
@@ -477,6 +484,8 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_block, randblock_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel, THREADS, 0);
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
+        c->max_main_grid = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
+        if (rc == SC_OK) rc = dev_alloc(c, &c->d_cand_cnt, fastP * c->max_main_grid);
     }
     if (rc != SC_OK) { sc_destroy(c); return rc; }
     *out = c;
@@ -488,8 +497,8 @@ void sc_destroy(sc_ctx* c) {
     DeviceGuard guard(c->device);
     cudaFree(c->d_segs); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
     cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate); cudaFree(c->d_sample);
-    cudaFree(c->d_cand_hist); cudaFree(c->d_cand); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_cbase);
-    cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt); cudaFree(c->d_reserve);
+    cudaFree(c->d_cand_hist); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_cbase);
+    cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt); cudaFree(c->d_cand_cnt);
     cudaFree(c->d_flagged); cudaFree(c->d_nslow); cudaFree(c->d_seeds); cudaFree(c->d_status);
     cudaFree(c->d_stage_grads); cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); cudaFree(c->d_stage_out);
     for (cudaEvent_t e : c->ev_worker) cudaEventDestroy(e);

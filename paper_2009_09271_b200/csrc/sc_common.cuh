@@ -31,11 +31,11 @@ struct SegEntry {
     uint32_t grp_begin;       // first pack group (PACK_GROUP tiles) of the segment inside a worker
     uint32_t fast;            // 1: large segment, top-k goes through the sampled-bracket path
     uint32_t sample_m;        // sample size of that path (multiple of 8)
-    uint32_t cand_cap;        // capacity of the segment's candidate list
+    uint32_t cand_cap;        // capacity of ONE main-pass CTA's region of the segment's candidate list
     uint32_t fast_index;      // index among the fast segments of a worker
     uint64_t cand_begin;      // first candidate slot of the segment inside a worker
     uint64_t flag_begin;      // first flagged-list slot of the segment inside a worker
-    uint32_t flag_cap;        // capacity of the segment's flagged list (k + candidate capacity)
+    uint32_t flag_cap;        // capacity of ONE main-pass CTA's region of the segment's flagged list
     uint32_t pad;
 };
 
@@ -79,7 +79,8 @@ struct FastState {
     uint32_t need2;        // 1-based rank of the threshold inside that bin (0: no candidate is kept)
     uint32_t cnt2;         // candidates copied into the short list
     uint32_t T, icut;      // kept <=> key > T, or key == T and coordinate < icut
-    uint32_t pad[4];
+    uint32_t overflow;     // a list region was full during the main pass
+    uint32_t pad[3];
 };
 
 constexpr uint32_t FAST_MIN_N = 1u << 20;

@@ -44,7 +44,8 @@ struct FastParams {
     uint32_t* tile_ccnt;       // candidates of the tile
     uint32_t* tile_fbase;      // first flagged slot of the tile (0xFFFFFFFF: the list was full, nothing written)
     uint32_t* tile_fcnt;       // flagged elements of the tile
-    unsigned long long* reserve;   // [W * nseg]: candidates reserved << 32 | flagged reserved
+    uint32_t* cand_cnt;        // [W * fast_per_worker][grid_main]: candidates each CTA of the main pass wrote
+    uint32_t grid_main;        // CTAs of the main pass: every list is cut into that many private regions
     uint32_t* n_failed;        // segments whose bracket missed
     uint32_t* offsets;         // [W][tiles_per_worker + 1]
     uint32_t* n_slow;          // segments that need the radix-select path
@@ -191,79 +192,99 @@ __device__ inline uint32_t warp_inclusive_scan(uint32_t v, uint32_t lane) {
 }
 __device__ inline uint32_t bytes_sum(uint32_t v) { return (v & 0xFFu) + ((v >> 8) & 0xFFu) + ((v >> 16) & 0xFFu) + (v >> 24); }
 
+struct MainTile {                  // where a work item lives (uniform over the CTA)
+    bool have, fast, full;
+    uint32_t w, lt, s;
+    SegEntry seg;
+    long long first;               // segment-local coordinate of the tile's first element
+    const float* g;
+    float* e;
+};
+__device__ inline MainTile main_decode(const FastParams& P, uint32_t item) {
+    const Layout& L = P.L;
+    MainTile t{};
+    t.have = item < P.total_items;
+    if (!t.have) return t;
+    t.w = item / L.tiles_per_worker;
+    t.lt = item - t.w * L.tiles_per_worker;
+    t.s = (L.nseg == 1) ? 0u : find_by_tile(L, t.lt);
+    t.seg = L.segs[t.s];
+    t.fast = t.seg.fast != 0;
+    const size_t row = (size_t)t.w * L.n_total + t.seg.offset;
+    t.g = P.grads + row;
+    t.e = P.residuals + row;
+    t.first = (long long)(t.lt - t.seg.tile_begin) * TILE - misalign_of(t.e);
+    t.full = t.first >= 0 && t.first + TILE <= (long long)t.seg.n;
+    return t;
+}
 __global__ void __launch_bounds__(THREADS)
 topk_main_kernel(FastParams P) {
-    __shared__ uint32_t sh[CAND_BINS];
-    __shared__ __align__(16) float s_p[QUADS][THREADS][4];           // the tile's p values, for the rare per-element work
+    __shared__ uint32_t sh[CAND_BINS];                                 // candidate histogram
+    __shared__ __align__(16) float s_p[TILE];                          // the tile's p values, for the per-element work
     __shared__ uint32_t s_wflag[2][WARPS], s_wcand[2][WARPS];
-    __shared__ unsigned long long s_base[2];
-    __shared__ uint32_t s_crun[2];                                    // running candidate slot inside the tile
     __shared__ uint32_t s_red[WARPS + 1];
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t off0 = warp * 512u + lane * 4u;                     // this thread's quad of row 0 inside a tile
+    // Each CTA appends to its own region of a segment's flagged and candidate lists (capacity / grid
+    // each), so a tile's slots follow from two running counters and no CTA waits for an atomic.
+    uint32_t run_flag = 0, run_cand = 0, fcap = 0, ccap = 0;
     for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) sh[b] = 0;
     __syncthreads();
     long long cur_prob = -1;
     size_t cur_fidx = 0;
     uint32_t lo = 0, hi = 0, shift = 0, parity = 0, my_sure = 0;
     for (uint32_t item = blockIdx.x; ; item += gridDim.x) {
-        // ---- which tile; flush the per-segment accumulators when the segment changes -------------
-        bool have = item < P.total_items;
-        uint32_t w = 0, lt = 0, s = 0;
-        SegEntry seg{};
-        if (have) {
-            w = item / L.tiles_per_worker;
-            lt = item - w * L.tiles_per_worker;
-            s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-            seg = L.segs[s];
-        }
-        const long long prob = have ? (long long)w * L.nseg + s : -2;
+        const MainTile T = main_decode(P, item);
+        // ---- flush the per-segment accumulators when the segment changes ---------------------------
+        const long long prob = T.have ? (long long)T.w * L.nseg + T.s : -2;
         if (prob != cur_prob && cur_prob >= 0) {                       // uniform over the CTA
             uint32_t total;
             block_exclusive_scan(my_sure, s_red, &total);              // (only the total is used)
-            if (threadIdx.x == 0 && total) atomicAdd(&P.state[cur_prob].sure_total, total);
+            if (threadIdx.x == 0) {
+                if (total) atomicAdd(&P.state[cur_prob].sure_total, total);
+                if (run_cand) atomicAdd(&P.state[cur_prob].cand_total, run_cand);
+                P.cand_cnt[cur_fidx * P.grid_main + blockIdx.x] = run_cand;
+            }
             for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
                 const uint32_t c = sh[b];
                 if (c) { atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c); sh[b] = 0; }
             }
             __syncthreads();
-            my_sure = 0;
+            my_sure = 0; run_flag = 0; run_cand = 0;
             cur_prob = -1;
         }
-        if (!have) break;
-        if (!seg.fast) continue;                                       // uniform over the CTA
+        if (!T.have) break;
+        if (!T.fast) continue;                                         // uniform over the CTA
+        const SegEntry& seg = T.seg;
         if (prob != cur_prob) {
             cur_prob = prob;
-            cur_fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
+            cur_fidx = (size_t)T.w * L.fast_per_worker + seg.fast_index;
             const FastState st = P.state[prob];
             lo = st.lo; hi = st.hi; shift = st.shift;
+            fcap = seg.flag_cap; ccap = seg.cand_cap;                  // per-CTA region sizes
         }
         parity ^= 1u;
-        const uint32_t t = lt - seg.tile_begin;
-        const size_t row = (size_t)w * L.n_total + seg.offset;
-        const float* g = P.grads + row;
-        float* e = P.residuals + row;
-        const uint32_t mis = misalign_of(e);
-        const long long first = (long long)t * TILE - mis;
-        const long long mine = first + warp * 512 + lane * 4;            // quad of row 0; row j at + 128 j
-        const bool full = first >= 0 && first + TILE <= (long long)seg.n;
+        float* e = T.e;
+        const long long mine = T.first + off0;                         // quad of row 0; row j at + 128 j
+        float* sp = s_p;                                               // each thread only touches its own 16 values
 
-        // ---- stream: p = g + e goes straight back to the residual and into shared memory ------------
+        // ---- stream: p = g + e goes straight back to the residual and stays in shared memory ----------
         uint32_t flag16 = 0;                                           // bit 4 j + c: key >= lo
-        if (full) {
+        if (T.full) {
             float4 ev[QUADS], gv[QUADS];
 #pragma unroll
             for (int j = 0; j < QUADS; ++j) {
                 ev[j] = __ldcs(reinterpret_cast<const float4*>(e + mine + 128 * j));
-                gv[j] = __ldcs(reinterpret_cast<const float4*>(g + mine + 128 * j));
+                gv[j] = __ldcs(reinterpret_cast<const float4*>(T.g + mine + 128 * j));
             }
 #pragma unroll
             for (int j = 0; j < QUADS; ++j) {
                 const float4 p = make_float4(gv[j].x + ev[j].x, gv[j].y + ev[j].y, gv[j].z + ev[j].z, gv[j].w + ev[j].w);
                 *reinterpret_cast<float4*>(e + mine + 128 * j) = p;
-                *reinterpret_cast<float4*>(&s_p[j][threadIdx.x][0]) = p;
-                flag16 |= (uint32_t)(key_of(p.x) >= lo) << (4 * j) | (uint32_t)(key_of(p.y) >= lo) << (4 * j + 1) |
-                          (uint32_t)(key_of(p.z) >= lo) << (4 * j + 2) | (uint32_t)(key_of(p.w) >= lo) << (4 * j + 3);
+                *reinterpret_cast<float4*>(sp + off0 + 128 * j) = p;
+                flag16 |= ((uint32_t)(key_of(p.x) >= lo) | (uint32_t)(key_of(p.y) >= lo) << 1 |
+                           (uint32_t)(key_of(p.z) >= lo) << 2 | (uint32_t)(key_of(p.w) >= lo) << 3) << (4 * j);
             }
         } else {
 #pragma unroll
@@ -271,14 +292,14 @@ topk_main_kernel(FastParams P) {
                 const long long base = mine + 128 * j;
                 float p[4], gq[4];
                 const uint32_t valid = load_quad(e, base, seg.n, p);
-                load_quad_stream(g, base, seg.n, gq);
+                load_quad_stream(T.g, base, seg.n, gq);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     p[c] = gq[c] + p[c];
                     flag16 |= (((valid >> c) & 1u) & (uint32_t)(key_of(p[c]) >= lo)) << (4 * j + c);
                 }
                 if (valid) store_quad(e, base, valid, p);
-                *reinterpret_cast<float4*>(&s_p[j][threadIdx.x][0]) = make_float4(p[0], p[1], p[2], p[3]);
+                *reinterpret_cast<float4*>(sp + off0 + 128 * j) = make_float4(p[0], p[1], p[2], p[3]);
             }
         }
         // ---- ranks of the flagged elements, in coordinate order ---------------------------------------
@@ -293,63 +314,60 @@ topk_main_kernel(FastParams P) {
             while (bits) {
                 const uint32_t i = (uint32_t)__ffs((int)bits) - 1u;
                 bits &= bits - 1u;
-                ccnt += key_of(s_p[i >> 2][threadIdx.x][i & 3u]) <= hi ? 1u : 0u;
+                ccnt += key_of(sp[off0 + 128u * (i >> 2) + (i & 3u)]) <= hi ? 1u : 0u;
             }
         }
-        const uint32_t wcand = __reduce_add_sync(0xFFFFFFFFu, ccnt);
+        const uint32_t cinc = warp_inclusive_scan(ccnt, lane);
+        const uint32_t wcand = __shfl_sync(0xFFFFFFFFu, cinc, 31);
         if (lane == 0) { s_wflag[parity][warp] = bytes_sum(ftot4); s_wcand[parity][warp] = wcand; }
         __syncthreads();
-        uint32_t tcand = 0, tflag = 0, fwbase = 0;
+        uint32_t tcand = 0, tflag = 0, fwbase = 0, cwbase = 0;
 #pragma unroll
         for (int i = 0; i < WARPS; ++i) {
-            const uint32_t f = s_wflag[parity][i];
+            const uint32_t f = s_wflag[parity][i], c = s_wcand[parity][i];
             fwbase += (i < (int)warp) ? f : 0u;
-            tcand += s_wcand[parity][i]; tflag += f;
+            cwbase += (i < (int)warp) ? c : 0u;
+            tcand += c; tflag += f;
         }
+        // this CTA's regions of the two lists, and where this tile's entries go inside them
+        const bool fits = run_flag + tflag <= fcap && run_cand + tcand <= ccap;
+        const uint32_t fbase = blockIdx.x * fcap + run_flag, cbase = blockIdx.x * ccap + run_cand;
         if (threadIdx.x == 0) {
-            unsigned long long base = 0;
-            if (tflag) base = atomicAdd(P.reserve + prob, ((unsigned long long)tcand << 32) | tflag);
-            const bool fits = (unsigned long long)(uint32_t)base + tflag <= seg.flag_cap &&
-                              (base >> 32) + tcand <= seg.cand_cap;
-            P.tile_fbase[item] = fits ? (uint32_t)base : 0xFFFFFFFFu;
+            P.tile_fbase[item] = fits ? fbase : 0xFFFFFFFFu;
             P.tile_fcnt[item] = tflag;
-            P.tile_cbase[item] = (uint32_t)(base >> 32);
+            P.tile_cbase[item] = cbase;
             P.tile_ccnt[item] = fits ? tcand : 0u;
-            s_base[parity] = fits ? base : ~0ull;
-            s_crun[parity] = (uint32_t)(base >> 32);
+            if (!fits) P.state[prob].overflow = 1u;                    // a region is full: the segment falls back
         }
-        if (tflag) {                                                   // uniform over the CTA
-            __syncthreads();
-            const unsigned long long base = s_base[parity];
-            if (base != ~0ull && flag16) {
-                // the tile's entries fit: write them, zero the sure ones in the residual (their values
-                // stay in the list, from where a fall-back restores them), histogram the candidates
-                uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + (uint32_t)base + fwbase;
-                uint2* clist = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin;
-                uint32_t bits = flag16, sure_here = 0;
-                // first slot of this lane's quad in each row, relative to the warp's slice (< 512: 16 bits each)
-                const uint32_t r0 = ftot4 & 0xFFu, r1 = (ftot4 >> 8) & 0xFFu, r2 = (ftot4 >> 16) & 0xFFu;
-                const uint32_t q01 = (ex4 & 0xFFu) | ((r0 + ((ex4 >> 8) & 0xFFu)) << 16);
-                const uint32_t q23 = (r0 + r1 + ((ex4 >> 16) & 0xFFu)) | ((r0 + r1 + r2 + (ex4 >> 24)) << 16);
-                const uint32_t mine32 = (uint32_t)mine;
-                while (bits) {
-                    const uint32_t i = (uint32_t)__ffs((int)bits) - 1u;
-                    bits &= bits - 1u;
-                    const uint32_t j = i >> 2;
-                    const float v = s_p[j][threadIdx.x][i & 3u];
-                    const uint32_t key = key_of(v);
-                    const uint32_t slot = (((j & 2u) ? q23 : q01) >> (16u * (j & 1u)) & 0xFFFFu) +
-                                          __popc(flag16 & ((1u << i) - 1u) & (0xFu << (4u * j)));
-                    const uint32_t coord = mine32 + 128u * j + (i & 3u);
-                    flist[slot] = make_uint2(__float_as_uint(v), coord);
-                    if (key > hi) { e[coord] = 0.0f; ++sure_here; }
-                    else {
-                        clist[atomicAdd(&s_crun[parity], 1u)] = make_uint2(key, coord);
-                        atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
-                    }
+        if (fits) { run_flag += tflag; run_cand += tcand; }
+        if (fits && flag16) {
+            // the tile's entries fit: write them, zero the sure ones in the residual (their values
+            // stay in the list, from where a fall-back restores them), histogram the candidates
+            uint2* flist = P.flagged + (size_t)T.w * L.flag_per_worker + seg.flag_begin + fbase + fwbase;
+            uint2* clist = P.cand + (size_t)T.w * L.cand_per_worker + seg.cand_begin + cbase + cwbase + (cinc - ccnt);
+            uint32_t bits = flag16, sure_here = 0;
+            // first slot of this lane's quad in each row, relative to the warp's slice (< 512: 16 bits each)
+            const uint32_t r0 = ftot4 & 0xFFu, r1 = (ftot4 >> 8) & 0xFFu, r2 = (ftot4 >> 16) & 0xFFu;
+            const uint32_t q01 = (ex4 & 0xFFu) | ((r0 + ((ex4 >> 8) & 0xFFu)) << 16);
+            const uint32_t q23 = (r0 + r1 + ((ex4 >> 16) & 0xFFu)) | ((r0 + r1 + r2 + (ex4 >> 24)) << 16);
+            const uint32_t mine32 = (uint32_t)mine;
+            while (bits) {
+                const uint32_t i = (uint32_t)__ffs((int)bits) - 1u;
+                bits &= bits - 1u;
+                const uint32_t j = i >> 2;
+                const float v = sp[off0 + 128u * j + (i & 3u)];
+                const uint32_t key = key_of(v);
+                const uint32_t slot = (((j & 2u) ? q23 : q01) >> (16u * (j & 1u)) & 0xFFFFu) +
+                                      __popc(flag16 & ((1u << i) - 1u) & (0xFu << (4u * j)));
+                const uint32_t coord = mine32 + 128u * j + (i & 3u);
+                flist[slot] = make_uint2(__float_as_uint(v), coord);
+                if (key > hi) { e[coord] = 0.0f; ++sure_here; }
+                else {
+                    *clist++ = make_uint2(key, coord);
+                    atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
                 }
-                if (sure_here) { atomicAdd(P.tile_sure + item, sure_here); my_sure += sure_here; }
             }
+            if (sure_here) { atomicAdd(P.tile_sure + item, sure_here); my_sure += sure_here; }
         }
     }
 }
@@ -366,10 +384,7 @@ topk_candbin_kernel(FastParams P) {
     FastState st = P.state[prob];
     if (st.path != PATH_FAST) return;
     const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
-    const unsigned long long rsv = P.reserve[prob];
-    st.cand_total = (uint32_t)(rsv >> 32);
-    const uint32_t flag_total = (uint32_t)rsv;
-    bool ok = flag_total <= seg.flag_cap && st.cand_total <= seg.cand_cap && st.sure_total <= seg.k &&
+    bool ok = st.overflow == 0u && st.sure_total <= seg.k &&
               (uint64_t)seg.k <= (uint64_t)st.sure_total + st.cand_total;
     uint32_t bin = 0, need_in = 0, cnt = 0;
     const uint32_t need = ok ? seg.k - st.sure_total : 0u;
@@ -406,15 +421,19 @@ topk_candfilter_kernel(FastParams P) {
     if (!seg.fast) return;
     const FastState* stp = P.state + prob;
     if (stp->path != PATH_FAST || stp->need2 == 0) return;
-    const uint32_t total = (uint32_t)(P.reserve[prob] >> 32);         // candidates (<= cand_cap on this path)
     const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
-    const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin;
-    uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
-    for (uint32_t i = blockIdx.x * THREADS + threadIdx.x; i < total; i += gridDim.x * THREADS) {
-        const uint2 c = list[i];
-        if (c.x >= lo2 && c.x <= hi2) {
-            const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
-            if (pos < LIST2_CAP) out[pos] = c;
+    const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
+    const uint32_t ccap = seg.cand_cap;
+    uint2* out = P.list2 + fidx * LIST2_CAP;
+    for (uint32_t r = blockIdx.x; r < P.grid_main; r += gridDim.x) {        // one region (one main-pass CTA) at a time
+        const uint32_t total = P.cand_cnt[fidx * P.grid_main + r];
+        const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + (size_t)r * ccap;
+        for (uint32_t i = threadIdx.x; i < total; i += THREADS) {
+            const uint2 c = list[i];
+            if (c.x >= lo2 && c.x <= hi2) {
+                const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
+                if (pos < LIST2_CAP) out[pos] = c;
+            }
         }
     }
 }
