@@ -522,6 +522,7 @@ topk_tilecount_kernel(FastParams P) {
     if (live && sub == 0) P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
 }
 
+constexpr int EMIT_DEPTH = 4;
 // ---- emit: one warp per tile walks the tile's slice of the flagged list -------------------------
 __global__ void __launch_bounds__(THREADS)
 topk_emit_kernel(FastParams P) {
@@ -529,45 +530,66 @@ topk_emit_kernel(FastParams P) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t lt_mask = (1u << lane) - 1u;
     const uint32_t warps_total = gridDim.x * WARPS;
+    // per-(worker, segment) constants stay in registers while the warp's tiles belong to the same one
+    uint32_t cw = 0xFFFFFFFFu, cs = 0xFFFFFFFFu, c_tile_end = 0;        // cached worker, segment, end of its tile range
+    uint32_t T = 0, icut = 0, hi = 0, seg_k = 0, idx0 = 0, tile_begin = 0, off_begin = 0;
+    bool live = false;
+    const uint2* flist0 = nullptr;
+    float* e = nullptr;
+    float* ovals = nullptr;
+    uint32_t* oidx = nullptr;
+    const uint32_t* off = nullptr;
     for (uint32_t item = blockIdx.x * WARPS + (threadIdx.x >> 5); item < P.total_items; item += warps_total) {
-        const uint32_t cnt = P.tile_fcnt[item];
-        if (cnt == 0u) continue;
         const uint32_t w = item / L.tiles_per_worker;
         const uint32_t lt = item - w * L.tiles_per_worker;
-        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-        const SegEntry seg = L.segs[s];
-        if (!seg.fast) continue;
-        const FastState* st = P.state + (size_t)w * L.nseg + s;
-        if (st->path != PATH_FAST) continue;
-        const uint32_t T = st->T, icut = st->icut, hi = st->hi;
-        const uint32_t base = P.tile_fbase[item];
-        const uint32_t* off = P.offsets + (size_t)w * (L.tiles_per_worker + 1);
-        uint32_t running = off[lt] - off[seg.tile_begin];               // kept coordinates of the segment before this tile
-        const uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + base;
-        float* e = P.residuals + (size_t)w * L.n_total + seg.offset;
-        float* ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
-        uint32_t* oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
-        const uint32_t idx0 = (uint32_t)seg.offset;
-        for (uint32_t b = 0; b < cnt; b += 128) {                       // four independent loads in flight per lane
-            uint2 a[4];
+        if (w != cw || lt < tile_begin || lt >= c_tile_end) {           // another (worker, segment): reload
+            cw = w;
+            cs = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+            const SegEntry seg = L.segs[cs];
+            tile_begin = seg.tile_begin; c_tile_end = L.segs[cs + 1].tile_begin;
+            const FastState* st = P.state + (size_t)w * L.nseg + cs;
+            live = seg.fast && st->path == PATH_FAST;
+            T = st->T; icut = st->icut; hi = st->hi; seg_k = seg.k; idx0 = (uint32_t)seg.offset;
+            off = P.offsets + (size_t)w * (L.tiles_per_worker + 1);
+            off_begin = off[tile_begin];
+            flist0 = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
+            e = P.residuals + (size_t)w * L.n_total + seg.offset;
+            ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
+            oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
+        }
+        if (!live) continue;
+        // the four words that place this tile: independent loads, one round trip
+        const uint32_t cnt = P.tile_fcnt[item], base = P.tile_fbase[item];
+        const uint32_t o0 = off[lt], o1 = off[lt + 1];
+        if (cnt == 0u) continue;
+        const uint32_t running = o0 - off_begin;                        // kept coordinates of the segment before this tile
+        if ((unsigned long long)running + (o1 - o0) > seg_k) {          // counts and k disagree: write nothing
+            if (lane == 0) atomicMin(P.status, ST_DEVICE_CHECK);
+            continue;
+        }
+        // entry i of the slice belongs to lane i % 32; message pointers advance with the running rank
+        float* ov = ovals + running;
+        uint32_t* oi = oidx + running;
+        const uint2* fl = flist0 + base + lane;
+        for (uint32_t b = 0; b < cnt; b += 32 * EMIT_DEPTH) {           // EMIT_DEPTH independent loads in flight per lane
+            uint2 a[EMIT_DEPTH];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t i = b + 32u * u + lane;
-                a[u] = i < cnt ? flist[i] : make_uint2(0u, 0u);
-            }
+            for (int u = 0; u < EMIT_DEPTH; ++u) a[u] = (b + 32u * u + lane < cnt) ? __ldg(fl + b + 32u * u) : make_uint2(0u, 0xFFFFFFFFu);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t i = b + 32u * u + lane;
+            for (int u = 0; u < EMIT_DEPTH; ++u) {
+                // a padding entry has key 0 and coordinate 2^32-1: kept only if T == 0 and icut == 2^32-1, which
+                // cannot happen (coordinates are < n < 2^32, so icut <= n)
                 const uint32_t key = a[u].x & 0x7FFFFFFFu;
-                const bool sel = i < cnt && fast_kept(key, a[u].y, T, icut);
+                const bool sel = key > T || (key == T && a[u].y < icut);
                 const uint32_t bal = __ballot_sync(0xFFFFFFFFu, sel);
                 if (sel) {
-                    const uint32_t rank = running + __popc(bal & lt_mask);
-                    if (rank < seg.k) { ovals[rank] = __uint_as_float(a[u].x); oidx[rank] = idx0 + a[u].y; }
-                    else atomicMin(P.status, ST_DEVICE_CHECK);
+                    const uint32_t r = __popc(bal & lt_mask);
+                    ov[r] = __uint_as_float(a[u].x);
+                    oi[r] = idx0 + a[u].y;
                     if (key <= hi) e[a[u].y] = 0.0f;                    // a kept candidate: the main pass left p there
                 }
-                running += __popc(bal);
+                const uint32_t adv = __popc(bal);
+                ov += adv; oi += adv;
             }
         }
     }
