@@ -382,6 +382,24 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "kernels": kernels,
     }
 
+    # ---- next row: aggregate fused with the model update (not part of the metric) ------------
+    if rank == 0 and K > 0:
+        xmodel = torch.zeros(n, device=dev)
+        tim = {}
+        for name, shared in (("aggregate_apply_ms", False), ("aggregate_apply_shared_ms", True)):
+            ctx.sc_aggregate_apply(W, vals, idx, K, n, xmodel, shared=shared)          # warm-up
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(3):
+                ctx.sc_aggregate_apply(W, vals, idx, K, n, xmodel, shared=shared)
+            b.record()
+            torch.cuda.synchronize()
+            tim[name] = round(a.elapsed_time(b) / 3, 4)
+        tim["note"] = ("x <- x - average applied at sent coordinates only, on the last scheme's messages; "
+                       "the dense sc_aggregate of the same messages is in kernels.agg_tiles")
+        line["next_rows"] = tim
+        del xmodel
+
     # ---- end to end through the C ABI with host buffers ------------------------------------
     if not args.no_e2e and rank == 0:
         line["e2e"] = run_e2e(args, ctx, sc, wl, w, sizes, W, schemes, codes, seg_t, res, n, dev)

@@ -120,6 +120,17 @@ int sc_aggregate(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, siz
 int sc_aggregate_shared(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
                         float* out, void* stream);
 
+/* Algorithm 1, aggregate line fused with the model-update line (x <- x - q, q read as the
+ * average as above): x[i] <- x[i] - (sum over w = 0..W-1, in order, from +0.0, of q^w[i]) / W
+ * for every coordinate some worker sent; all other x[i] are left untouched.  The result is
+ * bit-identical to computing the dense average with sc_aggregate and subtracting it, but the
+ * dense vector is never written or read.  Same message conventions as sc_aggregate; x[n] is
+ * updated in place.  The _shared form takes ONE row of coordinates for all workers. */
+int sc_aggregate_apply(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                       float* x, void* stream);
+int sc_aggregate_apply_shared(sc_ctx* ctx, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                              float* x, void* stream);
+
 /* The paper has no counterpart for this entry point: it is sc_aggregate for callers that
  * are not allowed to allocate device memory.  Every other entry point needs an sc_ctx, and
  * sc_create calls cudaMalloc.  That rules the library out for code that runs after a

@@ -225,6 +225,13 @@ def aggregate(vals: Sequence[np.ndarray], idx: Sequence[np.ndarray], n: int) -> 
     return out / np.float32(W)
 
 
+def aggregate_apply(x: np.ndarray, vals: Sequence[np.ndarray], idx: Sequence[np.ndarray]) -> np.ndarray:
+    """Algorithm 1, model-update line with the aggregate read as the average:
+    x_{t+1} = x_t - q_t, q_t = aggregate(...).  Returns the new x (fp32)."""
+    assert x.dtype == np.float32
+    return x - aggregate(vals, idx, x.size)
+
+
 def step(scheme: int, grads: Sequence[np.ndarray], residuals: Sequence[np.ndarray],
          segments: Sequence[Tuple[int, int, int]], seeds: Sequence[int]):
     """All W workers compress, then one aggregate.  Returns

@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_HERE, "libsparsecomm.so")
 
 EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_scratch_bytes", "sc_launch_count",
            "sc_topk_path_counts", "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
-           "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_aggregate_static", "sc_step", "sc_step_host"]
+           "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_aggregate_static", "sc_aggregate_apply",
+           "sc_aggregate_apply_shared", "sc_step", "sc_step_host"]
 
 
 class ScSegment(ctypes.Structure):
@@ -77,6 +78,9 @@ def load_library() -> ctypes.CDLL:
     lib.sc_aggregate.restype = ci
     lib.sc_aggregate_shared.argtypes = [vp, ci, vp, vp, sz, sz, vp, vp]
     lib.sc_aggregate_shared.restype = ci
+    for name in ("sc_aggregate_apply", "sc_aggregate_apply_shared"):
+        getattr(lib, name).argtypes = [vp, ci, vp, vp, sz, sz, vp, vp]
+        getattr(lib, name).restype = ci
     lib.sc_aggregate_static.argtypes = [ci, vp, vp, sz, sz, vp, vp]
     lib.sc_aggregate_static.restype = ci
     lib.sc_step.argtypes = [vp, ci, ci, vp, vp, sz, ctypes.POINTER(ScSegment), ci, ctypes.POINTER(u64),
@@ -227,6 +231,14 @@ class Context:
             raise ValueError("buffer sizes do not match W, k and n")
         _check(self._lib.sc_aggregate_shared(self._h, W, _ptr(vals), _ptr(idx), k, n, _ptr(out), _stream(stream)),
                "sc_aggregate_shared")
+
+    def sc_aggregate_apply(self, W: int, vals, idx, k: int, n: int, x, stream=None, shared: bool = False) -> None:
+        """x <- x - average of the W messages, touching only the coordinates that were sent."""
+        _want(vals, torch.float32, "vals"), _want(idx, torch.int32, "idx"), _want(x, torch.float32, "x")
+        if vals.numel() < W * k or idx.numel() < (k if shared else W * k) or x.numel() < n:
+            raise ValueError("buffer sizes do not match W, k and n")
+        fn = self._lib.sc_aggregate_apply_shared if shared else self._lib.sc_aggregate_apply
+        _check(fn(self._h, W, _ptr(vals), _ptr(idx), k, n, _ptr(x), _stream(stream)), "sc_aggregate_apply")
 
     def sc_step(self, scheme: int, grads, residuals, segs, seeds, out_vals, out_idx, out, stream=None) -> None:
         W, n = grads.shape

@@ -97,8 +97,11 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
                             if (s_off[mid] <= q) lo = mid; else hi = mid;
                         }
                         const size_t j = (size_t)(w0 + lo) * K + s_lo[lo] + (q - s_off[lo]);
-                        st_loc[q - cs] = idx[j] - tile_lo;
-                        st_val[q - cs] = vals[j];
+                        uint32_t loc = idx[j] - tile_lo;
+                        float v = vals[j];
+                        if (loc >= tile_n) { atomicMin(status, ST_DEVICE_CHECK); loc = 0xFFFFFFFFu; v = 0.0f; }   // never applied
+                        st_loc[q - cs] = loc;
+                        st_val[q - cs] = v;
                     }
                     __syncthreads();
                     for (uint32_t i = 0; i < wn; ++i) {
@@ -106,8 +109,7 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
                         if (a < b) {                             // uniform over the CTA
                             for (uint32_t q = a + threadIdx.x; q < b; q += THREADS) {
                                 const uint32_t loc = st_loc[q - cs];
-                                if (loc < tile_n) acc[loc] = acc[loc] + st_val[q - cs];
-                                else atomicMin(status, ST_DEVICE_CHECK);
+                                if (loc < ATILE) acc[loc] = acc[loc] + st_val[q - cs];
                             }
                             __syncthreads();
                         }
@@ -128,6 +130,108 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
             for (uint32_t i = threadIdx.x; i < tile_n; i += THREADS) o[i] = pow2 ? acc[i] * rW : acc[i] / fW;
         }
         __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Aggregate fused with the model update (Algorithm 1, update line: x <- x - q, q read as the
+// average): only coordinates that some worker sent are read and written, the dense q is never
+// materialised.  x - (+0.0) == x bit for bit, so skipping coordinates whose sum is zero gives
+// exactly what the dense formulation gives.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS)
+agg_apply_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
+                       const uint32_t* __restrict__ bounds, uint32_t W, uint32_t K, uint32_t n, uint32_t ntiles,
+                       float* __restrict__ x, int* __restrict__ status) {
+    __shared__ __align__(16) float acc[ATILE];
+    __shared__ uint32_t st_loc[AGG_STAGE];
+    __shared__ float st_val[AGG_STAGE];
+    __shared__ uint32_t s_lo[64], s_off[65];
+    const float fW = (float)W;
+    const bool pow2 = (W & (W - 1u)) == 0u;
+    const float rW = 1.0f / fW;
+    for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const uint32_t tile_lo = t * ATILE;
+        const uint32_t tile_n = min(ATILE, n - tile_lo);
+        bool zeroed = false;
+        for (uint32_t w0 = 0; w0 < W; w0 += 64) {
+            const uint32_t wn = min(64u, W - w0);
+            __syncthreads();
+            if (threadIdx.x < wn) {
+                const uint32_t* b = bounds + (size_t)(w0 + threadIdx.x) * (ntiles + 1) + t;
+                const uint32_t lo = b[0], hi = b[1];
+                s_lo[threadIdx.x] = lo;
+                s_off[threadIdx.x + 1] = hi - lo;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                uint32_t run = 0;
+                s_off[0] = 0;
+                for (uint32_t i = 0; i < wn; ++i) { run += s_off[i + 1]; s_off[i + 1] = run; }
+            }
+            __syncthreads();
+            const uint32_t total = s_off[wn];
+            if (total && !zeroed) {                              // uniform: the tile is touched, start from +0.0
+                for (uint32_t i = threadIdx.x; i < ATILE / 4; i += THREADS)
+                    reinterpret_cast<float4*>(acc)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                zeroed = true;
+                __syncthreads();
+            }
+            for (uint32_t cs = 0; cs < total; cs += AGG_STAGE) {
+                const uint32_t ce = min(total, cs + AGG_STAGE);
+                for (uint32_t q = cs + threadIdx.x; q < ce; q += THREADS) {
+                    uint32_t lo = 0, hi = wn;
+                    while (hi - lo > 1) {
+                        const uint32_t mid = (lo + hi) >> 1;
+                        if (s_off[mid] <= q) lo = mid; else hi = mid;
+                    }
+                    const size_t j = (size_t)(w0 + lo) * K + s_lo[lo] + (q - s_off[lo]);
+                    uint32_t loc = idx[j] - tile_lo;
+                    float v = vals[j];
+                    if (loc >= tile_n) { atomicMin(status, ST_DEVICE_CHECK); loc = 0xFFFFFFFFu; v = 0.0f; }   // never applied
+                    st_loc[q - cs] = loc;
+                    st_val[q - cs] = v;
+                }
+                __syncthreads();
+                for (uint32_t i = 0; i < wn; ++i) {
+                    const uint32_t a = max(s_off[i], cs), b = min(s_off[i + 1], ce);
+                    if (a < b) {                                 // uniform over the CTA
+                        for (uint32_t q = a + threadIdx.x; q < b; q += THREADS) {
+                            const uint32_t loc = st_loc[q - cs];
+                            if (loc < ATILE) acc[loc] = acc[loc] + st_val[q - cs];
+                        }
+                        __syncthreads();
+                    }
+                }
+            }
+        }
+        if (zeroed) {
+            __syncthreads();
+            for (uint32_t i = threadIdx.x; i < tile_n; i += THREADS) {
+                const float a = acc[i];
+                if (a != 0.0f) {                                   // also true for NaN
+                    const float q = pow2 ? a * rW : a / fW;
+                    x[tile_lo + i] = x[tile_lo + i] - q;
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// All workers kept the same coordinates: one thread per message slot.
+__global__ void __launch_bounds__(THREADS)
+agg_apply_shared_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx, uint32_t W, uint32_t K,
+                        uint32_t n, float* __restrict__ x, int* __restrict__ status) {
+    const float fW = (float)W;
+    const bool pow2 = (W & (W - 1u)) == 0u;
+    const float rW = 1.0f / fW;
+    for (uint32_t j = blockIdx.x * THREADS + threadIdx.x; j < K; j += gridDim.x * THREADS) {
+        const uint32_t i = idx[j];
+        float sum = 0.0f;
+        for (uint32_t w = 0; w < W; ++w) sum = sum + vals[(size_t)w * K + j];
+        if (i >= n) { atomicMin(status, ST_DEVICE_CHECK); continue; }
+        if (sum != 0.0f) x[i] = x[i] - (pow2 ? sum * rW : sum / fW);
     }
 }
 

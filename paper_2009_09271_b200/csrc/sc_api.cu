@@ -116,11 +116,12 @@ class DeviceGuard {
 
 enum { KIND_HIST0 = 0, KIND_RESOLVE, KIND_REFINE, KIND_PACK_TOPK, KIND_SCATTER, KIND_MASK_COUNT, KIND_ROW_SCAN,
        KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES, KIND_SAMPLE, KIND_BRACKET, KIND_MAIN,
-       KIND_CANDBIN, KIND_CANDFILTER, KIND_FINAL, KIND_TILECOUNT, KIND_EMIT, KIND_RESTORE, KIND_COUNT };
+       KIND_CANDBIN, KIND_CANDFILTER, KIND_FINAL, KIND_TILECOUNT, KIND_EMIT, KIND_RESTORE, KIND_AGG_APPLY, KIND_COUNT };
 const char* const kKindNames[KIND_COUNT] = {"topk_hist0", "topk_resolve", "topk_refine", "pack_topk", "randk_scatter",
                                             "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
                                             "agg_tiles", "topk_sample", "topk_bracket", "topk_main", "topk_candbin",
-                                            "topk_candfilter", "topk_final", "topk_tilecount", "topk_emit", "topk_restore"};
+                                            "topk_candfilter", "topk_final", "topk_tilecount", "topk_emit", "topk_restore",
+                                            "agg_apply"};
 
 // Counts a kernel launch and, when profiling is on, brackets it with two events.
 class Launch {
@@ -597,6 +598,40 @@ int sc_aggregate_shared(sc_ctx* c, int W, const float* vals, const uint32_t* idx
     if (rc != SC_OK) return rc;
     DeviceGuard guard(c->device);
     return aggregate_rows(c, W, vals, idx, true, k, n, out, static_cast<cudaStream_t>(stream));
+}
+
+int sc_aggregate_apply(sc_ctx* c, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                       float* x, void* stream) {
+    int rc = check_aggregate_args(c, W, vals, idx, k, n, x);
+    if (rc != SC_OK) return rc;
+    if (n == 0 || k == 0) return SC_OK;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
+    const uint64_t threads = (uint64_t)W * (ntiles + 1ull);
+    { Launch l(c, KIND_AGG_BOUNDS, st);
+      agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, st>>>(
+          idx, (uint32_t)W, (uint32_t)k, ntiles, c->d_bounds); }
+    { Launch l(c, KIND_AGG_APPLY, st);
+      agg_apply_tiles_kernel<<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, st>>>(
+          vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, x, c->d_status); }
+    SC_CUDA(cudaGetLastError());
+    return SC_OK;
+}
+
+int sc_aggregate_apply_shared(sc_ctx* c, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
+                              float* x, void* stream) {
+    int rc = check_aggregate_args(c, W, vals, idx, k, n, x);
+    if (rc != SC_OK) return rc;
+    if (n == 0 || k == 0) return SC_OK;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    { Launch l(c, KIND_AGG_APPLY, st);
+      const uint64_t blocks = (k + THREADS - 1) / THREADS;
+      agg_apply_shared_kernel<<<persistent_grid(c, 8, blocks), THREADS, 0, st>>>(
+          vals, idx, (uint32_t)W, (uint32_t)k, (uint32_t)n, x, c->d_status); }
+    SC_CUDA(cudaGetLastError());
+    return SC_OK;
 }
 
 int sc_step(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,

@@ -276,3 +276,26 @@ def test_argument_errors_leave_buffers_untouched(ctx):
     with pytest.raises(sc.SparseCommError):
         ctx.sc_compress(9, g, e, k, 0, vals, idx)
     assert sc.strerror(-2) == "size out of range"
+
+
+@pytest.mark.parametrize("W", [1, 4, 7, 16])
+def test_aggregate_apply_matches_dense_update(W):
+    """x <- x - average(messages), touched coordinates only, against the oracle's dense form."""
+    rng = np.random.default_rng(40 + W)
+    n, k = 300_007, 9000
+    c = sc.Context(max_n=n, max_W=16, max_segments=1)
+    idx = np.stack([np.sort(rng.choice(n, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+    vals = (rng.standard_normal((W, k)) * 10.0 ** rng.uniform(-3, 3, (W, k))).astype(np.float32)
+    vals[0, :5] = [np.inf, -np.inf, 0.0, -0.0, 1e-42]
+    x0 = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    x0[idx[0][2]] = -0.0
+    d_idx, d_vals = torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(vals).cuda()
+    x = torch.from_numpy(x0).cuda()
+    c.sc_aggregate_apply(W, d_vals, d_idx, k, n, x)
+    assert c.sc_sync_status() == 0
+    assert_bits_equal(x, O.aggregate_apply(x0, list(vals), list(idx)), "apply")
+    xs = torch.from_numpy(x0).cuda()
+    c.sc_aggregate_apply(W, d_vals, d_idx[0].contiguous(), k, n, xs, shared=True)
+    assert c.sc_sync_status() == 0
+    assert_bits_equal(xs, O.aggregate_apply(x0, list(vals), [idx[0]] * W), "apply shared")
+    c.close()

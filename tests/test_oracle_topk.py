@@ -206,3 +206,23 @@ def test_segments_layerwise_vs_manual():
             assert np.array_equal(vals[pos:pos + k_s], p[sel])
             pos += k_s
         assert pos == len(idx)
+
+
+def test_aggregate_apply_is_dense_subtraction_and_leaves_the_rest_alone():
+    rng = np.random.default_rng(11)
+    W, n, k = 6, 400, 37
+    idx = [np.sort(rng.choice(n, k, replace=False)).astype(np.uint32) for _ in range(W)]
+    vals = [f32(rng.standard_normal(k)) for _ in range(W)]
+    x = f32(rng.standard_normal(n))
+    x2 = O.aggregate_apply(x, vals, idx)
+    touched = np.zeros(n, bool)
+    for i in idx:
+        touched[i] = True
+    assert np.array_equal(x2[~touched].view(np.uint32), x[~touched].view(np.uint32))
+    for i in np.nonzero(touched)[0][:50]:
+        acc = np.float32(0)
+        for w in range(W):
+            hit = np.nonzero(idx[w] == i)[0]
+            if hit.size:
+                acc = np.float32(acc + vals[w][hit[0]])
+        assert x2[i] == np.float32(x[i] - np.float32(acc / np.float32(W)))
