@@ -13,11 +13,12 @@
 
 namespace sc {
 
-constexpr uint32_t ATILE = 4096;
+constexpr uint32_t ATILE = 4096;          // default tile of the dense output
+constexpr uint32_t ATILE_BIG = 8192;      // used when the messages are sparse enough to stage a whole tile at once
 
-// bounds[r][t] = first slot j of row r with idx[j] >= t * ATILE, t = 0..ntiles.
+// bounds[r][t] = first slot j of row r with idx[j] >= t * tile, t = 0..ntiles.
 __global__ void __launch_bounds__(THREADS)
-agg_bounds_kernel(const uint32_t* __restrict__ idx, uint32_t rows, uint32_t K, uint32_t ntiles,
+agg_bounds_kernel(const uint32_t* __restrict__ idx, uint32_t rows, uint32_t K, uint32_t ntiles, uint32_t tile,
                   uint32_t* __restrict__ bounds) {
     const uint64_t gid = (uint64_t)blockIdx.x * THREADS + threadIdx.x;
     const uint64_t per_row = (uint64_t)ntiles + 1;
@@ -25,7 +26,7 @@ agg_bounds_kernel(const uint32_t* __restrict__ idx, uint32_t rows, uint32_t K, u
     const uint32_t r = (uint32_t)(gid / per_row);
     const uint32_t t = (uint32_t)(gid - (uint64_t)r * per_row);
     const uint32_t* row = idx + (size_t)r * K;
-    const uint64_t target = (uint64_t)t * ATILE;
+    const uint64_t target = (uint64_t)t * tile;
     uint32_t lo = 0, hi = K;                         // first j with row[j] >= target
     while (lo < hi) {
         const uint32_t mid = lo + ((hi - lo) >> 1);
@@ -34,18 +35,19 @@ agg_bounds_kernel(const uint32_t* __restrict__ idx, uint32_t rows, uint32_t K, u
     bounds[gid] = lo;
 }
 
-constexpr uint32_t AGG_STAGE = 2048;     // message entries staged in shared memory per round
+constexpr uint32_t AGG_STAGE = 1536;     // message entries staged in shared memory per round
 
 // One CTA per tile of ATILE coordinates.  The slices of all W messages that fall into the
 // tile are first fetched together into shared memory (one wave of independent loads), then
 // applied to the accumulator worker by worker, so the per-coordinate sum runs in worker
 // order without one global-memory round trip per worker.  With shared coordinates every
 // slot j carries W values, summed in registers in worker order.
+template <uint32_t AT>
 __global__ void __launch_bounds__(THREADS)
 agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
                  const uint32_t* __restrict__ bounds, uint32_t W, uint32_t shared_idx, uint32_t K,
                  uint32_t n, uint32_t ntiles, float* __restrict__ out, int* __restrict__ status) {
-    __shared__ __align__(16) float acc[ATILE];
+    __shared__ __align__(16) float acc[AT];
     __shared__ uint32_t st_loc[AGG_STAGE];
     __shared__ float st_val[AGG_STAGE];
     __shared__ uint32_t s_lo[64], s_off[65];
@@ -55,9 +57,9 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
     const bool pow2 = (W & (W - 1u)) == 0u;
     const float rW = 1.0f / fW;
     for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        const uint32_t tile_lo = t * ATILE;
-        const uint32_t tile_n = min(ATILE, n - tile_lo);
-        for (uint32_t i = threadIdx.x; i < ATILE / 4; i += THREADS)
+        const uint32_t tile_lo = t * AT;
+        const uint32_t tile_n = min(AT, n - tile_lo);
+        for (uint32_t i = threadIdx.x; i < AT / 4; i += THREADS)
             reinterpret_cast<float4*>(acc)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         if (shared_idx) {
             const uint32_t lo = bounds[t], hi = bounds[t + 1];
@@ -109,7 +111,7 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
                         if (a < b) {                             // uniform over the CTA
                             for (uint32_t q = a + threadIdx.x; q < b; q += THREADS) {
                                 const uint32_t loc = st_loc[q - cs];
-                                if (loc < ATILE) acc[loc] = acc[loc] + st_val[q - cs];
+                                if (loc < AT) acc[loc] = acc[loc] + st_val[q - cs];
                             }
                             __syncthreads();
                         }
@@ -119,8 +121,8 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
             __syncthreads();
         }
         float* o = out + tile_lo;
-        if (tile_n == ATILE) {
-            for (uint32_t i = threadIdx.x; i < ATILE / 4; i += THREADS) {
+        if (tile_n == AT) {
+            for (uint32_t i = threadIdx.x; i < AT / 4; i += THREADS) {
                 float4 a = reinterpret_cast<const float4*>(acc)[i];
                 if (pow2) { a.x *= rW; a.y *= rW; a.z *= rW; a.w *= rW; }
                 else { a.x = a.x / fW; a.y = a.y / fW; a.z = a.z / fW; a.w = a.w / fW; }
@@ -139,11 +141,12 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
 // materialised.  x - (+0.0) == x bit for bit, so skipping coordinates whose sum is zero gives
 // exactly what the dense formulation gives.
 // ---------------------------------------------------------------------------------------------
+template <uint32_t AT>
 __global__ void __launch_bounds__(THREADS)
 agg_apply_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
                        const uint32_t* __restrict__ bounds, uint32_t W, uint32_t K, uint32_t n, uint32_t ntiles,
                        float* __restrict__ x, int* __restrict__ status) {
-    __shared__ __align__(16) float acc[ATILE];
+    __shared__ __align__(16) float acc[AT];
     __shared__ uint32_t st_loc[AGG_STAGE];
     __shared__ float st_val[AGG_STAGE];
     __shared__ uint32_t s_lo[64], s_off[65];
@@ -151,8 +154,8 @@ agg_apply_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restric
     const bool pow2 = (W & (W - 1u)) == 0u;
     const float rW = 1.0f / fW;
     for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        const uint32_t tile_lo = t * ATILE;
-        const uint32_t tile_n = min(ATILE, n - tile_lo);
+        const uint32_t tile_lo = t * AT;
+        const uint32_t tile_n = min(AT, n - tile_lo);
         bool zeroed = false;
         for (uint32_t w0 = 0; w0 < W; w0 += 64) {
             const uint32_t wn = min(64u, W - w0);
@@ -172,7 +175,7 @@ agg_apply_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restric
             __syncthreads();
             const uint32_t total = s_off[wn];
             if (total && !zeroed) {                              // uniform: the tile is touched, start from +0.0
-                for (uint32_t i = threadIdx.x; i < ATILE / 4; i += THREADS)
+                for (uint32_t i = threadIdx.x; i < AT / 4; i += THREADS)
                     reinterpret_cast<float4*>(acc)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 zeroed = true;
                 __syncthreads();
@@ -198,7 +201,7 @@ agg_apply_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restric
                     if (a < b) {                                 // uniform over the CTA
                         for (uint32_t q = a + threadIdx.x; q < b; q += THREADS) {
                             const uint32_t loc = st_loc[q - cs];
-                            if (loc < ATILE) acc[loc] = acc[loc] + st_val[q - cs];
+                            if (loc < AT) acc[loc] = acc[loc] + st_val[q - cs];
                         }
                         __syncthreads();
                     }

@@ -68,7 +68,7 @@ struct sc_ctx {
     uint32_t epoch = 0;
     uint64_t launches = 0;
 
-    int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1;
+    int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1, occ_agg_big = 1;
 
     // optional per-kernel timing (sc_profile)
     bool prof_on = false;
@@ -379,18 +379,31 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
     return SC_OK;
 }
 
+// Tile of the dense output: the larger one halves the per-tile overhead, but only pays while all
+// slices of a tile fit the shared-memory staging area in one round.
+inline uint32_t aggregate_tile(int W, size_t k, size_t n) {
+    const double per_big_tile = (double)ATILE_BIG * (double)W * (double)k / (double)std::max<size_t>(n, 1);
+    return per_big_tile <= 0.9 * AGG_STAGE ? ATILE_BIG : ATILE;
+}
+
 int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, bool shared_idx, size_t k, size_t n,
                    float* out, cudaStream_t stream) {
     if (n == 0) return SC_OK;
-    const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
+    const uint32_t tile = aggregate_tile(shared_idx ? 1 : W, k, n);
+    const uint32_t ntiles = (uint32_t)((n + tile - 1) / tile);
     const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
     const uint64_t threads = (uint64_t)rows * (ntiles + 1ull);
     { Launch l(c, KIND_AGG_BOUNDS, stream);
       agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
-          idx, rows, (uint32_t)k, ntiles, c->d_bounds); }
+          idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds); }
     { Launch l(c, KIND_AGG_TILES, stream);
-      agg_tiles_kernel<<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, stream>>>(
-          vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status); }
+      const uint32_t grid = persistent_grid(c, tile == ATILE_BIG ? c->occ_agg_big : c->occ_agg, ntiles);
+      if (tile == ATILE_BIG)
+          agg_tiles_kernel<ATILE_BIG><<<grid, THREADS, 0, stream>>>(
+              vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+      else
+          agg_tiles_kernel<ATILE><<<grid, THREADS, 0, stream>>>(
+              vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status); }
     SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
@@ -483,7 +496,8 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_topk, pack_kernel<PACK_TOPK>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_mask, randk_pack_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_block, randblock_kernel, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel<ATILE>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_big, agg_tiles_kernel<ATILE_BIG>, THREADS, 0);
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
         c->max_main_grid = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
         if (rc == SC_OK) rc = dev_alloc(c, &c->d_cand_cnt, fastP * c->max_main_grid);
@@ -611,9 +625,9 @@ int sc_aggregate_apply(sc_ctx* c, int W, const float* vals, const uint32_t* idx,
     const uint64_t threads = (uint64_t)W * (ntiles + 1ull);
     { Launch l(c, KIND_AGG_BOUNDS, st);
       agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, st>>>(
-          idx, (uint32_t)W, (uint32_t)k, ntiles, c->d_bounds); }
+          idx, (uint32_t)W, (uint32_t)k, ntiles, ATILE, c->d_bounds); }
     { Launch l(c, KIND_AGG_APPLY, st);
-      agg_apply_tiles_kernel<<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, st>>>(
+      agg_apply_tiles_kernel<ATILE><<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, st>>>(
           vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, x, c->d_status); }
     SC_CUDA(cudaGetLastError());
     return SC_OK;
@@ -772,10 +786,10 @@ int sc_aggregate_static(int W, const float* vals, const uint32_t* idx, size_t k,
     const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
     const uint64_t threads = (uint64_t)W * (ntiles + 1ull);
     agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, st>>>(
-        idx, (uint32_t)W, (uint32_t)k, ntiles, bounds);
+        idx, (uint32_t)W, (uint32_t)k, ntiles, ATILE, bounds);
     const uint32_t grid = std::max(1u, std::min<uint32_t>(ntiles, (uint32_t)d.sm_count * 4u));
-    agg_tiles_kernel<<<grid, THREADS, 0, st>>>(vals, idx, bounds, (uint32_t)W, 0u, (uint32_t)k, (uint32_t)n, ntiles,
-                                               out, status);
+    agg_tiles_kernel<ATILE><<<grid, THREADS, 0, st>>>(vals, idx, bounds, (uint32_t)W, 0u, (uint32_t)k, (uint32_t)n, ntiles,
+                                                      out, status);
     SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
