@@ -28,6 +28,7 @@ struct sc_ctx {
     size_t scratch_bytes = 0;
 
     SegEntry* d_segs = nullptr;
+    uint32_t* d_fast_list = nullptr;
     uint32_t* d_hist = nullptr;
     TopkState* d_state = nullptr;
     unsigned long long* d_desc = nullptr;
@@ -157,6 +158,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         std::memcmp(c->cached_segs.data(), segs, sizeof(sc_segment) * nseg) == 0)
         return SC_OK;
     std::vector<SegEntry> h(nseg + 1);
+    std::vector<uint32_t> fast_list;
     uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0, cand = 0, flag = 0;
     uint32_t fast_count = 0, slow_count = 0, max_m = 0, max_cap = 0;
     for (int s = 0; s < nseg; ++s) {
@@ -173,6 +175,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             uint64_t m = (g.n / 16) & ~7ull;
             m = std::min<uint64_t>(std::max<uint64_t>(m, SAMPLE_MIN), SAMPLE_MAX);
             e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
+            fast_list.push_back((uint32_t)s);
             // The main pass gives each of its CTAs a private region of the segment's flagged and
             // candidate lists.  A CTA sees at most ceil(tiles / CTAs) tiles of the segment; a region
             // holds that many tiles' share of (k + slack) resp. slack entries, slack = n / 32 + 16384.
@@ -217,8 +220,11 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw; sentinel.grp_begin = (uint32_t)groups;
     h[nseg] = sentinel;
     SC_CUDA(cudaMemcpyAsync(c->d_segs, h.data(), sizeof(SegEntry) * (nseg + 1), cudaMemcpyHostToDevice, stream));
+    if (!fast_list.empty())
+        SC_CUDA(cudaMemcpyAsync(c->d_fast_list, fast_list.data(), sizeof(uint32_t) * fast_list.size(),
+                                cudaMemcpyHostToDevice, stream));
     Layout L{};
-    L.segs = c->d_segs; L.nseg = (uint32_t)nseg; L.tiles_per_worker = (uint32_t)tiles; L.groups_per_worker = (uint32_t)groups;
+    L.segs = c->d_segs; L.fast_list = c->d_fast_list; L.nseg = (uint32_t)nseg; L.tiles_per_worker = (uint32_t)tiles; L.groups_per_worker = (uint32_t)groups;
     L.scat_per_group = (uint32_t)scat; L.K_total = (uint32_t)msg; L.n_total = n; L.mask_words_per_group = maskw;
     L.cand_per_worker = cand; L.flag_per_worker = flag; L.fast_per_worker = fast_count;
     c->layout = L;
@@ -273,6 +279,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
         const uint32_t counters[2] = {n_slow0, 0u};
         SC_CUDA(cudaMemcpyAsync(c->d_nslow, counters, sizeof(counters), cudaMemcpyHostToDevice, stream));
         if (L.fast_per_worker) {
+            const uint32_t PF = (uint32_t)W * L.fast_per_worker;       // fast (worker, segment) pairs
             FastParams fp{};
             fp.L = L; fp.grads = grads; fp.residuals = residuals; fp.out_vals = out_vals; fp.out_idx = out_idx;
             fp.state = c->d_fstate; fp.sample = c->d_sample; fp.cand_hist = c->d_cand_hist;
@@ -285,17 +292,17 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             SC_CUDA(cudaMemsetAsync(c->d_tile_sure, 0, (size_t)items * sizeof(uint32_t), stream));
             SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
             { Launch l(c, KIND_SAMPLE, stream);
-              topk_sample_kernel<<<dim3((c->max_sample_m / 8 + THREADS - 1) / THREADS, P), THREADS, 0, stream>>>(fp); }
+              topk_sample_kernel<<<dim3((c->max_sample_m / 8 + THREADS - 1) / THREADS, PF), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_BRACKET, stream);
-              topk_bracket_kernel<<<P, THREADS, 0, stream>>>(fp); }
+              topk_bracket_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_MAIN, stream);
               topk_main_kernel<<<fp.grid_main, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDBIN, stream);
-              topk_candbin_kernel<<<P, THREADS, 0, stream>>>(fp); }
+              topk_candbin_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDFILTER, stream);
-              topk_candfilter_kernel<<<dim3(fp.grid_main, P), THREADS, 0, stream>>>(fp); }
+              topk_candfilter_kernel<<<dim3(std::min<uint32_t>(fp.grid_main, 64u), PF), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_FINAL, stream);
-              topk_final_kernel<<<P, THREADS, 0, stream>>>(fp); }
+              topk_final_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_RESTORE, stream);
               const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
               topk_restore_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
@@ -463,6 +470,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     const size_t fastP = (size_t)max_W * c->max_fast_per_worker;
     int rc = SC_OK;
     if ((rc = dev_alloc(c, &c->d_segs, (size_t)max_segments + 1)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_fast_list, (size_t)max_segments)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_hist, P * HIST_WORDS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_state, P)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_desc, (size_t)max_W * c->max_tiles_per_worker * 2)) == SC_OK &&
@@ -510,7 +518,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
 void sc_destroy(sc_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
-    cudaFree(c->d_segs); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
+    cudaFree(c->d_segs); cudaFree(c->d_fast_list); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
     cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate); cudaFree(c->d_sample);
     cudaFree(c->d_cand_hist); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_cbase);
     cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt); cudaFree(c->d_cand_cnt);

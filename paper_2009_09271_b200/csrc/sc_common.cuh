@@ -41,6 +41,7 @@ struct SegEntry {
 
 struct Layout {
     const SegEntry* segs;     // device array, nseg + 1 entries (last = sentinel with the totals)
+    const uint32_t* fast_list; // device array: segment index of the i-th fast segment
     uint32_t nseg;
     uint32_t tiles_per_worker;
     uint32_t groups_per_worker;

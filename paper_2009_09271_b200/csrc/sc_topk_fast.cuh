@@ -53,6 +53,14 @@ struct FastParams {
     uint32_t total_items;
 };
 
+// The per-segment kernels of this path are launched over the fast segments only: block index
+// f = w * fast_per_worker + fast_index, mapped to the segment through the layout's fast list.
+__device__ inline uint32_t fast_problem(const Layout& L, uint32_t f, uint32_t& w, uint32_t& s) {
+    w = f / L.fast_per_worker;
+    s = L.fast_list[f - w * L.fast_per_worker];
+    return w * L.nseg + s;
+}
+
 // ---- shared helper: walk a histogram from its highest bin down to the bin that holds the
 // need-th largest element.  All THREADS threads call it; results are uniform.
 template <uint32_t BINS, typename HistPtr>
@@ -91,10 +99,9 @@ __device__ inline bool find_from_top(HistPtr h, uint32_t need, uint32_t* s_tmp /
 __global__ void __launch_bounds__(THREADS)
 topk_sample_kernel(FastParams P) {
     const Layout& L = P.L;
-    const uint32_t prob = blockIdx.y;
-    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    uint32_t w, s;
+    fast_problem(L, blockIdx.y, w, s);
     const SegEntry seg = L.segs[s];
-    if (!seg.fast) return;
     const uint32_t c = blockIdx.x * THREADS + threadIdx.x;            // sector of the sample
     if (c >= seg.sample_m / 8u) return;
     const size_t row = (size_t)w * L.n_total + seg.offset;
@@ -120,10 +127,9 @@ topk_bracket_kernel(FastParams P) {
     __shared__ uint32_t hA[1024], hB[1024];
     __shared__ uint32_t s_tmp[WARPS + 4];
     const Layout& L = P.L;
-    const uint32_t prob = blockIdx.x;
-    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    uint32_t w, s;
+    const uint32_t prob = fast_problem(L, blockIdx.x, w, s);
     const SegEntry seg = L.segs[s];
-    if (!seg.fast) return;
     const uint32_t m = seg.sample_m;
     const uint4* smp = reinterpret_cast<const uint4*>(P.sample + ((size_t)w * L.fast_per_worker + seg.fast_index) * SAMPLE_MAX);
     // ranks (from the top) that bracket the k-th largest of the segment
@@ -377,10 +383,9 @@ __global__ void __launch_bounds__(THREADS)
 topk_candbin_kernel(FastParams P) {
     __shared__ uint32_t s_tmp[WARPS + 4];
     const Layout& L = P.L;
-    const uint32_t prob = blockIdx.x;
-    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    uint32_t w, s;
+    const uint32_t prob = fast_problem(L, blockIdx.x, w, s);
     const SegEntry seg = L.segs[s];
-    if (!seg.fast) return;
     FastState st = P.state[prob];
     if (st.path != PATH_FAST) return;
     const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
@@ -415,10 +420,9 @@ topk_candbin_kernel(FastParams P) {
 __global__ void __launch_bounds__(THREADS)
 topk_candfilter_kernel(FastParams P) {
     const Layout& L = P.L;
-    const uint32_t prob = blockIdx.y;
-    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    uint32_t w, s;
+    const uint32_t prob = fast_problem(L, blockIdx.y, w, s);
     const SegEntry seg = L.segs[s];
-    if (!seg.fast) return;
     const FastState* stp = P.state + prob;
     if (stp->path != PATH_FAST || stp->need2 == 0) return;
     const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
@@ -443,9 +447,8 @@ __global__ void __launch_bounds__(THREADS)
 topk_final_kernel(FastParams P) {
     __shared__ unsigned long long srt[LIST2_CAP];
     const Layout& L = P.L;
-    const uint32_t prob = blockIdx.x;
-    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
-    if (!L.segs[s].fast) return;
+    uint32_t w, s;
+    const uint32_t prob = fast_problem(L, blockIdx.x, w, s);
     FastState st = P.state[prob];
     if (st.path != PATH_FAST || st.need2 == 0) return;
     const uint32_t cnt = st.cnt2;
