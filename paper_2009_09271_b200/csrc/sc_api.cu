@@ -29,6 +29,8 @@ struct sc_ctx {
 
     SegEntry* d_segs = nullptr;
     uint32_t* d_fast_list = nullptr;
+    uint32_t* d_lists = nullptr;     // slow tiles | fast tiles | slow pack groups | fast pack groups (each max_tiles long)
+    uint32_t n_slow_tiles = 0, n_fast_tiles = 0, n_slow_groups = 0, n_fast_groups = 0;
     uint32_t* d_hist = nullptr;
     TopkState* d_state = nullptr;
     unsigned long long* d_desc = nullptr;
@@ -47,7 +49,6 @@ struct sc_ctx {
     uint32_t* d_tile_ccnt = nullptr;
     uint32_t* d_tile_fbase = nullptr;
     uint32_t* d_tile_fcnt = nullptr;
-    uint32_t* d_cand_cnt = nullptr;  // [W * fast_per_worker][main grid]
     size_t max_main_grid = 0;
     uint2* d_flagged = nullptr;      // grown on demand: its size depends on k
     size_t flagged_slots = 0;
@@ -158,8 +159,8 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         std::memcmp(c->cached_segs.data(), segs, sizeof(sc_segment) * nseg) == 0)
         return SC_OK;
     std::vector<SegEntry> h(nseg + 1);
-    std::vector<uint32_t> fast_list;
-    uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0, cand = 0, flag = 0;
+    std::vector<uint32_t> fast_list, lists[4];
+    uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0, cand = 0, flag = 0, smp = 0;
     uint32_t fast_count = 0, slow_count = 0, max_m = 0, max_cap = 0;
     for (int s = 0; s < nseg; ++s) {
         const sc_segment& g = segs[s];
@@ -175,27 +176,34 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             uint64_t m = (g.n / 16) & ~7ull;
             m = std::min<uint64_t>(std::max<uint64_t>(m, SAMPLE_MIN), SAMPLE_MAX);
             e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
+            e.sample_begin = smp; smp += m;
             fast_list.push_back((uint32_t)s);
-            // The main pass gives each of its CTAs a private region of the segment's flagged and
-            // candidate lists.  A CTA sees at most ceil(tiles / CTAs) tiles of the segment; a region
-            // holds that many tiles' share of (k + slack) resp. slack entries, slack = n / 32 + 16384.
-            const uint64_t slack = g.n / 32 + 16384;
-            const uint64_t ctas = std::max<uint64_t>(1, std::min<uint64_t>(c->max_main_grid, seg_tiles));
-            const uint64_t tiles_per_cta = (seg_tiles + ctas - 1) / ctas;
-            const uint64_t cand_region = tiles_per_cta * ((slack + seg_tiles - 1) / seg_tiles + 16);
-            const uint64_t flag_region = tiles_per_cta * ((g.k + slack + seg_tiles - 1) / seg_tiles + 16);
-            if (flag_region * c->max_main_grid > 0xFFFFFFFFull) return SC_ERR_RANGE;
-            e.cand_cap = (uint32_t)cand_region;          // per CTA
-            e.flag_cap = (uint32_t)flag_region;          // per CTA
+            // The main pass appends to private regions of the segment's flagged and candidate lists:
+            // one region per tile when the segment has no more tiles than the pass has CTAs, else one
+            // per CTA (which sees at most ceil(tiles / CTAs) tiles of the segment).  A region holds its
+            // tiles' share of (k + slack) resp. slack entries plus a little room per tile.
+            const bool per_tile = seg_tiles <= c->max_main_grid;
+            const uint64_t slack = per_tile ? g.n / 16 + 1024 : g.n / 32 + 16384;
+            const uint64_t regions = per_tile ? seg_tiles : c->max_main_grid;
+            const uint64_t tiles_per_region = per_tile ? 1 : (seg_tiles + regions - 1) / regions;
+            const uint64_t cand_region = tiles_per_region * ((slack + seg_tiles - 1) / seg_tiles + 16);
+            const uint64_t flag_region = tiles_per_region * ((g.k + slack + seg_tiles - 1) / seg_tiles + 16);
+            if (flag_region * regions > 0xFFFFFFFFull) return SC_ERR_RANGE;
+            e.region_per_tile = per_tile ? 1u : 0u;
+            e.cand_cap = (uint32_t)cand_region;
+            e.flag_cap = (uint32_t)flag_region;
             e.cand_begin = cand;
             e.flag_begin = flag;
-            cand += cand_region * c->max_main_grid;
-            flag += flag_region * c->max_main_grid;
+            cand += cand_region * regions;
+            flag += flag_region * regions;
             max_m = std::max(max_m, e.sample_m);
         } else {
             ++slow_count;
         }
         h[s] = e;
+        const int which = e.fast ? 1 : 0;
+        for (uint64_t t = 0; t < seg_tiles; ++t) lists[which].push_back((uint32_t)(tiles + t));
+        for (uint64_t t = 0; t < (seg_tiles + PACK_GROUP - 1) / PACK_GROUP; ++t) lists[2 + which].push_back((uint32_t)(groups + t));
         tiles += seg_tiles;
         groups += (seg_tiles + PACK_GROUP - 1) / PACK_GROUP;
         scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
@@ -204,29 +212,37 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     }
     if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
     if (fast_count > c->max_fast_per_worker) return SC_ERR_RANGE;
-    if ((size_t)c->max_W * (flag + cand) > c->flagged_slots) {   // the lists follow k: grow them (synchronous, rare)
+    const size_t smp_slots = ((size_t)c->max_W * smp + 1) / 2 + 1;  // sample keys are 4 bytes, list entries 8; +1 to align
+    if ((size_t)c->max_W * (flag + cand) + smp_slots > c->flagged_slots) {   // the lists follow k: grow them (synchronous, rare)
         SC_CUDA(cudaStreamSynchronize(stream));
         cudaFree(c->d_flagged); c->d_flagged = nullptr;
         c->scratch_bytes -= c->flagged_slots * sizeof(uint2);
         c->flagged_slots = 0;
-        const size_t want = (size_t)c->max_W * (flag + cand);
+        const size_t want = (size_t)c->max_W * (flag + cand) + smp_slots;
         if (cudaMalloc(reinterpret_cast<void**>(&c->d_flagged), want * sizeof(uint2)) != cudaSuccess) return SC_ERR_WORKSPACE;
         c->flagged_slots = want;
         c->scratch_bytes += want * sizeof(uint2);
     }
     c->d_cand = c->d_flagged + (size_t)c->max_W * flag;         // candidate lists live behind the flagged lists
+    c->d_sample = reinterpret_cast<uint32_t*>(c->d_flagged + (((size_t)c->max_W * (flag + cand) + 1) & ~(size_t)1));   // then the sample keys, 16-byte aligned
     SegEntry sentinel{};
     sentinel.offset = n; sentinel.msg_off = (uint32_t)msg; sentinel.tile_begin = (uint32_t)tiles;
     sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw; sentinel.grp_begin = (uint32_t)groups;
     h[nseg] = sentinel;
     SC_CUDA(cudaMemcpyAsync(c->d_segs, h.data(), sizeof(SegEntry) * (nseg + 1), cudaMemcpyHostToDevice, stream));
+    for (int i = 0; i < 4; ++i)
+        if (!lists[i].empty())
+            SC_CUDA(cudaMemcpyAsync(c->d_lists + (size_t)i * c->max_tiles_per_worker, lists[i].data(),
+                                    sizeof(uint32_t) * lists[i].size(), cudaMemcpyHostToDevice, stream));
+    c->n_slow_tiles = (uint32_t)lists[0].size(); c->n_fast_tiles = (uint32_t)lists[1].size();
+    c->n_slow_groups = (uint32_t)lists[2].size(); c->n_fast_groups = (uint32_t)lists[3].size();
     if (!fast_list.empty())
         SC_CUDA(cudaMemcpyAsync(c->d_fast_list, fast_list.data(), sizeof(uint32_t) * fast_list.size(),
                                 cudaMemcpyHostToDevice, stream));
     Layout L{};
     L.segs = c->d_segs; L.fast_list = c->d_fast_list; L.nseg = (uint32_t)nseg; L.tiles_per_worker = (uint32_t)tiles; L.groups_per_worker = (uint32_t)groups;
     L.scat_per_group = (uint32_t)scat; L.K_total = (uint32_t)msg; L.n_total = n; L.mask_words_per_group = maskw;
-    L.cand_per_worker = cand; L.flag_per_worker = flag; L.fast_per_worker = fast_count;
+    L.cand_per_worker = cand; L.flag_per_worker = flag; L.sample_per_worker = smp; L.fast_per_worker = fast_count;
     c->layout = L;
     c->slow_segments = slow_count; c->max_sample_m = max_m; c->max_flag_cap = max_cap;
     c->cached_segs.assign(segs, segs + nseg);
@@ -285,10 +301,8 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             fp.state = c->d_fstate; fp.sample = c->d_sample; fp.cand_hist = c->d_cand_hist;
             fp.list2 = c->d_list2; fp.cand = c->d_cand; fp.tile_sure = c->d_tile_sure; fp.tile_cbase = c->d_tile_cbase;
             fp.tile_ccnt = c->d_tile_ccnt; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
-            fp.flagged = c->d_flagged; fp.cand_cnt = c->d_cand_cnt; fp.offsets = c->d_offsets;
-            fp.grid_main = persistent_grid(c, c->occ_main, items);
+            fp.flagged = c->d_flagged; fp.offsets = c->d_offsets;
             fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
-            SC_CUDA(cudaMemsetAsync(c->d_cand_cnt, 0, (size_t)W * L.fast_per_worker * fp.grid_main * sizeof(uint32_t), stream));
             SC_CUDA(cudaMemsetAsync(c->d_tile_sure, 0, (size_t)items * sizeof(uint32_t), stream));
             SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
             { Launch l(c, KIND_SAMPLE, stream);
@@ -296,11 +310,11 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             { Launch l(c, KIND_BRACKET, stream);
               topk_bracket_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_MAIN, stream);
-              topk_main_kernel<<<fp.grid_main, THREADS, 0, stream>>>(fp); }
+              topk_main_kernel<<<persistent_grid(c, c->occ_main, items), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDBIN, stream);
               topk_candbin_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDFILTER, stream);
-              topk_candfilter_kernel<<<dim3(std::min<uint32_t>(fp.grid_main, 64u), PF), THREADS, 0, stream>>>(fp); }
+              topk_candfilter_kernel<<<(uint32_t)(((uint64_t)items * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_FINAL, stream);
               topk_final_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_RESTORE, stream);
@@ -314,19 +328,36 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
               topk_emit_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
         }
-        { Launch l(c, KIND_HIST0, stream);
-          topk_hist0_kernel<<<persistent_grid(c, c->occ_hist, items), THREADS, 0, stream>>>(
-              L, grads, residuals, c->d_hist, c->d_fstate, c->d_nslow, items); }
+        // Radix select: once over the small segments (if any), once over the large ones, where the
+        // launch returns at once unless some segment's bracket missed.
+        WorkList lists[2];
+        lists[0] = WorkList{c->d_lists, c->d_nslow, c->n_slow_tiles, 0u};
+        lists[1] = WorkList{c->d_lists + c->max_tiles_per_worker, c->d_nslow + 1, c->n_fast_tiles, 0u};
+        for (int pass = 0; pass < 2; ++pass) {
+            if (!lists[pass].len) continue;
+            const uint32_t n_it = (uint32_t)W * lists[pass].len;
+            Launch l(c, KIND_HIST0, stream);
+            topk_hist0_kernel<<<persistent_grid(c, c->occ_hist, n_it), THREADS, 0, stream>>>(
+                L, grads, residuals, c->d_hist, c->d_fstate, lists[pass], n_it);
+        }
         { Launch l(c, KIND_RESOLVE, stream);
           topk_resolve_kernel<0><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
-        { Launch l(c, KIND_REFINE, stream);
-          topk_refine_kernel<1><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
-              L, residuals, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, items); }
+        for (int pass = 0; pass < 2; ++pass) {
+            if (!lists[pass].len) continue;
+            const uint32_t n_it = (uint32_t)W * lists[pass].len;
+            Launch l(c, KIND_REFINE, stream);
+            topk_refine_kernel<1><<<persistent_grid(c, c->occ_refine, n_it), THREADS, 0, stream>>>(
+                L, residuals, c->d_hist, c->d_state, c->d_fstate, lists[pass], n_it);
+        }
         { Launch l(c, KIND_RESOLVE, stream);
           topk_resolve_kernel<1><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
-        { Launch l(c, KIND_REFINE, stream);
-          topk_refine_kernel<2><<<persistent_grid(c, c->occ_refine, items), THREADS, 0, stream>>>(
-              L, residuals, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, items); }
+        for (int pass = 0; pass < 2; ++pass) {
+            if (!lists[pass].len) continue;
+            const uint32_t n_it = (uint32_t)W * lists[pass].len;
+            Launch l(c, KIND_REFINE, stream);
+            topk_refine_kernel<2><<<persistent_grid(c, c->occ_refine, n_it), THREADS, 0, stream>>>(
+                L, residuals, c->d_hist, c->d_state, c->d_fstate, lists[pass], n_it);
+        }
         { Launch l(c, KIND_RESOLVE, stream);
           topk_resolve_kernel<2><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
     } else {
@@ -369,19 +400,22 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
     PackParams pp{};
     pp.L = L; pp.grads = grads; pp.residuals = residuals; pp.out_vals = out_vals; pp.out_idx = out_idx;
     pp.state = c->d_state; pp.mask = c->d_mask; pp.mask_per_worker = 0u;
-    pp.fstate = c->d_fstate; pp.n_slow = c->d_nslow;
-    SC_CUDA(cudaMemsetAsync(c->d_ticket, 0, sizeof(unsigned long long), stream));
-    if (++c->epoch >= (1u << 28)) {            // tags wrapped: forget every old word
-        SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), stream));
-        c->epoch = 1;
+    pp.fstate = c->d_fstate;
+    pp.ticket = c->d_ticket; pp.desc = c->d_desc; pp.status = c->d_status;
+    for (int pass = 0; pass < 2; ++pass) {
+        const uint32_t len = pass == 0 ? c->n_slow_groups : c->n_fast_groups;
+        if (!len) continue;
+        pp.wl = WorkList{c->d_lists + (size_t)(2 + pass) * c->max_tiles_per_worker, c->d_nslow + pass, len, 0u};
+        SC_CUDA(cudaMemsetAsync(c->d_ticket, 0, sizeof(unsigned long long), stream));
+        if (++c->epoch >= (1u << 28)) {        // tags wrapped: forget every old word
+            SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), stream));
+            c->epoch = 1;
+        }
+        const uint32_t gitems = (uint32_t)W * len;
+        pp.epoch = c->epoch; pp.total_items = gitems;
+        Launch l(c, KIND_PACK_TOPK, stream);
+        pack_kernel<PACK_TOPK><<<persistent_grid(c, c->occ_pack_topk, gitems), THREADS, 0, stream>>>(pp);
     }
-    const uint32_t gitems = (uint32_t)W * L.groups_per_worker;
-    pp.epoch = c->epoch; pp.total_items = gitems;
-    pp.ticket = c->d_ticket;
-    pp.desc = c->d_desc; pp.status = c->d_status;
-    const uint32_t grid = persistent_grid(c, c->occ_pack_topk, gitems);
-    { Launch l(c, KIND_PACK_TOPK, stream);
-      pack_kernel<PACK_TOPK><<<grid, THREADS, 0, stream>>>(pp); }
     SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
@@ -464,13 +498,14 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     c->max_mask_words = (max_n + 31) / 32 + (size_t)max_segments;
     c->max_atiles = (max_n + ATILE - 1) / ATILE;
     const size_t P = (size_t)max_W * max_segments;
-    c->max_fast_per_worker = std::min<size_t>((size_t)max_segments, std::max<size_t>(1, max_n >> 20));
+    c->max_fast_per_worker = std::min<size_t>((size_t)max_segments, std::max<size_t>(1, max_n >> 16));
     c->max_cand_per_worker = max_n / 32 + c->max_fast_per_worker * 16384;
     const size_t items_max = (size_t)max_W * c->max_tiles_per_worker;
     const size_t fastP = (size_t)max_W * c->max_fast_per_worker;
     int rc = SC_OK;
     if ((rc = dev_alloc(c, &c->d_segs, (size_t)max_segments + 1)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_fast_list, (size_t)max_segments)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_lists, 4 * c->max_tiles_per_worker)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_hist, P * HIST_WORDS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_state, P)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_desc, (size_t)max_W * c->max_tiles_per_worker * 2)) == SC_OK &&
@@ -479,7 +514,6 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_bounds, (size_t)max_W * (c->max_atiles + 1))) == SC_OK &&
         (rc = dev_alloc(c, &c->d_offsets, (size_t)max_W * (c->max_tiles_per_worker + 1))) == SC_OK &&
         (rc = dev_alloc(c, &c->d_fstate, P)) == SC_OK &&
-        (rc = dev_alloc(c, &c->d_sample, fastP * SAMPLE_MAX)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_cand_hist, fastP * CAND_BINS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_list2, fastP * LIST2_CAP)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_sure, items_max)) == SC_OK &&
@@ -508,7 +542,6 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_big, agg_tiles_kernel<ATILE_BIG>, THREADS, 0);
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
         c->max_main_grid = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
-        if (rc == SC_OK) rc = dev_alloc(c, &c->d_cand_cnt, fastP * c->max_main_grid);
     }
     if (rc != SC_OK) { sc_destroy(c); return rc; }
     *out = c;
@@ -518,10 +551,10 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
 void sc_destroy(sc_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
-    cudaFree(c->d_segs); cudaFree(c->d_fast_list); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
-    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate); cudaFree(c->d_sample);
+    cudaFree(c->d_segs); cudaFree(c->d_fast_list); cudaFree(c->d_lists); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
+    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate);
     cudaFree(c->d_cand_hist); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_cbase);
-    cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt); cudaFree(c->d_cand_cnt);
+    cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt);
     cudaFree(c->d_flagged); cudaFree(c->d_nslow); cudaFree(c->d_seeds); cudaFree(c->d_status);
     cudaFree(c->d_stage_grads); cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); cudaFree(c->d_stage_out);
     for (cudaEvent_t e : c->ev_worker) cudaEventDestroy(e);

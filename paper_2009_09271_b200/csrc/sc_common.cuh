@@ -31,12 +31,13 @@ struct SegEntry {
     uint32_t grp_begin;       // first pack group (PACK_GROUP tiles) of the segment inside a worker
     uint32_t fast;            // 1: large segment, top-k goes through the sampled-bracket path
     uint32_t sample_m;        // sample size of that path (multiple of 8)
-    uint32_t cand_cap;        // capacity of ONE main-pass CTA's region of the segment's candidate list
+    uint32_t cand_cap;        // capacity of ONE region of the segment's candidate list
     uint32_t fast_index;      // index among the fast segments of a worker
     uint64_t cand_begin;      // first candidate slot of the segment inside a worker
     uint64_t flag_begin;      // first flagged-list slot of the segment inside a worker
-    uint32_t flag_cap;        // capacity of ONE main-pass CTA's region of the segment's flagged list
-    uint32_t pad;
+    uint32_t flag_cap;        // capacity of ONE region of the segment's flagged list
+    uint32_t region_per_tile; // 1: one list region per tile (few tiles), 0: one per CTA of the main pass
+    uint64_t sample_begin;    // first sample key of the segment inside a worker
 };
 
 struct Layout {
@@ -51,7 +52,17 @@ struct Layout {
     uint64_t mask_words_per_group;
     uint64_t cand_per_worker; // candidate slots per worker (all fast segments)
     uint64_t flag_per_worker; // flagged-list slots per worker
+    uint64_t sample_per_worker; // sample keys per worker
     uint32_t fast_per_worker; // fast segments per worker
+    uint32_t pad;
+};
+
+// The tiles (or pack groups) one launch of a radix-select kernel walks: indices inside a worker row,
+// the same list for every worker.  The launch returns at once when *gate == 0.
+struct WorkList {
+    const uint32_t* ids;
+    const uint32_t* gate;
+    uint32_t len;
     uint32_t pad;
 };
 
@@ -84,8 +95,8 @@ struct FastState {
     uint32_t pad[3];
 };
 
-constexpr uint32_t FAST_MIN_N = 1u << 20;
-constexpr uint32_t SAMPLE_MIN = 1u << 14, SAMPLE_MAX = 1u << 18;
+constexpr uint32_t FAST_MIN_N = 1u << 16;
+constexpr uint32_t SAMPLE_MIN = 1u << 12, SAMPLE_MAX = 1u << 18;
 constexpr uint32_t CAND_BINS = 2048;
 constexpr uint32_t LIST2_CAP = 4096;
 

@@ -33,7 +33,7 @@ struct PackParams {
     uint32_t* out_idx;
     const TopkState* state;          // PACK_TOPK
     const FastState* fstate;         // segments already served by the sampled-bracket path are skipped
-    const uint32_t* n_slow;          // 0: nothing to do for this launch
+    WorkList wl;                     // the pack groups this launch walks
     const uint32_t* mask;            // PACK_MASK
     uint32_t mask_per_worker;        // 1: worker w uses mask group w, 0: all use group 0
     uint32_t epoch;                  // tag of this launch inside the descriptor words
@@ -151,7 +151,7 @@ pack_kernel(PackParams P) {
     __shared__ uint32_t s_grp_excl[2];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const Layout& L = P.L;
-    if (*P.n_slow == 0u) return;
+    if (*P.wl.gate == 0u) return;
 
     while (true) {
         if (threadIdx.x == 0) {
@@ -159,8 +159,8 @@ pack_kernel(PackParams P) {
             uint32_t item = tk < (unsigned long long)P.total_items ? (uint32_t)tk : 0xFFFFFFFFu;
             s_dec[0] = item;
             if (item != 0xFFFFFFFFu) {
-                uint32_t w = item / L.groups_per_worker;
-                uint32_t lg = item - w * L.groups_per_worker;
+                uint32_t w = item / P.wl.len;
+                uint32_t lg = P.wl.ids[item - w * P.wl.len];
                 uint32_t s = find_by_group(L, lg);
                 const SegEntry sg = L.segs[s];
                 uint32_t gi = lg - sg.grp_begin;                              // group inside the segment

@@ -31,17 +31,17 @@ __device__ inline void flush_hist(uint32_t* sh, uint32_t* __restrict__ gh) {
 __global__ void __launch_bounds__(THREADS)
 topk_hist0_kernel(Layout L, const float* __restrict__ grads, float* __restrict__ residuals,
                   uint32_t* __restrict__ hist, const FastState* __restrict__ fstate,
-                  const uint32_t* __restrict__ n_slow, uint32_t total_items) {
+                  WorkList wl, uint32_t total_items) {
     __shared__ uint32_t sh[HIST0_BINS];
     __shared__ uint32_t s_dec[4];
-    if (*n_slow == 0u) return;
+    if (*wl.gate == 0u) return;
     for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) sh[b] = 0;
     __syncthreads();
     long long cur_prob = -1;
     for (uint32_t item = blockIdx.x; item < total_items; item += gridDim.x) {
         if (threadIdx.x == 0) {
-            uint32_t w = item / L.tiles_per_worker;
-            uint32_t lt = item - w * L.tiles_per_worker;
+            uint32_t w = item / wl.len;
+            uint32_t lt = wl.ids[item - w * wl.len];
             uint32_t s = find_by_tile(L, lt);
             s_dec[0] = w; s_dec[1] = s; s_dec[2] = lt - L.segs[s].tile_begin;
             s_dec[3] = fstate[(size_t)w * L.nseg + s].path;
@@ -96,19 +96,19 @@ template <int LEVEL>
 __global__ void __launch_bounds__(THREADS)
 topk_refine_kernel(Layout L, const float* __restrict__ residuals, uint32_t* __restrict__ hist,
                    const TopkState* __restrict__ state, const FastState* __restrict__ fstate,
-                   const uint32_t* __restrict__ n_slow, uint32_t total_items) {
+                   WorkList wl, uint32_t total_items) {
     constexpr uint32_t SHIFT = (LEVEL == 1) ? 10u : 0u;
     constexpr uint32_t HOFF = (LEVEL == 1) ? HIST0_BINS : HIST0_BINS + HIST1_BINS;
     __shared__ uint32_t sh[1024];
     __shared__ uint32_t s_dec[3];
-    if (*n_slow == 0u) return;
+    if (*wl.gate == 0u) return;
     for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) sh[b] = 0;
     __syncthreads();
     long long cur_prob = -1;
     for (uint32_t item = blockIdx.x; item < total_items; item += gridDim.x) {
         if (threadIdx.x == 0) {
-            uint32_t w = item / L.tiles_per_worker;
-            uint32_t lt = item - w * L.tiles_per_worker;
+            uint32_t w = item / wl.len;
+            uint32_t lt = wl.ids[item - w * wl.len];
             uint32_t s = find_by_tile(L, lt);
             s_dec[0] = w; s_dec[1] = s; s_dec[2] = lt - L.segs[s].tile_begin;
         }

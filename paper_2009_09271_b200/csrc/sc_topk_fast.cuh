@@ -34,7 +34,7 @@ struct FastParams {
     float* out_vals;
     uint32_t* out_idx;
     FastState* state;          // [W * nseg]
-    uint32_t* sample;          // [W * fast_per_worker][SAMPLE_MAX]
+    uint32_t* sample;          // [W][sample_per_worker]
     uint32_t* cand_hist;       // [W * fast_per_worker][CAND_BINS]
     uint2* list2;              // [W * fast_per_worker][LIST2_CAP]
     uint2* flagged;            // [W][flag_per_worker] (value bits, coordinate inside the segment)
@@ -44,8 +44,6 @@ struct FastParams {
     uint32_t* tile_ccnt;       // candidates of the tile
     uint32_t* tile_fbase;      // first flagged slot of the tile (0xFFFFFFFF: the list was full, nothing written)
     uint32_t* tile_fcnt;       // flagged elements of the tile
-    uint32_t* cand_cnt;        // [W * fast_per_worker][grid_main]: candidates each CTA of the main pass wrote
-    uint32_t grid_main;        // CTAs of the main pass: every list is cut into that many private regions
     uint32_t* n_failed;        // segments whose bracket missed
     uint32_t* offsets;         // [W][tiles_per_worker + 1]
     uint32_t* n_slow;          // segments that need the radix-select path
@@ -116,7 +114,7 @@ topk_sample_kernel(FastParams P) {
     uint4 k0, k1;
     k0.x = key_of(g0.x + e0.x); k0.y = key_of(g0.y + e0.y); k0.z = key_of(g0.z + e0.z); k0.w = key_of(g0.w + e0.w);
     k1.x = key_of(g1.x + e1.x); k1.y = key_of(g1.y + e1.y); k1.z = key_of(g1.z + e1.z); k1.w = key_of(g1.w + e1.w);
-    uint4* out = reinterpret_cast<uint4*>(P.sample + ((size_t)w * L.fast_per_worker + seg.fast_index) * SAMPLE_MAX + (size_t)c * 8u);
+    uint4* out = reinterpret_cast<uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin + (size_t)c * 8u);
     out[0] = k0; out[1] = k1;
 }
 
@@ -131,7 +129,7 @@ topk_bracket_kernel(FastParams P) {
     const uint32_t prob = fast_problem(L, blockIdx.x, w, s);
     const SegEntry seg = L.segs[s];
     const uint32_t m = seg.sample_m;
-    const uint4* smp = reinterpret_cast<const uint4*>(P.sample + ((size_t)w * L.fast_per_worker + seg.fast_index) * SAMPLE_MAX);
+    const uint4* smp = reinterpret_cast<const uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin);
     // ranks (from the top) that bracket the k-th largest of the segment
     const double q = (double)seg.k / (double)seg.n;
     const double centre = q * (double)m;
@@ -232,9 +230,10 @@ topk_main_kernel(FastParams P) {
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t off0 = warp * 512u + lane * 4u;                     // this thread's quad of row 0 inside a tile
-    // Each CTA appends to its own region of a segment's flagged and candidate lists (capacity / grid
-    // each), so a tile's slots follow from two running counters and no CTA waits for an atomic.
-    uint32_t run_flag = 0, run_cand = 0, fcap = 0, ccap = 0;
+    // A segment's flagged and candidate lists are cut into regions: one per CTA of this kernel when the
+    // segment has more tiles than CTAs (a tile's slots then follow from two running counters), else one
+    // per tile.  Either way no CTA waits for an atomic and the layout does not depend on scheduling.
+    uint32_t run_flag = 0, run_cand = 0, tot_cand = 0, fcap = 0, ccap = 0;
     for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) sh[b] = 0;
     __syncthreads();
     long long cur_prob = -1;
@@ -249,15 +248,14 @@ topk_main_kernel(FastParams P) {
             block_exclusive_scan(my_sure, s_red, &total);              // (only the total is used)
             if (threadIdx.x == 0) {
                 if (total) atomicAdd(&P.state[cur_prob].sure_total, total);
-                if (run_cand) atomicAdd(&P.state[cur_prob].cand_total, run_cand);
-                P.cand_cnt[cur_fidx * P.grid_main + blockIdx.x] = run_cand;
+                if (tot_cand) atomicAdd(&P.state[cur_prob].cand_total, tot_cand);
             }
             for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
                 const uint32_t c = sh[b];
                 if (c) { atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c); sh[b] = 0; }
             }
             __syncthreads();
-            my_sure = 0; run_flag = 0; run_cand = 0;
+            my_sure = 0; run_flag = 0; run_cand = 0; tot_cand = 0;
             cur_prob = -1;
         }
         if (!T.have) break;
@@ -336,8 +334,11 @@ topk_main_kernel(FastParams P) {
             tcand += c; tflag += f;
         }
         // this CTA's regions of the two lists, and where this tile's entries go inside them
+        const uint32_t tseg = T.lt - seg.tile_begin;                   // tile inside the segment
+        if (seg.region_per_tile) { run_flag = 0; run_cand = 0; }
+        const uint32_t region = seg.region_per_tile ? tseg : blockIdx.x;
         const bool fits = run_flag + tflag <= fcap && run_cand + tcand <= ccap;
-        const uint32_t fbase = blockIdx.x * fcap + run_flag, cbase = blockIdx.x * ccap + run_cand;
+        const uint32_t fbase = region * fcap + run_flag, cbase = region * ccap + run_cand;
         if (threadIdx.x == 0) {
             P.tile_fbase[item] = fits ? fbase : 0xFFFFFFFFu;
             P.tile_fcnt[item] = tflag;
@@ -345,7 +346,7 @@ topk_main_kernel(FastParams P) {
             P.tile_ccnt[item] = fits ? tcand : 0u;
             if (!fits) P.state[prob].overflow = 1u;                    // a region is full: the segment falls back
         }
-        if (fits) { run_flag += tflag; run_cand += tcand; }
+        if (fits) { run_flag += tflag; run_cand += tcand; tot_cand += tcand; }
         if (fits && flag16) {
             // the tile's entries fit: write them, zero the sure ones in the residual (their values
             // stay in the list, from where a fall-back restores them), histogram the candidates
@@ -416,28 +417,31 @@ topk_candbin_kernel(FastParams P) {
     }
 }
 
-// ---- filter: copy the candidates of the threshold's bin into the short list --------------------
+// ---- filter: copy the candidates of the threshold's bin into the short list (8 lanes per tile) -------
 __global__ void __launch_bounds__(THREADS)
 topk_candfilter_kernel(FastParams P) {
     const Layout& L = P.L;
-    uint32_t w, s;
-    const uint32_t prob = fast_problem(L, blockIdx.y, w, s);
+    const uint32_t sub = threadIdx.x & 7u;
+    const uint32_t item = (blockIdx.x * THREADS + threadIdx.x) >> 3;
+    if (item >= P.total_items) return;
+    const uint32_t cnt = P.tile_ccnt[item];
+    if (cnt == 0u) return;
+    const uint32_t w = item / L.tiles_per_worker;
+    const uint32_t lt = item - w * L.tiles_per_worker;
+    const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
     const SegEntry seg = L.segs[s];
+    if (!seg.fast) return;
+    const size_t prob = (size_t)w * L.nseg + s;
     const FastState* stp = P.state + prob;
     if (stp->path != PATH_FAST || stp->need2 == 0) return;
     const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
-    const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
-    const uint32_t ccap = seg.cand_cap;
-    uint2* out = P.list2 + fidx * LIST2_CAP;
-    for (uint32_t r = blockIdx.x; r < P.grid_main; r += gridDim.x) {        // one region (one main-pass CTA) at a time
-        const uint32_t total = P.cand_cnt[fidx * P.grid_main + r];
-        const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + (size_t)r * ccap;
-        for (uint32_t i = threadIdx.x; i < total; i += THREADS) {
-            const uint2 c = list[i];
-            if (c.x >= lo2 && c.x <= hi2) {
-                const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
-                if (pos < LIST2_CAP) out[pos] = c;
-            }
+    const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + P.tile_cbase[item];
+    uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
+    for (uint32_t i = sub; i < cnt; i += 8) {
+        const uint2 c = list[i];
+        if (c.x >= lo2 && c.x <= hi2) {
+            const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
+            if (pos < LIST2_CAP) out[pos] = c;
         }
     }
 }
