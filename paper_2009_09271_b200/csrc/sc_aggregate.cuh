@@ -136,6 +136,93 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
 }
 
 // ---------------------------------------------------------------------------------------------
+// Sparse messages with different coordinates per worker (top-k at the usual densities): one WARP
+// owns 1024 coordinates.  It reads, for eight workers at a time, the workers' slices of the
+// enclosing 4096-coordinate tile (a few dozen entries each, all loads of the batch in flight
+// together), keeps the entries that fall into its own quarter and adds them in worker order.
+// No shared staging area, no CTA-wide barrier: the warps of a CTA never wait for each other.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t AWARP = 1024;                 // coordinates per warp
+constexpr uint32_t AWARP_BATCH = 8;              // workers whose slices are fetched together
+constexpr uint32_t AWARP_MAX_SLICE = 64;         // entries of one worker in one 4096-tile served by the fast loop
+
+__global__ void __launch_bounds__(THREADS)
+agg_warp_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
+                const uint32_t* __restrict__ bounds /* at ATILE granularity */, uint32_t W, uint32_t K, uint32_t n,
+                uint32_t ntiles, float* __restrict__ out, int* __restrict__ status) {
+    __shared__ __align__(16) float acc_all[WARPS][AWARP];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    float* acc = acc_all[warp];
+    const float fW = (float)W;
+    const bool pow2 = (W & (W - 1u)) == 0u;
+    const float rW = 1.0f / fW;
+    const uint32_t nq = (n + AWARP - 1) / AWARP;                       // quarter-tiles
+    const uint32_t warps_total = gridDim.x * WARPS;
+    for (uint32_t q = blockIdx.x * WARPS + warp; q < nq; q += warps_total) {
+        const uint32_t t = q / (ATILE / AWARP);                          // enclosing tile of the bounds table
+        const uint32_t base = q * AWARP;
+        const uint32_t cnt_here = min(AWARP, n - base);
+#pragma unroll
+        for (int i = 0; i < (int)(AWARP / 128); ++i)
+            reinterpret_cast<float4*>(acc)[i * 32 + lane] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        __syncwarp();
+        for (uint32_t w0 = 0; w0 < W; w0 += AWARP_BATCH) {
+            uint32_t lo[AWARP_BATCH], hi[AWARP_BATCH];
+            uint32_t ix[AWARP_BATCH][2];
+            float vv[AWARP_BATCH][2];
+#pragma unroll
+            for (uint32_t u = 0; u < AWARP_BATCH; ++u) {
+                lo[u] = 0; hi[u] = 0;
+                if (w0 + u < W) {
+                    const uint32_t* b = bounds + (size_t)(w0 + u) * (ntiles + 1) + t;
+                    lo[u] = __ldg(b); hi[u] = __ldg(b + 1);
+                }
+            }
+#pragma unroll
+            for (uint32_t u = 0; u < AWARP_BATCH; ++u) {
+                const size_t row = (size_t)(w0 + u) * K;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t j = lo[u] + 32u * h + lane;
+                    ix[u][h] = 0xFFFFFFFFu; vv[u][h] = 0.0f;
+                    if (j < hi[u]) { ix[u][h] = __ldg(idx + row + j); vv[u][h] = __ldg(vals + row + j); }
+                }
+            }
+#pragma unroll
+            for (uint32_t u = 0; u < AWARP_BATCH; ++u) {                 // worker order
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t loc = ix[u][h] - base;
+                    if (loc < cnt_here) acc[loc] = acc[loc] + vv[u][h];
+                }
+                if (hi[u] - lo[u] > AWARP_MAX_SLICE) {                    // a long slice: finish it before the next worker
+                    const size_t row = (size_t)(w0 + u) * K;
+                    for (uint32_t j = lo[u] + AWARP_MAX_SLICE + lane; j < hi[u]; j += 32) {
+                        const uint32_t loc = __ldg(idx + row + j) - base;
+                        if (loc < cnt_here) acc[loc] = acc[loc] + __ldg(vals + row + j);
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        float* o = out + base;
+        if (cnt_here == AWARP) {
+#pragma unroll
+            for (int i = 0; i < (int)(AWARP / 128); ++i) {
+                float4 a = reinterpret_cast<const float4*>(acc)[i * 32 + lane];
+                if (pow2) { a.x *= rW; a.y *= rW; a.z *= rW; a.w *= rW; }
+                else { a.x = a.x / fW; a.y = a.y / fW; a.z = a.z / fW; a.w = a.w / fW; }
+                __stcs(reinterpret_cast<float4*>(o) + i * 32 + lane, a);
+            }
+        } else {
+            for (uint32_t i = lane; i < cnt_here; i += 32) o[i] = pow2 ? acc[i] * rW : acc[i] / fW;
+        }
+        __syncwarp();
+    }
+    (void)status;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Aggregate fused with the model update (Algorithm 1, update line: x <- x - q, q read as the
 // average): only coordinates that some worker sent are read and written, the dense q is never
 // materialised.  x - (+0.0) == x bit for bit, so skipping coordinates whose sum is zero gives

@@ -70,7 +70,7 @@ struct sc_ctx {
     uint32_t epoch = 0;
     uint64_t launches = 0;
 
-    int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1, occ_agg_big = 1;
+    int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1, occ_agg_big = 1, occ_agg_warp = 1;
 
     // optional per-kernel timing (sc_profile)
     bool prof_on = false;
@@ -430,7 +430,9 @@ inline uint32_t aggregate_tile(int W, size_t k, size_t n) {
 int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, bool shared_idx, size_t k, size_t n,
                    float* out, cudaStream_t stream) {
     if (n == 0) return SC_OK;
-    const uint32_t tile = aggregate_tile(shared_idx ? 1 : W, k, n);
+    // sparse messages with private coordinates: warp-owned quarter tiles (slices of ~k/n*4096 entries)
+    const bool by_warp = !shared_idx && (double)k * ATILE <= 0.6 * AWARP_MAX_SLICE * (double)n;
+    const uint32_t tile = by_warp ? ATILE : aggregate_tile(shared_idx ? 1 : W, k, n);
     const uint32_t ntiles = (uint32_t)((n + tile - 1) / tile);
     const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
     const uint64_t threads = (uint64_t)rows * (ntiles + 1ull);
@@ -438,13 +440,19 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
       agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
           idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds); }
     { Launch l(c, KIND_AGG_TILES, stream);
-      const uint32_t grid = persistent_grid(c, tile == ATILE_BIG ? c->occ_agg_big : c->occ_agg, ntiles);
-      if (tile == ATILE_BIG)
-          agg_tiles_kernel<ATILE_BIG><<<grid, THREADS, 0, stream>>>(
-              vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
-      else
-          agg_tiles_kernel<ATILE><<<grid, THREADS, 0, stream>>>(
-              vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status); }
+      if (by_warp) {
+          const uint64_t nq = (n + AWARP - 1) / AWARP;
+          agg_warp_kernel<<<persistent_grid(c, c->occ_agg_warp, (nq + WARPS - 1) / WARPS), THREADS, 0, stream>>>(
+              vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+      } else {
+          const uint32_t grid = persistent_grid(c, tile == ATILE_BIG ? c->occ_agg_big : c->occ_agg, ntiles);
+          if (tile == ATILE_BIG)
+              agg_tiles_kernel<ATILE_BIG><<<grid, THREADS, 0, stream>>>(
+                  vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+          else
+              agg_tiles_kernel<ATILE><<<grid, THREADS, 0, stream>>>(
+                  vals, idx, c->d_bounds, (uint32_t)W, shared_idx ? 1u : 0u, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+      } }
     SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
@@ -540,6 +548,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_block, randblock_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel<ATILE>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_big, agg_tiles_kernel<ATILE_BIG>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_warp, agg_warp_kernel, THREADS, 0);
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
         c->max_main_grid = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
     }
