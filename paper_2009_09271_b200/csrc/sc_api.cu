@@ -431,7 +431,8 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
                    float* out, cudaStream_t stream) {
     if (n == 0) return SC_OK;
     // sparse messages with private coordinates: warp-owned quarter tiles (slices of ~k/n*4096 entries)
-    const bool by_warp = !shared_idx && (double)k * ATILE <= 0.6 * AWARP_MAX_SLICE * (double)n;
+    const double slice = (double)k * ATILE / (double)std::max<size_t>(n, 1);       // entries of one worker per 4096-tile
+    const bool by_warp = !shared_idx && slice >= 8.0 && slice <= 0.75 * AWARP_MAX_SLICE;
     const uint32_t tile = by_warp ? ATILE : aggregate_tile(shared_idx ? 1 : W, k, n);
     const uint32_t ntiles = (uint32_t)((n + tile - 1) / tile);
     const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
