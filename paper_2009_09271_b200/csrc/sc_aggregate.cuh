@@ -223,6 +223,122 @@ agg_warp_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same ownership for denser messages (slices of about 50 to 800 entries per worker and
+// 4096-tile).  Reading the whole tile slice in each of its four warps would quadruple the
+// traffic from L2, so each warp first narrows the tile's slice to its own 1024 coordinates: lane
+// u of the lower half searches the first entry >= base for worker u of the batch, lane u of the
+// upper half the first entry >= base + 1024 (binary search inside the tile slice, all workers of
+// the batch at once).  Then H rounds of 32 entries per worker are fetched for B workers together
+// and added in worker order; what exceeds 32 H entries is finished before the next worker.
+// ---------------------------------------------------------------------------------------------
+template <int H, int B>
+__global__ void __launch_bounds__(THREADS)
+agg_warp_fine_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
+                     const uint32_t* __restrict__ bounds /* at ATILE granularity */, uint32_t W, uint32_t K, uint32_t n,
+                     uint32_t ntiles, float* __restrict__ out, int* __restrict__ status) {
+    static_assert(B <= 16, "a batch lies inside one group of 16 workers");
+    __shared__ __align__(16) float acc_all[WARPS][AWARP];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    float* acc = acc_all[warp];
+    const float fW = (float)W;
+    const bool pow2 = (W & (W - 1u)) == 0u;
+    const float rW = 1.0f / fW;
+    const uint32_t nq = (n + AWARP - 1) / AWARP;
+    const uint32_t warps_total = gridDim.x * WARPS;
+    for (uint32_t q = blockIdx.x * WARPS + warp; q < nq; q += warps_total) {
+        const uint32_t t = q / (ATILE / AWARP);
+        const uint32_t base = q * AWARP;
+        const uint32_t cnt_here = min(AWARP, n - base);
+#pragma unroll
+        for (int i = 0; i < (int)(AWARP / 128); ++i)
+            reinterpret_cast<float4*>(acc)[i * 32 + lane] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        __syncwarp();
+        for (uint32_t g0 = 0; g0 < W; g0 += 16) {
+        // boundaries of this quarter inside the tile slices of workers g0 .. g0+15: lane u the first
+        // entry, lane 16+u the end; an 8-way search (7 probes in flight per step) keeps the chain of
+        // dependent loads to three or four for slices of several hundred entries
+        uint32_t found = 0;
+        {
+            const uint32_t u = lane & 15u, upper = lane >> 4;
+            if (g0 + u < W) {
+                const uint32_t* b = bounds + (size_t)(g0 + u) * (ntiles + 1) + t;
+                uint32_t a = __ldg(b), e = __ldg(b + 1);
+                const uint32_t target = base + (upper ? AWARP : 0u);
+                const uint32_t* row = idx + (size_t)(g0 + u) * K;
+                const uint32_t qi = q % (ATILE / AWARP);
+                if (!upper && qi == 0) e = a;                             // the tile's own first coordinate
+                else if (upper && qi == ATILE / AWARP - 1) a = e;         // the tile's end
+                while (a < e) {
+                    const uint32_t len = e - a;
+                    uint32_t c = 0;
+#pragma unroll
+                    for (uint32_t i = 1; i < 8; ++i) c += (__ldg(row + a + ((len * i) >> 3)) < target) ? 1u : 0u;
+                    const uint32_t na = c ? a + ((len * c) >> 3) + 1u : a;
+                    const uint32_t ne = c < 7 ? a + ((len * (c + 1u)) >> 3) : e;
+                    a = na; e = ne;
+                }
+                found = a;
+            }
+        }
+        const uint32_t gend = min(W, g0 + 16u);
+        for (uint32_t w0 = g0; w0 < gend; w0 += B) {
+            uint32_t lo[B], hi[B];
+#pragma unroll
+            for (int u = 0; u < B; ++u) {
+                const uint32_t gu = w0 - g0 + u;                               // position in the group of 16
+                const uint32_t l = __shfl_sync(0xFFFFFFFFu, found, gu & 15u);
+                const uint32_t h = __shfl_sync(0xFFFFFFFFu, found, 16u + (gu & 15u));
+                lo[u] = gu < 16u ? l : 0u;
+                hi[u] = gu < 16u ? h : 0u;
+            }
+            uint32_t ix[B][H];
+            float vv[B][H];
+#pragma unroll
+            for (int u = 0; u < B; ++u) {
+                const size_t row = (size_t)(w0 + u) * K;
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    const uint32_t j = lo[u] + 32u * h + lane;
+                    ix[u][h] = 0xFFFFFFFFu; vv[u][h] = 0.0f;
+                    if (j < hi[u]) { ix[u][h] = __ldg(idx + row + j); vv[u][h] = __ldg(vals + row + j); }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < B; ++u) {                                    // worker order
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    const uint32_t loc = ix[u][h] - base;
+                    if (loc < cnt_here) acc[loc] = acc[loc] + vv[u][h];
+                }
+                if (hi[u] - lo[u] > 32u * H) {                               // a long slice: finish it before the next worker
+                    const size_t row = (size_t)(w0 + u) * K;
+                    for (uint32_t j = lo[u] + 32u * H + lane; j < hi[u]; j += 32) {
+                        const uint32_t loc = __ldg(idx + row + j) - base;
+                        if (loc < cnt_here) acc[loc] = acc[loc] + __ldg(vals + row + j);
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        }
+        float* o = out + base;
+        if (cnt_here == AWARP) {
+#pragma unroll
+            for (int i = 0; i < (int)(AWARP / 128); ++i) {
+                float4 a = reinterpret_cast<const float4*>(acc)[i * 32 + lane];
+                if (pow2) { a.x *= rW; a.y *= rW; a.z *= rW; a.w *= rW; }
+                else { a.x = a.x / fW; a.y = a.y / fW; a.z = a.z / fW; a.w = a.w / fW; }
+                __stcs(reinterpret_cast<float4*>(o) + i * 32 + lane, a);
+            }
+        } else {
+            for (uint32_t i = lane; i < cnt_here; i += 32) o[i] = pow2 ? acc[i] * rW : acc[i] / fW;
+        }
+        __syncwarp();
+    }
+    (void)status;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Aggregate fused with the model update (Algorithm 1, update line: x <- x - q, q read as the
 // average): only coordinates that some worker sent are read and written, the dense q is never
 // materialised.  x - (+0.0) == x bit for bit, so skipping coordinates whose sum is zero gives

@@ -71,6 +71,7 @@ struct sc_ctx {
     uint64_t launches = 0;
 
     int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1, occ_agg_big = 1, occ_agg_warp = 1;
+    int occ_agg_fine[3] = {1, 1, 1};
 
     // optional per-kernel timing (sc_profile)
     bool prof_on = false;
@@ -303,7 +304,6 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             fp.tile_ccnt = c->d_tile_ccnt; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
             fp.flagged = c->d_flagged; fp.offsets = c->d_offsets;
             fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
-            SC_CUDA(cudaMemsetAsync(c->d_tile_sure, 0, (size_t)items * sizeof(uint32_t), stream));
             SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
             { Launch l(c, KIND_SAMPLE, stream);
               topk_sample_kernel<<<dim3((c->max_sample_m / 8 + THREADS - 1) / THREADS, PF), THREADS, 0, stream>>>(fp); }
@@ -422,6 +422,18 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
 
 // Tile of the dense output: the larger one halves the per-tile overhead, but only pays while all
 // slices of a tile fit the shared-memory staging area in one round.
+// Largest expected slice of one worker per 1024 coordinates served with 2, 4 and 6 rounds of 32 entries held
+// in registers (a longer slice is still correct: its remainder is read in a loop of its own).
+#ifndef AGG_FINE_Q0
+#define AGG_FINE_Q0 43.0
+#endif
+#ifndef AGG_FINE_Q1
+#define AGG_FINE_Q1 120.0
+#endif
+#ifndef AGG_FINE_Q2
+#define AGG_FINE_Q2 200.0
+#endif
+
 inline uint32_t aggregate_tile(int W, size_t k, size_t n) {
     const double per_big_tile = (double)ATILE_BIG * (double)W * (double)k / (double)std::max<size_t>(n, 1);
     return per_big_tile <= 0.9 * AGG_STAGE ? ATILE_BIG : ATILE;
@@ -433,7 +445,12 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
     // sparse messages with private coordinates: warp-owned quarter tiles (slices of ~k/n*4096 entries)
     const double slice = (double)k * ATILE / (double)std::max<size_t>(n, 1);       // entries of one worker per 4096-tile
     const bool by_warp = !shared_idx && slice >= 8.0 && slice <= 0.75 * AWARP_MAX_SLICE;
-    const uint32_t tile = by_warp ? ATILE : aggregate_tile(shared_idx ? 1 : W, k, n);
+    // denser private coordinates: the same ownership with per-quarter boundaries; H rounds of 32 entries per
+    // worker cover the expected quarter slice with a 30 % margin
+    const double qslice = slice / (ATILE / AWARP);
+    const int fine = (shared_idx || by_warp || slice < 8.0) ? -1
+                     : qslice <= AGG_FINE_Q0 ? 0 : qslice <= AGG_FINE_Q1 ? 1 : qslice <= AGG_FINE_Q2 ? 2 : -1;
+    const uint32_t tile = (by_warp || fine >= 0) ? ATILE : aggregate_tile(shared_idx ? 1 : W, k, n);
     const uint32_t ntiles = (uint32_t)((n + tile - 1) / tile);
     const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
     const uint64_t threads = (uint64_t)rows * (ntiles + 1ull);
@@ -441,10 +458,21 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
       agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
           idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds); }
     { Launch l(c, KIND_AGG_TILES, stream);
+      const uint64_t nq = (n + AWARP - 1) / AWARP;
       if (by_warp) {
-          const uint64_t nq = (n + AWARP - 1) / AWARP;
           agg_warp_kernel<<<persistent_grid(c, c->occ_agg_warp, (nq + WARPS - 1) / WARPS), THREADS, 0, stream>>>(
               vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+      } else if (fine >= 0) {
+          const uint32_t grid = persistent_grid(c, c->occ_agg_fine[fine], (nq + WARPS - 1) / WARPS);
+          if (fine == 0)
+              agg_warp_fine_kernel<2, 8><<<grid, THREADS, 0, stream>>>(
+                  vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+          else if (fine == 1)
+              agg_warp_fine_kernel<4, 4><<<grid, THREADS, 0, stream>>>(
+                  vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+          else
+              agg_warp_fine_kernel<6, 3><<<grid, THREADS, 0, stream>>>(
+                  vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
       } else {
           const uint32_t grid = persistent_grid(c, tile == ATILE_BIG ? c->occ_agg_big : c->occ_agg, ntiles);
           if (tile == ATILE_BIG)
@@ -550,6 +578,9 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel<ATILE>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_big, agg_tiles_kernel<ATILE_BIG>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_warp, agg_warp_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_fine[0], agg_warp_fine_kernel<2, 8>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_fine[1], agg_warp_fine_kernel<4, 4>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_fine[2], agg_warp_fine_kernel<6, 3>, THREADS, 0);
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
         c->max_main_grid = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
     }

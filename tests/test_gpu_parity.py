@@ -232,6 +232,40 @@ def test_aggregate_generic_shared_and_collisions(ctx):
     assert_bits_equal(out, want, "single coordinate")
 
 
+@pytest.mark.parametrize("W,n,density,clumped", [
+    (16, 300_000, 0.02, False), (5, 300_001, 0.05, False), (16, 262_144, 0.10, False),
+    (3, 200_003, 0.18, False), (8, 150_000, 0.30, False), (6, 250_000, 0.04, True), (16, 99_999, 0.10, True)])
+def test_aggregate_private_coordinates_by_density(ctx, W, n, density, clumped):
+    """Private coordinate sets from 2 % to 30 % kept (each range of slice lengths has its own kernel);
+    'clumped' puts most of every message into a few stretches of 1024 coordinates."""
+    if W > 8:
+        own = sc.Context(max_n=n, max_W=W, max_segments=1)
+    else:
+        own = ctx
+    rng = np.random.default_rng(int(n + 1000 * density) + W)
+    k = int(n * density)
+    rows = []
+    for w in range(W):
+        if clumped:
+            hot = rng.choice(n // 1024, 3, replace=False) * 1024
+            pool = np.concatenate([np.arange(h, min(h + 1024, n)) for h in hot])
+            take_hot = min(k * 3 // 4, pool.size - 7)
+            a = rng.choice(pool, take_hot, replace=False)
+            rest = np.setdiff1d(np.arange(n), a, assume_unique=False)
+            b = rng.choice(rest, k - take_hot, replace=False)
+            rows.append(np.sort(np.concatenate([a, b])))
+        else:
+            rows.append(np.sort(rng.choice(n, k, replace=False)))
+    idx = np.stack(rows).astype(np.uint32)
+    vals = (rng.standard_normal((W, k)) * 10.0 ** rng.uniform(-3, 3, (W, k))).astype(np.float32)
+    out = torch.full((n,), float("nan"), device="cuda")
+    own.sc_aggregate(W, torch.from_numpy(vals).cuda(), torch.from_numpy(idx.view(np.int32)).cuda(), k, n, out)
+    assert own.sc_sync_status() == 0
+    assert_bits_equal(out, O.aggregate(list(vals), list(idx), n), "aggregate by density")
+    if own is not ctx:
+        own.close()
+
+
 def test_host_buffer_step(ctx):
     W, n = 4, 3 * TILE + 9
     g = torch.stack([rand(n, 500 + w) for w in range(W)])
