@@ -58,7 +58,7 @@ struct sc_ctx {
     uint32_t slow_segments = 0;      // segments of the cached table that take the radix-select path
     uint32_t max_sample_m = 0;
     uint32_t max_flag_cap = 0, max_cand_cap = 0;
-    int occ_main = 1, occ_emit = 1;
+    int occ_main = 1, occ_emit = 1, occ_emit_v[4] = {1, 1, 1, 1};
     uint64_t* d_seeds = nullptr;
     int* d_status = nullptr;
 
@@ -89,6 +89,10 @@ struct sc_ctx {
     cudaEvent_t ev_start = nullptr;
     std::vector<cudaEvent_t> ev_worker;
 };
+
+// Emit variants by the average number of flagged entries per tile: 8 or 16 lanes per tile for sparse slices
+// (4 or 2 tiles per warp side by side), the whole warp with 4 or 8 entries per lane for longer ones.
+constexpr double EMIT_MAX_8 = 12.0, EMIT_MAX_16 = 80.0, EMIT_MAX_32 = 200.0;
 
 namespace {
 
@@ -175,7 +179,11 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         const uint64_t seg_tiles = (g.n + 31 + TILE - 1) / TILE;   // a tile grid shifted by up to 31 elements
         if (g.n >= FAST_MIN_N) {
             uint64_t m = (g.n / 16) & ~7ull;
-            m = std::min<uint64_t>(std::max<uint64_t>(m, SAMPLE_MIN), SAMPLE_MAX);
+            // a larger sample narrows the bracket (candidates ~ sqrt(q / m) n) but costs time itself: the cap that
+            // balanced the two on 350 M elements is 2^18 below 0.3 % kept, 2^19 up to 3 %, 2^20 beyond
+            const double q = (double)g.k / (double)g.n;
+            const uint64_t cap = q >= 0.03 ? SAMPLE_MAX : q >= 0.003 ? SAMPLE_MAX / 2 : SAMPLE_MAX / 4;
+            m = std::min<uint64_t>(std::max<uint64_t>(m, SAMPLE_MIN), cap);
             e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
             e.sample_begin = smp; smp += m;
             fast_list.push_back((uint32_t)s);
@@ -308,7 +316,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             { Launch l(c, KIND_SAMPLE, stream);
               topk_sample_kernel<<<dim3((c->max_sample_m / 8 + THREADS - 1) / THREADS, PF), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_BRACKET, stream);
-              topk_bracket_kernel<<<PF, THREADS, 0, stream>>>(fp); }
+              topk_bracket_kernel<<<PF * BRACKET_CTAS, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_MAIN, stream);
               topk_main_kernel<<<persistent_grid(c, c->occ_main, items), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDBIN, stream);
@@ -325,8 +333,16 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             { Launch l(c, KIND_ROW_SCAN, stream);
               row_scan_kernel<<<W, THREADS, 0, stream>>>(c->d_offsets, L.tiles_per_worker); }
             { Launch l(c, KIND_EMIT, stream);
-              const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
-              topk_emit_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
+              // flagged entries per tile, on average (the list holds the kept elements and a few per cent more)
+              const double per_tile = 1.05 * (double)L.K_total * TILE / (double)std::max<size_t>(L.n_total, 1);
+              const int v = per_tile <= EMIT_MAX_8 ? 0 : per_tile <= EMIT_MAX_16 ? 1 : per_tile <= EMIT_MAX_32 ? 2 : 3;
+              const uint32_t tiles_per_warp = v == 0 ? 4u : v == 1 ? 2u : 1u;
+              const uint64_t warps = (items + tiles_per_warp - 1) / tiles_per_warp;
+              const uint32_t blocks = persistent_grid(c, c->occ_emit_v[v], (warps + WARPS - 1) / WARPS);
+              if (v == 0) topk_emit_kernel<8, 4><<<blocks, THREADS, 0, stream>>>(fp);
+              else if (v == 1) topk_emit_kernel<16, 4><<<blocks, THREADS, 0, stream>>>(fp);
+              else if (v == 2) topk_emit_kernel<32, 4><<<blocks, THREADS, 0, stream>>>(fp);
+              else topk_emit_kernel<32, 8><<<blocks, THREADS, 0, stream>>>(fp); }
         }
         // Radix select: once over the small segments (if any), once over the large ones, where the
         // launch returns at once unless some segment's bracket missed.
@@ -570,7 +586,11 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     if (rc == SC_OK) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main, topk_main_kernel, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit, topk_emit_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit, topk_restore_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[0], topk_emit_kernel<8, 4>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[1], topk_emit_kernel<16, 4>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[2], topk_emit_kernel<32, 4>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[3], topk_emit_kernel<32, 8>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_refine, topk_refine_kernel<1>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_topk, pack_kernel<PACK_TOPK>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_mask, randk_pack_kernel, THREADS, 0);

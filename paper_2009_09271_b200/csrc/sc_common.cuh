@@ -96,7 +96,7 @@ struct FastState {
 };
 
 constexpr uint32_t FAST_MIN_N = 1u << 16;
-constexpr uint32_t SAMPLE_MIN = 1u << 12, SAMPLE_MAX = 1u << 18;
+constexpr uint32_t SAMPLE_MIN = 1u << 12, SAMPLE_MAX = 1u << 20;
 constexpr uint32_t CAND_BINS = 2048;
 constexpr uint32_t LIST2_CAP = 4096;
 

@@ -23,6 +23,8 @@
 //            back from the flagged list.
 // No CTA waits on another anywhere on this path.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "sc_common.cuh"
 
 namespace sc {
@@ -118,18 +120,31 @@ topk_sample_kernel(FastParams P) {
     out[0] = k0; out[1] = k1;
 }
 
-// ---- bracket: two order statistics of the sample, to 21 bits (one CTA per problem) ------
-__global__ void __launch_bounds__(THREADS)
+// ---- bracket: two order statistics of the sample, to 21 bits -----------------------------------
+// One thread-block cluster of BRACKET_CTAS CTAs per problem: every CTA histograms its share of the
+// sample in its own shared memory, CTA 0 adds the shares up through distributed shared memory, walks
+// the total and hands the two bins back the same way; a second round refines them by ten more bits.
+// The cluster barriers are the hardware's; no CTA leaves before the last one (a peer's shared memory
+// must stay alive while it is read).
+constexpr uint32_t BRACKET_CTAS = 8;
+__global__ void __cluster_dims__(BRACKET_CTAS, 1, 1) __launch_bounds__(THREADS)
 topk_bracket_kernel(FastParams P) {
+    namespace cg = cooperative_groups;
     __shared__ uint32_t h0[HIST0_BINS];
     __shared__ uint32_t hA[1024], hB[1024];
     __shared__ uint32_t s_tmp[WARPS + 4];
+    __shared__ uint32_t s_bins[4];                                     // binA, binB, needA, needB (valid in CTA 0)
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t rank = cluster.block_rank();
     const Layout& L = P.L;
     uint32_t w, s;
-    const uint32_t prob = fast_problem(L, blockIdx.x, w, s);
+    const uint32_t prob = fast_problem(L, blockIdx.x / BRACKET_CTAS, w, s);
     const SegEntry seg = L.segs[s];
     const uint32_t m = seg.sample_m;
     const uint4* smp = reinterpret_cast<const uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin);
+    // this CTA's share of the sample (in groups of four keys)
+    const uint32_t per = (m / 4u + BRACKET_CTAS - 1u) / BRACKET_CTAS;
+    const uint32_t i_begin = min(rank * per, m / 4u), i_end = min(i_begin + per, m / 4u);
     // ranks (from the top) that bracket the k-th largest of the segment
     const double q = (double)seg.k / (double)seg.n;
     const double centre = q * (double)m;
@@ -141,20 +156,32 @@ topk_bracket_kernel(FastParams P) {
     for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) h0[b] = 0;
     for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) { hA[b] = 0; hB[b] = 0; }
     __syncthreads();
-    for (uint32_t i = threadIdx.x; i < m / 4u; i += THREADS) {
+    for (uint32_t i = i_begin + threadIdx.x; i < i_end; i += THREADS) {
         const uint4 k = smp[i];
         atomicAdd(&h0[k.x >> 20], 1u); atomicAdd(&h0[k.y >> 20], 1u);
         atomicAdd(&h0[k.z >> 20], 1u); atomicAdd(&h0[k.w >> 20], 1u);
     }
-    __syncthreads();
+    cluster.sync();
     // when k is so small that no sample rank lies safely above the threshold there is no "sure"
     // set (hi stays at the largest key); the candidate histogram then spans up to the largest
     // sample key and everything above it shares the last bin
-    const uint32_t rankA = have_hi ? (uint32_t)j_hi : 1u;
-    uint32_t binA = 0, needA = 0, binB = 0, needB = 0, cnt = 0;
-    find_from_top<HIST0_BINS>(h0, rankA, s_tmp, binA, needA, cnt);
-    if (have_lo) find_from_top<HIST0_BINS>(h0, (uint32_t)j_lo, s_tmp, binB, needB, cnt);
-    for (uint32_t i = threadIdx.x; i < m / 4u; i += THREADS) {
+    if (rank == 0) {
+        for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) {
+            uint32_t v = h0[b];
+            for (uint32_t r = 1; r < BRACKET_CTAS; ++r) v += cluster.map_shared_rank(h0, r)[b];
+            h0[b] = v;
+        }
+        __syncthreads();
+        const uint32_t rankA = have_hi ? (uint32_t)j_hi : 1u;
+        uint32_t binA = 0, needA = 0, binB = 0, needB = 0, cnt = 0;
+        find_from_top<HIST0_BINS>(h0, rankA, s_tmp, binA, needA, cnt);
+        if (have_lo) find_from_top<HIST0_BINS>(h0, (uint32_t)j_lo, s_tmp, binB, needB, cnt);
+        if (threadIdx.x == 0) { s_bins[0] = binA; s_bins[1] = binB; s_bins[2] = needA; s_bins[3] = needB; }
+    }
+    cluster.sync();
+    const uint32_t* bins0 = cluster.map_shared_rank(s_bins, 0);
+    const uint32_t binA = bins0[0], binB = bins0[1];
+    for (uint32_t i = i_begin + threadIdx.x; i < i_end; i += THREADS) {
         const uint4 k = smp[i];
         const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
 #pragma unroll
@@ -163,19 +190,32 @@ topk_bracket_kernel(FastParams P) {
             if (have_lo && (kk[c] >> 20) == binB) atomicAdd(&hB[(kk[c] >> 10) & 1023u], 1u);
         }
     }
-    __syncthreads();
-    uint32_t top = 0x7FFFFFFFu, lo = 0u, bin1 = 0, need1 = 0;
-    if (find_from_top<1024>(hA, needA, s_tmp, bin1, need1, cnt)) top = (binA << 20) | (bin1 << 10) | 1023u;
-    if (have_lo && find_from_top<1024>(hB, needB, s_tmp, bin1, need1, cnt)) lo = (binB << 20) | (bin1 << 10);
-    const uint32_t hi = have_hi ? top : 0x7FFFFFFFu;
-    if (lo > top) lo = top;                                            // (cannot happen; keeps the bracket sane)
-    if (threadIdx.x == 0) {
-        const uint32_t width_m1 = top - lo;
-        const uint32_t bits = width_m1 ? 32u - (uint32_t)__clz((int)width_m1) : 0u;
-        FastState st = {};
-        st.path = PATH_FAST; st.lo = lo; st.hi = hi; st.shift = bits > 11u ? bits - 11u : 0u;
-        P.state[prob] = st;
+    cluster.sync();
+    if (rank == 0) {
+        for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) {
+            uint32_t va = hA[b], vb = hB[b];
+            for (uint32_t r = 1; r < BRACKET_CTAS; ++r) {
+                va += cluster.map_shared_rank(hA, r)[b];
+                vb += cluster.map_shared_rank(hB, r)[b];
+            }
+            hA[b] = va; hB[b] = vb;
+        }
+        __syncthreads();
+        const uint32_t needA = s_bins[2], needB = s_bins[3];
+        uint32_t top = 0x7FFFFFFFu, lo = 0u, bin1 = 0, need1 = 0, cnt = 0;
+        if (find_from_top<1024>(hA, needA, s_tmp, bin1, need1, cnt)) top = (binA << 20) | (bin1 << 10) | 1023u;
+        if (have_lo && find_from_top<1024>(hB, needB, s_tmp, bin1, need1, cnt)) lo = (binB << 20) | (bin1 << 10);
+        const uint32_t hi = have_hi ? top : 0x7FFFFFFFu;
+        if (lo > top) lo = top;                                        // (cannot happen; keeps the bracket sane)
+        if (threadIdx.x == 0) {
+            const uint32_t width_m1 = top - lo;
+            const uint32_t bits = width_m1 ? 32u - (uint32_t)__clz((int)width_m1) : 0u;
+            FastState st = {};
+            st.path = PATH_FAST; st.lo = lo; st.hi = hi; st.shift = bits > 11u ? bits - 11u : 0u;
+            P.state[prob] = st;
+        }
     }
+    cluster.sync();                                                    // peers stay until CTA 0 has read their histograms
 }
 
 // ---- main streaming pass ---------------------------------------------------------------
@@ -577,15 +617,25 @@ topk_tilecount_kernel(FastParams P) {
     if (live && sub == 0) P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
 }
 
-constexpr int EMIT_DEPTH = 4;
-// ---- emit: one warp per tile walks the tile's slice of the flagged list -------------------------
+// ---- emit: G lanes per tile walk the tile's slice of the flagged list ----------------------------
+// Sparse slices (a few dozen entries) take a part of a warp per tile, i.e. several tiles per warp
+// side by side; long slices take the whole warp and more entries per lane.  One batch covers
+// G x D entries.  (Loading the placement words two tiles ahead and asking L2 for the next slice
+// one tile ahead changed nothing: the kernel is not bound by its chain of dependent loads.)
+template <int G, int D>
 __global__ void __launch_bounds__(THREADS)
 topk_emit_kernel(FastParams P) {
+    static_assert(G == 8 || G == 16 || G == 32, "lanes per tile");
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    const uint32_t warps_total = gridDim.x * WARPS;
-    // per-(worker, segment) constants stay in registers while the warp's tiles belong to the same one
+    constexpr uint32_t TPW = 32 / G;                                    // tiles per warp
+    const uint32_t grp = lane / G, gl = lane % G;
+    const uint32_t gshift = grp * G;
+    const uint32_t gmask = (G == 32) ? 0xFFFFFFFFu : ((1u << G) - 1u);
+    const uint32_t lt_mask = (1u << gl) - 1u;
+    const uint32_t stride = gridDim.x * WARPS * TPW;
+    const uint32_t rounds = (P.total_items + stride - 1) / stride;      // the same for every lane: ballots stay whole
+    // per-(worker, segment) constants stay in registers while the group's tiles belong to the same one
     uint32_t cw = 0xFFFFFFFFu, cs = 0xFFFFFFFFu, c_tile_end = 0;        // cached worker, segment, end of its tile range
     uint32_t T = 0, icut = 0, hi = 0, seg_k = 0, idx0 = 0, tile_begin = 0, off_begin = 0;
     bool live = false;
@@ -593,50 +643,55 @@ topk_emit_kernel(FastParams P) {
     float* e = nullptr;
     float* ovals = nullptr;
     uint32_t* oidx = nullptr;
-    const uint32_t* off = nullptr;
-    for (uint32_t item = blockIdx.x * WARPS + (threadIdx.x >> 5); item < P.total_items; item += warps_total) {
-        const uint32_t w = item / L.tiles_per_worker;
-        const uint32_t lt = item - w * L.tiles_per_worker;
-        if (w != cw || lt < tile_begin || lt >= c_tile_end) {           // another (worker, segment): reload
-            cw = w;
-            cs = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-            const SegEntry seg = L.segs[cs];
-            tile_begin = seg.tile_begin; c_tile_end = L.segs[cs + 1].tile_begin;
-            const FastState* st = P.state + (size_t)w * L.nseg + cs;
-            live = seg.fast && st->path == PATH_FAST;
-            T = st->T; icut = st->icut; hi = st->hi; seg_k = seg.k; idx0 = (uint32_t)seg.offset;
-            off = P.offsets + (size_t)w * (L.tiles_per_worker + 1);
-            off_begin = off[tile_begin];
-            flist0 = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
-            e = P.residuals + (size_t)w * L.n_total + seg.offset;
-            ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
-            oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
+    uint32_t item = (blockIdx.x * WARPS + (threadIdx.x >> 5)) * TPW + grp;
+    for (uint32_t round = 0; round < rounds; ++round, item += stride) {
+        uint32_t cnt = 0, base = 0, running = 0;
+        if (item < P.total_items) {
+            const uint32_t w = item / L.tiles_per_worker;
+            const uint32_t lt = item - w * L.tiles_per_worker;
+            if (w != cw || lt < tile_begin || lt >= c_tile_end) {       // another (worker, segment): reload
+                cw = w;
+                cs = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+                const SegEntry seg = L.segs[cs];
+                tile_begin = seg.tile_begin; c_tile_end = L.segs[cs + 1].tile_begin;
+                const FastState* st = P.state + (size_t)w * L.nseg + cs;
+                live = seg.fast && st->path == PATH_FAST;
+                T = st->T; icut = st->icut; hi = st->hi; seg_k = seg.k; idx0 = (uint32_t)seg.offset;
+                off_begin = P.offsets[(size_t)w * (L.tiles_per_worker + 1) + tile_begin];
+                flist0 = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
+                e = P.residuals + (size_t)w * L.n_total + seg.offset;
+                ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
+                oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
+            }
+            if (live) {
+                // the four words that place this tile: independent loads, one round trip
+                const uint32_t* o = P.offsets + (size_t)w * (L.tiles_per_worker + 1) + lt;
+                cnt = __ldg(P.tile_fcnt + item); base = __ldg(P.tile_fbase + item);
+                const uint32_t o0 = __ldg(o), o1 = __ldg(o + 1);
+                running = o0 - off_begin;                               // kept coordinates of the segment before this tile
+                if (cnt && (unsigned long long)running + (o1 - o0) > seg_k) {   // counts and k disagree: write nothing
+                    if (gl == 0) atomicMin(P.status, ST_DEVICE_CHECK);
+                    cnt = 0;
+                }
+            }
         }
-        if (!live) continue;
-        // the four words that place this tile: independent loads, one round trip
-        const uint32_t cnt = P.tile_fcnt[item], base = P.tile_fbase[item];
-        const uint32_t o0 = off[lt], o1 = off[lt + 1];
-        if (cnt == 0u) continue;
-        const uint32_t running = o0 - off_begin;                        // kept coordinates of the segment before this tile
-        if ((unsigned long long)running + (o1 - o0) > seg_k) {          // counts and k disagree: write nothing
-            if (lane == 0) atomicMin(P.status, ST_DEVICE_CHECK);
-            continue;
-        }
-        // entry i of the slice belongs to lane i % 32; message pointers advance with the running rank
+        const uint32_t maxcnt = __reduce_max_sync(0xFFFFFFFFu, cnt);
+        // entry i of the slice belongs to lane i % G of the group; message pointers advance with the running rank
         float* ov = ovals + running;
         uint32_t* oi = oidx + running;
-        const uint2* fl = flist0 + base + lane;
-        for (uint32_t b = 0; b < cnt; b += 32 * EMIT_DEPTH) {           // EMIT_DEPTH independent loads in flight per lane
-            uint2 a[EMIT_DEPTH];
+        const uint2* fl = flist0 + base + gl;
+        for (uint32_t b = 0; b < maxcnt; b += G * D) {                  // D independent loads in flight per lane
+            uint2 a[D];
 #pragma unroll
-            for (int u = 0; u < EMIT_DEPTH; ++u) a[u] = (b + 32u * u + lane < cnt) ? __ldg(fl + b + 32u * u) : make_uint2(0u, 0xFFFFFFFFu);
+            for (int u = 0; u < D; ++u) a[u] = (b + G * u + gl < cnt) ? __ldg(fl + b + G * u) : make_uint2(0u, 0xFFFFFFFFu);
 #pragma unroll
-            for (int u = 0; u < EMIT_DEPTH; ++u) {
+            for (int u = 0; u < D; ++u) {
                 // a padding entry has key 0 and coordinate 2^32-1: kept only if T == 0 and icut == 2^32-1, which
-                // cannot happen (coordinates are < n < 2^32, so icut <= n)
+                // cannot happen (coordinates are < n < 2^32, so icut <= n); a group without a tile has cnt == 0 and
+                // T, icut from its last tile or 0, so its padding entries are never kept either
                 const uint32_t key = a[u].x & 0x7FFFFFFFu;
-                const bool sel = key > T || (key == T && a[u].y < icut);
-                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, sel);
+                const bool sel = (b + G * u + gl < cnt) && (key > T || (key == T && a[u].y < icut));
+                const uint32_t bal = (__ballot_sync(0xFFFFFFFFu, sel) >> gshift) & gmask;
                 if (sel) {
                     const uint32_t r = __popc(bal & lt_mask);
                     ov[r] = __uint_as_float(a[u].x);
