@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/sparsecomm.h: argument checks, scratch
 // ownership, the device-side segment table and the launch sequences.
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -56,7 +57,7 @@ struct sc_ctx {
     size_t max_fast_per_worker = 0, max_cand_per_worker = 0;
     uint32_t last_topk_problems = 0; // (worker, segment) pairs of the most recent top-k call
     uint32_t slow_segments = 0;      // segments of the cached table that take the radix-select path
-    uint32_t max_sample_m = 0;
+    uint32_t max_sample_m = 0, fast_big = 0;
     uint32_t max_flag_cap = 0, max_cand_cap = 0;
     int occ_main = 1, occ_emit = 1, occ_emit_v[4] = {1, 1, 1, 1};
     uint64_t* d_seeds = nullptr;
@@ -178,12 +179,16 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         e.mask_word_begin = maskw; e.grp_begin = (uint32_t)groups;
         const uint64_t seg_tiles = (g.n + 31 + TILE - 1) / TILE;   // a tile grid shifted by up to 31 elements
         if (g.n >= FAST_MIN_N) {
-            uint64_t m = (g.n / 16) & ~7ull;
-            // a larger sample narrows the bracket (candidates ~ sqrt(q / m) n) but costs time itself: the cap that
-            // balanced the two on 350 M elements is 2^18 below 0.3 % kept, 2^19 up to 3 %, 2^20 beyond
+            // Sample size.  A larger sample narrows the bracket (candidates ~ 12 sqrt(q (1 - q) / m) n) but costs
+            // time itself (one scattered 32-byte read per 8 keys): the two balance at m ~ (n sqrt(q))^(2/3), scaled
+            // so that 350 M elements at 10 % kept get 2^20 keys (measured optimum there: 2^18 at 0.1 %, 2^19 at
+            // 1 %, 2^20 at 10 %).  The second term keeps the candidates within a fraction of the list capacity.
             const double q = (double)g.k / (double)g.n;
-            const uint64_t cap = q >= 0.03 ? SAMPLE_MAX : q >= 0.003 ? SAMPLE_MAX / 2 : SAMPLE_MAX / 4;
-            m = std::min<uint64_t>(std::max<uint64_t>(m, SAMPLE_MIN), cap);
+            const double balance = 1048576.0 * std::pow(((double)g.n / 350e6) * std::sqrt(std::max(q, 1e-9) / 0.1), 2.0 / 3.0);
+            const double capacity = 230400.0 * q * (1.0 - q);
+            uint64_t m = (uint64_t)std::max(balance, capacity);
+            m = std::min<uint64_t>(std::min<uint64_t>(m, g.n / 16), SAMPLE_MAX);
+            m = std::max<uint64_t>(m, SAMPLE_MIN) & ~7ull;
             e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
             e.sample_begin = smp; smp += m;
             fast_list.push_back((uint32_t)s);
@@ -194,7 +199,9 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             const bool per_tile = seg_tiles <= c->max_main_grid;
             const uint64_t slack = per_tile ? g.n / 16 + 1024 : g.n / 32 + 16384;
             const uint64_t regions = per_tile ? seg_tiles : c->max_main_grid;
-            const uint64_t tiles_per_region = per_tile ? 1 : (seg_tiles + regions - 1) / regions;
+            // (a CTA takes groups of MAIN_GROUP consecutive tiles, every regions-th group: the segment overlaps at
+            // most seg_tiles / MAIN_GROUP + 2 groups)
+            const uint64_t tiles_per_region = per_tile ? 1 : MAIN_GROUP * ((seg_tiles / MAIN_GROUP + 2 + regions - 1) / regions);
             const uint64_t cand_region = tiles_per_region * ((slack + seg_tiles - 1) / seg_tiles + 16);
             const uint64_t flag_region = tiles_per_region * ((g.k + slack + seg_tiles - 1) / seg_tiles + 16);
             if (flag_region * regions > 0xFFFFFFFFull) return SC_ERR_RANGE;
@@ -218,6 +225,20 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
         maskw += (g.n + 31) / 32;
         msg += g.k;
+    }
+    // The fast list starts with the segments whose sample is large enough for a cluster of CTAs to pay
+    // (the bracket kernel takes them eight CTAs at a time, the rest one CTA each); the position in the
+    // list is the segment's fast index, and the sample keys are stored in list order.
+    std::stable_sort(fast_list.begin(), fast_list.end(), [&](uint32_t a, uint32_t b) {
+        return (h[a].sample_m >= BRACKET_BIG_SAMPLE) > (h[b].sample_m >= BRACKET_BIG_SAMPLE);
+    });
+    uint32_t big_count = 0;
+    smp = 0;
+    for (size_t i = 0; i < fast_list.size(); ++i) {
+        SegEntry& e = h[fast_list[i]];
+        e.fast_index = (uint32_t)i;
+        e.sample_begin = smp; smp += e.sample_m;
+        if (e.sample_m >= BRACKET_BIG_SAMPLE) ++big_count;
     }
     if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
     if (fast_count > c->max_fast_per_worker) return SC_ERR_RANGE;
@@ -253,7 +274,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     L.scat_per_group = (uint32_t)scat; L.K_total = (uint32_t)msg; L.n_total = n; L.mask_words_per_group = maskw;
     L.cand_per_worker = cand; L.flag_per_worker = flag; L.sample_per_worker = smp; L.fast_per_worker = fast_count;
     c->layout = L;
-    c->slow_segments = slow_count; c->max_sample_m = max_m; c->max_flag_cap = max_cap;
+    c->slow_segments = slow_count; c->fast_big = big_count; c->max_sample_m = max_m; c->max_flag_cap = max_cap;
     c->cached_segs.assign(segs, segs + nseg);
     c->cached_n = n;
     c->layout_valid = true;
@@ -314,11 +335,21 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
             SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
             { Launch l(c, KIND_SAMPLE, stream);
-              topk_sample_kernel<<<dim3((c->max_sample_m / 8 + THREADS - 1) / THREADS, PF), THREADS, 0, stream>>>(fp); }
+              topk_sample_kernel<<<dim3((uint32_t)((L.sample_per_worker / 8 + THREADS - 1) / THREADS), W), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_BRACKET, stream);
-              topk_bracket_kernel<<<PF * BRACKET_CTAS, THREADS, 0, stream>>>(fp); }
+              const uint32_t big = c->fast_big, small = L.fast_per_worker - big;
+              if (big) {                                               // clusters of BRACKET_CTAS CTAs, one per problem
+                  cudaLaunchConfig_t cfg = {};
+                  cfg.gridDim = dim3(big * (uint32_t)W * BRACKET_CTAS); cfg.blockDim = dim3(THREADS); cfg.stream = stream;
+                  cudaLaunchAttribute attr;
+                  attr.id = cudaLaunchAttributeClusterDimension;
+                  attr.val.clusterDim.x = BRACKET_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+                  cfg.attrs = &attr; cfg.numAttrs = 1;
+                  SC_CUDA(cudaLaunchKernelEx(&cfg, topk_bracket_kernel<BRACKET_CTAS>, fp, 0u, big));
+              }
+              if (small) topk_bracket_kernel<1><<<small * (uint32_t)W, THREADS, 0, stream>>>(fp, big, small); }
             { Launch l(c, KIND_MAIN, stream);
-              topk_main_kernel<<<persistent_grid(c, c->occ_main, items), THREADS, 0, stream>>>(fp); }
+              topk_main_kernel<<<persistent_grid(c, c->occ_main, (items + MAIN_GROUP - 1) / MAIN_GROUP), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDBIN, stream);
               topk_candbin_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDFILTER, stream);
@@ -382,7 +413,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
 
     if (scheme == SC_RANDBLOCK) {
         { Launch l(c, KIND_RANDBLOCK, stream);
-          randblock_kernel<<<persistent_grid(c, c->occ_block, items), THREADS, 0, stream>>>(
+          randblock_kernel<<<persistent_grid(c, c->occ_block, (items + STREAM_GROUP - 1) / STREAM_GROUP), THREADS, 0, stream>>>(
               L, grads, residuals, c->d_seeds, out_vals, out_idx, items); }
         SC_CUDA(cudaGetLastError());
         return SC_OK;
@@ -406,7 +437,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               row_scan_kernel<<<groups, THREADS, 0, stream>>>(c->d_offsets, L.tiles_per_worker); }
         }
         { Launch l(c, KIND_RANDK_PACK, stream);
-          randk_pack_kernel<<<persistent_grid(c, c->occ_pack_mask, items), THREADS, 0, stream>>>(
+          randk_pack_kernel<<<persistent_grid(c, c->occ_pack_mask, (items + STREAM_GROUP - 1) / STREAM_GROUP), THREADS, 0, stream>>>(
               L, grads, residuals, c->d_mask, c->d_offsets, shared_seeds ? 0u : 1u, out_vals, out_idx, items,
               c->d_status); }
         SC_CUDA(cudaGetLastError());

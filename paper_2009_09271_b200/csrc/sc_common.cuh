@@ -96,6 +96,17 @@ struct FastState {
 };
 
 constexpr uint32_t FAST_MIN_N = 1u << 16;
+// The top-k streaming pass hands out tiles in groups of MAIN_GROUP consecutive tiles: CTA b takes groups
+// b, b + grid, b + 2 grid, ...  Consecutive tiles mostly belong to the same segment, so the per-segment
+// bookkeeping of a CTA is flushed once per group instead of once per tile when segments are short.
+#ifndef SC_MAIN_GROUP
+#define SC_MAIN_GROUP 8
+#endif
+constexpr uint32_t MAIN_GROUP = SC_MAIN_GROUP;
+#ifndef SC_STREAM_GROUP
+#define SC_STREAM_GROUP 4
+#endif
+constexpr uint32_t STREAM_GROUP = SC_STREAM_GROUP;        // the same for the random-k and block-random-k streams
 constexpr uint32_t SAMPLE_MIN = 1u << 12, SAMPLE_MAX = 1u << 20;
 constexpr uint32_t CAND_BINS = 2048;
 constexpr uint32_t LIST2_CAP = 4096;
@@ -231,7 +242,7 @@ __device__ inline uint32_t key_of(float p) { return __float_as_uint(p) & 0x7FFFF
 
 // Tiles are laid on the 128-byte grid of the row, so that a warp's 512-byte access covers four
 // whole cache lines: elements of the segment before its first 128-byte boundary (0..31).
-// A persistent kernel takes tile `item + gridDim.x` after tile `item`.  While the top-k pass works on a
+// A persistent kernel knows which tile it takes next.  While the top-k pass works on a
 // tile's flagged elements its CTA has no loads in flight, so each thread asks L2 for one 128-byte line of
 // the tile that comes next (g by the lower half of the CTA, e by the upper half) and the next round of
 // loads finds its data in L2.  Only that kernel uses it: the random-k and block-random-k streams, which

@@ -43,7 +43,9 @@ randblock_kernel(Layout L, const float* __restrict__ grads, float* __restrict__ 
                  const uint64_t* __restrict__ seeds, float* __restrict__ out_vals,
                  uint32_t* __restrict__ out_idx, uint32_t total_items) {
     __shared__ uint32_t s_dec[4];
-    for (uint32_t item = blockIdx.x; item < total_items; item += gridDim.x) {
+    const uint32_t group_step = (gridDim.x - 1u) * STREAM_GROUP + 1u;
+    for (uint32_t item = blockIdx.x * STREAM_GROUP, ig = 0; item < total_items;
+         item += (ig + 1u == STREAM_GROUP ? group_step : 1u), ig = (ig + 1u == STREAM_GROUP ? 0u : ig + 1u)) {
         if (threadIdx.x == 0) {
             uint32_t w = item / L.tiles_per_worker;
             uint32_t lt = item - w * L.tiles_per_worker;
@@ -161,7 +163,9 @@ randk_pack_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
     __shared__ uint32_t s_wtot[2][WARPS];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     uint32_t parity = 0;
-    for (uint32_t item = blockIdx.x; item < total_items; item += gridDim.x, parity ^= 1u) {
+    const uint32_t group_step = (gridDim.x - 1u) * STREAM_GROUP + 1u;
+    for (uint32_t item = blockIdx.x * STREAM_GROUP, ig = 0; item < total_items;
+         item += (ig + 1u == STREAM_GROUP ? group_step : 1u), ig = (ig + 1u == STREAM_GROUP ? 0u : ig + 1u), parity ^= 1u) {
         const uint32_t w = item / L.tiles_per_worker;
         const uint32_t lt = item - w * L.tiles_per_worker;
         const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);

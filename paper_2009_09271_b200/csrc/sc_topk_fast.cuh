@@ -99,11 +99,17 @@ __device__ inline bool find_from_top(HistPtr h, uint32_t need, uint32_t* s_tmp /
 __global__ void __launch_bounds__(THREADS)
 topk_sample_kernel(FastParams P) {
     const Layout& L = P.L;
-    uint32_t w, s;
-    fast_problem(L, blockIdx.y, w, s);
-    const SegEntry seg = L.segs[s];
-    const uint32_t c = blockIdx.x * THREADS + threadIdx.x;            // sector of the sample
-    if (c >= seg.sample_m / 8u) return;
+    const uint32_t w = blockIdx.y;
+    const uint64_t pos = ((uint64_t)blockIdx.x * THREADS + threadIdx.x) * 8u;   // first key of this thread's sector
+    if (pos >= L.sample_per_worker) return;
+    // the samples of a worker's large segments lie one after the other, in fast-list order: find the segment
+    uint32_t f0 = 0, f1 = L.fast_per_worker - 1u;
+    while (f0 < f1) {
+        const uint32_t mid = (f0 + f1 + 1u) >> 1;
+        if (L.segs[L.fast_list[mid]].sample_begin <= pos) f0 = mid; else f1 = mid - 1u;
+    }
+    const SegEntry seg = L.segs[L.fast_list[f0]];
+    const uint32_t c = (uint32_t)((pos - seg.sample_begin) / 8u);      // sector of the segment's sample
     const size_t row = (size_t)w * L.n_total + seg.offset;
     const float* g = P.grads + row;
     const float* e = P.residuals + row;
@@ -126,24 +132,29 @@ topk_sample_kernel(FastParams P) {
 // the total and hands the two bins back the same way; a second round refines them by ten more bits.
 // The cluster barriers are the hardware's; no CTA leaves before the last one (a peer's shared memory
 // must stay alive while it is read).
+// Segments with a small sample take one CTA each (C = 1: no cluster calls at all).  `first` and `count`
+// select a range of the fast list; the grid covers count problems of every worker.
 constexpr uint32_t BRACKET_CTAS = 8;
-__global__ void __cluster_dims__(BRACKET_CTAS, 1, 1) __launch_bounds__(THREADS)
-topk_bracket_kernel(FastParams P) {
+constexpr uint32_t BRACKET_BIG_SAMPLE = 1u << 15;                      // samples from this size up take a cluster
+template <uint32_t C>
+__global__ void __launch_bounds__(THREADS)
+topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     namespace cg = cooperative_groups;
     __shared__ uint32_t h0[HIST0_BINS];
     __shared__ uint32_t hA[1024], hB[1024];
     __shared__ uint32_t s_tmp[WARPS + 4];
     __shared__ uint32_t s_bins[4];                                     // binA, binB, needA, needB (valid in CTA 0)
     cg::cluster_group cluster = cg::this_cluster();
-    const uint32_t rank = cluster.block_rank();
+    const uint32_t rank = C > 1 ? cluster.block_rank() : 0u;
     const Layout& L = P.L;
     uint32_t w, s;
-    const uint32_t prob = fast_problem(L, blockIdx.x / BRACKET_CTAS, w, s);
+    const uint32_t pidx = blockIdx.x / C;                              // problem of this launch: (worker, position in the range)
+    const uint32_t prob = fast_problem(L, (pidx / count) * L.fast_per_worker + first + pidx % count, w, s);
     const SegEntry seg = L.segs[s];
     const uint32_t m = seg.sample_m;
     const uint4* smp = reinterpret_cast<const uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin);
     // this CTA's share of the sample (in groups of four keys)
-    const uint32_t per = (m / 4u + BRACKET_CTAS - 1u) / BRACKET_CTAS;
+    const uint32_t per = (m / 4u + C - 1u) / C;
     const uint32_t i_begin = min(rank * per, m / 4u), i_end = min(i_begin + per, m / 4u);
     // ranks (from the top) that bracket the k-th largest of the segment
     const double q = (double)seg.k / (double)seg.n;
@@ -161,14 +172,14 @@ topk_bracket_kernel(FastParams P) {
         atomicAdd(&h0[k.x >> 20], 1u); atomicAdd(&h0[k.y >> 20], 1u);
         atomicAdd(&h0[k.z >> 20], 1u); atomicAdd(&h0[k.w >> 20], 1u);
     }
-    cluster.sync();
+    if (C > 1) cluster.sync();
     // when k is so small that no sample rank lies safely above the threshold there is no "sure"
     // set (hi stays at the largest key); the candidate histogram then spans up to the largest
     // sample key and everything above it shares the last bin
     if (rank == 0) {
         for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) {
             uint32_t v = h0[b];
-            for (uint32_t r = 1; r < BRACKET_CTAS; ++r) v += cluster.map_shared_rank(h0, r)[b];
+            for (uint32_t r = 1; r < C; ++r) v += cluster.map_shared_rank(h0, r)[b];
             h0[b] = v;
         }
         __syncthreads();
@@ -178,8 +189,9 @@ topk_bracket_kernel(FastParams P) {
         if (have_lo) find_from_top<HIST0_BINS>(h0, (uint32_t)j_lo, s_tmp, binB, needB, cnt);
         if (threadIdx.x == 0) { s_bins[0] = binA; s_bins[1] = binB; s_bins[2] = needA; s_bins[3] = needB; }
     }
-    cluster.sync();
-    const uint32_t* bins0 = cluster.map_shared_rank(s_bins, 0);
+    if (C > 1) cluster.sync();
+    if (C == 1) __syncthreads();
+    const uint32_t* bins0 = C > 1 ? cluster.map_shared_rank(s_bins, 0) : s_bins;
     const uint32_t binA = bins0[0], binB = bins0[1];
     for (uint32_t i = i_begin + threadIdx.x; i < i_end; i += THREADS) {
         const uint4 k = smp[i];
@@ -190,11 +202,11 @@ topk_bracket_kernel(FastParams P) {
             if (have_lo && (kk[c] >> 20) == binB) atomicAdd(&hB[(kk[c] >> 10) & 1023u], 1u);
         }
     }
-    cluster.sync();
+    if (C > 1) cluster.sync();
     if (rank == 0) {
         for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) {
             uint32_t va = hA[b], vb = hB[b];
-            for (uint32_t r = 1; r < BRACKET_CTAS; ++r) {
+            for (uint32_t r = 1; r < C; ++r) {
                 va += cluster.map_shared_rank(hA, r)[b];
                 vb += cluster.map_shared_rank(hB, r)[b];
             }
@@ -215,7 +227,7 @@ topk_bracket_kernel(FastParams P) {
             P.state[prob] = st;
         }
     }
-    cluster.sync();                                                    // peers stay until CTA 0 has read their histograms
+    if (C > 1) cluster.sync();                                                    // peers stay until CTA 0 has read their histograms
 }
 
 // ---- main streaming pass ---------------------------------------------------------------
@@ -288,7 +300,9 @@ topk_main_kernel(FastParams P) {
     uint32_t slot3 = 0;                                                // counter pair of the current tile
     uint32_t pend_item = 0xFFFFFFFFu, pend_slot = 0, pend_room = 0;    // tile whose counts are not written yet
     bool pend_accumulates = false;
-    for (uint32_t item = blockIdx.x; ; item += gridDim.x) {
+    const uint32_t group_step = (gridDim.x - 1u) * MAIN_GROUP + 1u;    // from a group's last tile to the next group's first
+    for (uint32_t item = blockIdx.x * MAIN_GROUP, ig = 0; ;
+         item += (ig + 1u == MAIN_GROUP ? group_step : 1u), ig = (ig + 1u == MAIN_GROUP ? 0u : ig + 1u)) {
         const MainTile T = main_decode(P, item);
         // ---- flush the per-segment accumulators when the segment changes ---------------------------
         const long long prob = T.have ? (long long)T.w * L.nseg + T.s : -2;
@@ -366,8 +380,15 @@ topk_main_kernel(FastParams P) {
         }
         // the loads of this tile have landed: ask L2 for the tile this CTA takes next, so that DRAM stays busy
         // during the per-element work below (measured on 350 M x 16 at 1 %: 12.3 -> 10.85 ms)
-        if (SC_PREFETCH_DIST && T.full && T.lt + gridDim.x * SC_PREFETCH_DIST + 1u < L.segs[T.s + 1].tile_begin)
-            prefetch_tile_l2(T.g, e, T.first + (long long)gridDim.x * SC_PREFETCH_DIST * TILE);
+        if (SC_PREFETCH_DIST) {
+            const uint32_t ahead = ig + 1u == MAIN_GROUP ? group_step : 1u;    // distance to this CTA's next tile
+            if (T.full && T.lt + ahead + 1u < L.segs[T.s + 1].tile_begin) {
+                prefetch_tile_l2(T.g, e, T.first + (long long)ahead * TILE);
+            } else {                                                   // the next tile lies in another segment: locate it
+                const MainTile N = main_decode(P, item + ahead);
+                if (N.have && N.fast && N.full) prefetch_tile_l2(N.g, N.e, N.first);
+            }
+        }
         // ---- ranks of the flagged elements, in coordinate order ---------------------------------------
         const uint32_t fcnt4 = pack_counts(flag16);
         const uint32_t finc4 = warp_inclusive_scan(fcnt4, lane);
