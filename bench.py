@@ -31,7 +31,7 @@ UNIT = "elements/s"
 CONTRACT_PEAK_GBS = 8000.0        # the nominal B200 HBM figure the target is stated against
 FALLBACK_PEAK_GBS = 6650.0        # used only if MEASURED_PEAKS.json is absent
 # DRAM bytes per gradient element of the streaming kernels, measured once with ncu on a small case
-NCU_DRAM_BYTES_PER_ELEMENT = {"topk_main": 11.84, "randk_pack": 11.93, "randblock": 11.81}
+NCU_DRAM_BYTES_PER_ELEMENT = {"topk_main": 11.85, "randk_pack": 11.93, "randblock": 11.80}
 
 
 def parse_args():
@@ -355,7 +355,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         if per_elem is not None:
             roofline["traffic"] = per_elem * n * W
             roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum per element from one ncu capture "
-                                        "at n=1e8, W=2 (profiles/topk_main_kernel_n100M_W2.md), scaled by n*W")
+                                        "at n=1e8, W=2 (profiles/streaming_kernels_n100M_W2.md), scaled by n*W")
     step_roof = {}
     for s in schemes:
         t_s = per_scheme_ms[s] / args.steps * 1e-3
