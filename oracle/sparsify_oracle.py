@@ -30,6 +30,13 @@ project's design notes):
  * Random-k: k DISTINCT coordinates, {pi(j) : j < k} for a keyed bijection pi
    of [0, n) (a Feistel network with cycle walking, specified below).
  * Block-random-k: the block does not wrap; its start is uniform on [0, n-k].
+   Variant RANDBLOCK_WRAP: the start is uniform on [0, n) and the block wraps
+   around the end of the segment, so every coordinate is kept with the same
+   probability k/n (without the wrap the first and last k-1 coordinates are
+   kept less often).
+ * Step size: with gamma != 1 the accumulate line is evaluated as ONE fused
+   multiply-add, p = round(gamma * g + e) (a single fp32 rounding); gamma = 1
+   gives the plain add bit for bit.
  * "Same seed state": the seed is an argument; equal seeds give equal
    coordinates on every worker.
  * Scope (layer-wise or global): a segment table; segment s of a call uses the
@@ -39,7 +46,9 @@ Parity pins (tests/test_oracle_*.py): brute-force ordering by Python tuples on
 tiny inputs, set equality with torch.topk on distinct magnitudes, k = 0 / k = n
 limits, e' + q == p, exact telescoping sums on integer-valued gradients, the
 dense limit against a three-line loop, enumeration of pi for every small n,
-chi-square tests of inclusion frequencies and block starts.
+chi-square tests of inclusion frequencies and block starts; the fused
+multiply-add against exact rational arithmetic (fractions.Fraction) on random
+and constructed halfway cases.
 Parity unpinned: agreement of the random generator with the authors' own code
 (the paper names no generator; the one below is this project's specification).
 """
@@ -49,8 +58,8 @@ from typing import List, Sequence, Tuple
 
 import numpy as np
 
-TOPK, RANDK, RANDBLOCK = 0, 1, 2
-SCHEMES = {"topk": TOPK, "randk": RANDK, "randblock": RANDBLOCK}
+TOPK, RANDK, RANDBLOCK, RANDBLOCK_WRAP = 0, 1, 2, 3
+SCHEMES = {"topk": TOPK, "randk": RANDK, "randblock": RANDBLOCK, "randblock_wrap": RANDBLOCK_WRAP}
 
 _M64 = (1 << 64) - 1
 _M32 = (1 << 32) - 1
@@ -101,6 +110,13 @@ def block_start(seed_s: int, n: int, k: int) -> int:
     64-bit hash h of the segment seed, so 0 <= a <= n-k (no wrap-around)."""
     h = mix64(seed_s, SALT_BLOCK)
     return (h * (n - k + 1)) >> 64
+
+
+def block_start_wrap(seed_s: int, n: int) -> int:
+    """Start a of the wrapping block {(a + j) mod n : j < k}: floor(h * n / 2^64)
+    for the same 64-bit hash h, so 0 <= a < n (a = 0 for an empty segment)."""
+    h = mix64(seed_s, SALT_BLOCK)
+    return (h * n) >> 64
 
 
 def feistel_params(seed_s: int, n: int) -> Tuple[int, int, List[int]]:
@@ -177,29 +193,70 @@ def select(scheme: int, p: np.ndarray, k: int, seed_s: int) -> np.ndarray:
     if scheme == RANDBLOCK:
         a = block_start(seed_s, n, k)
         return np.arange(a, a + k, dtype=np.uint32)
+    if scheme == RANDBLOCK_WRAP:
+        if n == 0:
+            return np.zeros(0, np.uint32)
+        a = block_start_wrap(seed_s, n)
+        return np.sort((a + np.arange(k, dtype=np.int64)) % n).astype(np.uint32)
     raise ValueError("unknown scheme")
 
 
 # ---------------------------------------------------------------------------
 # Algorithm 1, per worker: accumulate, compress, residual
 # ---------------------------------------------------------------------------
+def fma32(a: np.ndarray, b, c: np.ndarray) -> np.ndarray:
+    """round_fp32(a * b + c) with a single rounding, elementwise on fp32 inputs.
+
+    The product of two fp32 numbers is exact in fp64.  The fp64 sum s = prod + c
+    is rounded once; its exact error follows from the classical two-sum identity.
+    Replacing s by its round-to-odd neighbour when it is inexact (truncate towards
+    zero, then set the last mantissa bit) makes the final fp64 -> fp32 rounding
+    come out as if the exact sum had been rounded directly (fp64 carries more
+    than 2 x 24 + 2 bits)."""
+    a64 = np.asarray(a, np.float32).astype(np.float64)
+    b64 = np.asarray(b, np.float32).astype(np.float64)
+    c64 = np.asarray(c, np.float32).astype(np.float64)
+    with np.errstate(invalid="ignore", over="ignore"):
+        prod = a64 * b64
+        s = prod + c64
+        bb = s - prod
+        err = (prod - (s - bb)) + (c64 - bb)
+    inexact = np.isfinite(s) & np.isfinite(err) & (err != 0.0)
+    bits = np.ascontiguousarray(s).view(np.int64).copy()
+    sign = bits & np.int64(-0x8000000000000000)
+    mag = bits & np.int64(0x7FFFFFFFFFFFFFFF)
+    shrink = inexact & ((err > 0.0) != (s > 0.0))                   # |exact| < |s|: step towards zero
+    mag = mag - shrink.astype(np.int64)
+    mag = mag | inexact.astype(np.int64)
+    s_odd = (sign | mag).view(np.float64)
+    with np.errstate(over="ignore"):
+        return s_odd.astype(np.float32)
+
+
+def accumulate(grad: np.ndarray, residual: np.ndarray, gamma: float = 1.0) -> np.ndarray:
+    """Algorithm 1, accumulate line: p = gamma * g + e.  gamma == 1: one fp32 add."""
+    if np.float32(gamma) == np.float32(1.0):
+        return grad + residual
+    return fma32(np.float32(gamma), grad, residual)
+
+
 def compress(scheme: int, grad: np.ndarray, residual: np.ndarray, k: int, seed: int,
-             ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+             gamma: float = 1.0) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     """One worker, global scope.  Returns (vals[k], idx[k] ascending, new residual)."""
-    vals, idx, e_new = compress_segments(scheme, grad, residual, [(0, grad.size, k)], seed)
+    vals, idx, e_new = compress_segments(scheme, grad, residual, [(0, grad.size, k)], seed, gamma)
     return vals, idx, e_new
 
 
 def compress_segments(scheme: int, grad: np.ndarray, residual: np.ndarray,
                       segments: Sequence[Tuple[int, int, int]], seed: int,
-                      ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+                      gamma: float = 1.0) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     """One worker, a table of (offset, n_s, k_s).  Message slots of segment s
     follow those of segment s-1; coordinates are global (offset added)."""
     assert grad.dtype == np.float32 and residual.dtype == np.float32
     e_new = residual.copy()
     vals_all, idx_all = [], []
     for s, (off, n_s, k_s) in enumerate(segments):
-        p = grad[off:off + n_s] + residual[off:off + n_s]            # p = gamma*g + e   (one fp32 add)
+        p = accumulate(grad[off:off + n_s], residual[off:off + n_s], gamma)   # p = gamma*g + e (one rounding)
         sel = select(scheme, p, k_s, segment_seed(seed, s))            # coordinates kept by C(p)
         vals_all.append(p[sel].copy())                                 # q^w on its support
         idx_all.append(sel.astype(np.uint32) + np.uint32(off))
@@ -233,11 +290,11 @@ def aggregate_apply(x: np.ndarray, vals: Sequence[np.ndarray], idx: Sequence[np.
 
 
 def step(scheme: int, grads: Sequence[np.ndarray], residuals: Sequence[np.ndarray],
-         segments: Sequence[Tuple[int, int, int]], seeds: Sequence[int]):
+         segments: Sequence[Tuple[int, int, int]], seeds: Sequence[int], gamma: float = 1.0):
     """All W workers compress, then one aggregate.  Returns
     (vals list, idx list, new residual list, dense average)."""
     vals, idx, res = [], [], []
     for g, e, sd in zip(grads, residuals, seeds):
-        v, i, r = compress_segments(scheme, g, e, segments, sd)
+        v, i, r = compress_segments(scheme, g, e, segments, sd, gamma)
         vals.append(v), idx.append(i), res.append(r)
     return vals, idx, res, aggregate(vals, idx, grads[0].size)
