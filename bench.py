@@ -397,6 +397,24 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             tim[name] = round(a.elapsed_time(b) / 3, 4)
         tim["note"] = ("x <- x - average applied at sent coordinates only, on the last scheme's messages; "
                        "the dense sc_aggregate of the same messages is in kernels.agg_tiles")
+
+        # ---- next row: the block that wraps around, and the accumulate line with a step size -------
+        def timed_step(code, gamma):
+            e_tmp = res[schemes[-1]]                           # any residual buffer: the metric's run is over
+            ctx.sc_set_gamma(gamma)
+            ctx.sc_step(code, grads[0], e_tmp, seg_t, seeds(0), vals, idx, out)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for t in range(3):
+                ctx.sc_step(code, grads[t % pool], e_tmp, seg_t, seeds(t + 1), vals, idx, out)
+            b.record()
+            torch.cuda.synchronize()
+            ctx.sc_set_gamma(1.0)
+            return round(a.elapsed_time(b) / 3, 4)
+        tim["randblock_wrap_step_ms"] = timed_step(sc.SC_RANDBLOCK_WRAP, 1.0)
+        tim["topk_step_gamma_0.1_ms"] = timed_step(sc.SC_TOPK, 0.1)
+        tim["note_steps"] = ("whole sc_step (compress + aggregate) on this workload: wrap-around block scheme; "
+                             "top-k with p = fma(0.1, g, e)")
         line["next_rows"] = tim
         del xmodel
 

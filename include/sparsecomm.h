@@ -45,7 +45,11 @@ typedef struct sc_ctx sc_ctx;
 /* Compressor C(.) -- Methodology, "compressor or sparsification scheme". */
 enum { SC_TOPK = 0,       /* k largest |p|, ties to the lowest coordinate            */
        SC_RANDK = 1,      /* k distinct coordinates from a seeded bijection of [0,n)  */
-       SC_RANDBLOCK = 2   /* one seeded start a in [0,n-k], coordinates a..a+k-1      */ };
+       SC_RANDBLOCK = 2,  /* one seeded start a in [0,n-k], coordinates a..a+k-1      */
+       SC_RANDBLOCK_WRAP = 3 /* start a in [0,n), coordinates (a+j) mod n: a variant of the
+                               block scheme (Methodology, Block-random-k) in which every
+                               coordinate is kept with the same probability k/n; the
+                               message is still ascending (wrapped head first)          */ };
 
 enum { SC_OK = 0,
        SC_ERR_INVALID = -1,      /* null pointer, misaligned base pointer, unknown scheme, bad table */
@@ -64,6 +68,13 @@ typedef struct { uint64_t offset, n, k; } sc_segment;
 int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments);
 void sc_destroy(sc_ctx* ctx);
 const char* sc_strerror(int code);
+
+/* Step size of the accumulate line of Algorithm 1, p = gamma * g + e.  The default, 1, is the plain
+ * fp32 add (the caller has folded gamma into g).  Any other value makes every later compress call of
+ * this context evaluate the line as ONE fused multiply-add per element (a single rounding), so the
+ * caller can pass the raw gradient.  Host-side state, no device work; always returns SC_OK for a
+ * valid context. */
+int sc_set_gamma(sc_ctx* ctx, float gamma);
 
 /* Synchronises `stream`, then returns (and clears) the sticky device status. */
 int sc_sync_status(sc_ctx* ctx, void* stream);

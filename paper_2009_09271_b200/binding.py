@@ -12,13 +12,13 @@ from typing import Optional, Sequence
 
 import torch
 
-SC_TOPK, SC_RANDK, SC_RANDBLOCK = 0, 1, 2
-SCHEMES = {"topk": SC_TOPK, "randk": SC_RANDK, "randblock": SC_RANDBLOCK}
+SC_TOPK, SC_RANDK, SC_RANDBLOCK, SC_RANDBLOCK_WRAP = 0, 1, 2, 3
+SCHEMES = {"topk": SC_TOPK, "randk": SC_RANDK, "randblock": SC_RANDBLOCK, "randblock_wrap": SC_RANDBLOCK_WRAP}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsparsecomm.so")
 
-EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_scratch_bytes", "sc_launch_count",
+EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_set_gamma", "sc_scratch_bytes", "sc_launch_count",
            "sc_topk_path_counts", "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
            "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_aggregate_static", "sc_aggregate_apply",
            "sc_aggregate_apply_shared", "sc_step", "sc_step_host"]
@@ -53,6 +53,8 @@ def load_library() -> ctypes.CDLL:
     lib.sc_destroy.restype = None
     lib.sc_strerror.argtypes = [ci]
     lib.sc_strerror.restype = ctypes.c_char_p
+    lib.sc_set_gamma.argtypes = [vp, ctypes.c_float]
+    lib.sc_set_gamma.restype = ci
     lib.sc_sync_status.argtypes = [vp, vp]
     lib.sc_sync_status.restype = ci
     lib.sc_scratch_bytes.argtypes = [vp]
@@ -195,6 +197,9 @@ class Context:
         return {self._lib.sc_profile_name(i).decode(): (ms[i], cnt[i]) for i in range(kinds)}
 
     # -- the C ABI, one method per entry point ---------------------------------
+    def sc_set_gamma(self, gamma: float) -> None:
+        _check(self._lib.sc_set_gamma(self._h, float(gamma)), "sc_set_gamma")
+
     def sc_sync_status(self, stream=None) -> int:
         return self._lib.sc_sync_status(self._h, _stream(stream))
 

@@ -58,6 +58,7 @@ struct sc_ctx {
     uint32_t last_topk_problems = 0; // (worker, segment) pairs of the most recent top-k call
     uint32_t slow_segments = 0;      // segments of the cached table that take the radix-select path
     uint32_t max_sample_m = 0, fast_big = 0;
+    float gamma = 1.0f;                  // step size of the accumulate line (sc_set_gamma)
     uint32_t max_flag_cap = 0, max_cand_cap = 0;
     int occ_main = 1, occ_emit = 1, occ_emit_v[4] = {1, 1, 1, 1};
     uint64_t* d_seeds = nullptr;
@@ -285,7 +286,7 @@ int check_batch_args(const sc_ctx* c, int scheme, int W, const void* grads, cons
                      const sc_segment* segs, int nseg, const uint64_t* seeds, const void* out_vals,
                      const void* out_idx) {
     if (!c || !segs || !seeds) return SC_ERR_INVALID;
-    if (scheme != SC_TOPK && scheme != SC_RANDK && scheme != SC_RANDBLOCK) return SC_ERR_INVALID;
+    if (scheme != SC_TOPK && scheme != SC_RANDK && scheme != SC_RANDBLOCK && scheme != SC_RANDBLOCK_WRAP) return SC_ERR_INVALID;
     if (W < 1 || W > c->max_W || nseg < 1 || nseg > c->max_seg) return SC_ERR_RANGE;
     if (n >= (1ull << 32) || n > c->max_n) return SC_ERR_RANGE;
     uint64_t K = 0;
@@ -310,7 +311,8 @@ inline uint32_t persistent_grid(const sc_ctx* c, int occ, uint64_t items) {
 int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
                   const uint64_t* h_seeds, bool shared_seeds, bool mask_ready,
                   float* out_vals, uint32_t* out_idx, cudaStream_t stream) {
-    const Layout& L = c->layout;
+    Layout L = c->layout;
+    L.gamma = c->gamma;
     if (n == 0 || L.tiles_per_worker == 0) return SC_OK;
     const uint64_t items64 = (uint64_t)W * L.tiles_per_worker;
     if (items64 > 0xFFFFFFF0ull) return SC_ERR_RANGE;
@@ -411,10 +413,10 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
         SC_CUDA(cudaMemcpyAsync(c->d_seeds, h_seeds, sizeof(uint64_t) * W, cudaMemcpyHostToDevice, stream));
     }
 
-    if (scheme == SC_RANDBLOCK) {
+    if (scheme == SC_RANDBLOCK || scheme == SC_RANDBLOCK_WRAP) {
         { Launch l(c, KIND_RANDBLOCK, stream);
           randblock_kernel<<<persistent_grid(c, c->occ_block, (items + STREAM_GROUP - 1) / STREAM_GROUP), THREADS, 0, stream>>>(
-              L, grads, residuals, c->d_seeds, out_vals, out_idx, items); }
+              L, grads, residuals, c->d_seeds, out_vals, out_idx, items, scheme == SC_RANDBLOCK_WRAP ? 1u : 0u); }
         SC_CUDA(cudaGetLastError());
         return SC_OK;
     }
@@ -655,6 +657,12 @@ void sc_destroy(sc_ctx* c) {
     if (c->ev_start) cudaEventDestroy(c->ev_start);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     delete c;
+}
+
+int sc_set_gamma(sc_ctx* c, float gamma) {
+    if (!c) return SC_ERR_INVALID;
+    c->gamma = gamma;
+    return SC_OK;
 }
 
 int sc_sync_status(sc_ctx* c, void* stream) {

@@ -54,7 +54,7 @@ struct Layout {
     uint64_t flag_per_worker; // flagged-list slots per worker
     uint64_t sample_per_worker; // sample keys per worker
     uint32_t fast_per_worker; // fast segments per worker
-    uint32_t pad;
+    float gamma;              // step size of the accumulate line, p = gamma g + e (1: the plain add)
 };
 
 // The tiles (or pack groups) one launch of a radix-select kernel walks: indices inside a worker row,
@@ -132,6 +132,20 @@ __host__ __device__ inline uint32_t mix32(uint32_t x) {
 constexpr uint64_t SALT_BLOCK = 0x626C6F636Bull;
 constexpr uint64_t SALT_RANDK = 0x72616E646B00ull;
 constexpr int FEISTEL_ROUNDS = 6;
+
+// Algorithm 1, accumulate line: p = gamma g + e as ONE fused multiply-add (a single rounding);
+// fmaf(1, g, e) is the plain fp32 add, bit for bit.
+__device__ inline float accumulate(float gamma, float g, float e) { return fmaf(gamma, g, e); }
+__device__ inline float4 accumulate(float gamma, const float4& g, const float4& e) {
+    return make_float4(fmaf(gamma, g.x, e.x), fmaf(gamma, g.y, e.y), fmaf(gamma, g.z, e.z), fmaf(gamma, g.w, e.w));
+}
+
+// Wrap-around variant of the block scheme: the start is uniform on [0, n) and the block is
+// {(a + j) mod n : j < k}, which keeps every coordinate with the same probability k / n.
+__device__ inline uint32_t block_start_wrap(uint64_t seed_s, uint32_t n) {
+    uint64_t h = mix64(seed_s, SALT_BLOCK);
+    return (uint32_t)__umul64hi(h, (uint64_t)n);
+}
 
 __device__ inline uint32_t block_start(uint64_t seed_s, uint32_t n, uint32_t k) {
     uint64_t h = mix64(seed_s, SALT_BLOCK);

@@ -209,8 +209,8 @@ pack_kernel(PackParams P) {
 #pragma unroll
                         for (int j = 0; j < QUADS; ++j) {
                             const float4 gv = __ldcs(pg + j);
-                            q[j].x = gv.x + q[j].x; q[j].y = gv.y + q[j].y;
-                            q[j].z = gv.z + q[j].z; q[j].w = gv.w + q[j].w;
+                            q[j].x = accumulate(P.L.gamma, gv.x, q[j].x); q[j].y = accumulate(P.L.gamma, gv.y, q[j].y);
+                            q[j].z = accumulate(P.L.gamma, gv.z, q[j].z); q[j].w = accumulate(P.L.gamma, gv.w, q[j].w);
                         }
                         float4* po = reinterpret_cast<float4*>(e + mine);
 #pragma unroll
@@ -245,7 +245,7 @@ pack_kernel(PackParams P) {
                             float gv[4];
                             load_quad_stream(g, base, seg.n, gv);
 #pragma unroll
-                            for (int c = 0; c < 4; ++c) p[c] = gv[c] + p[c];
+                            for (int c = 0; c < 4; ++c) p[c] = accumulate(P.L.gamma, gv[c], p[c]);
                             if (valid) store_quad(e, base, valid, p);
 #pragma unroll
                             for (int c = 0; c < 4; ++c)

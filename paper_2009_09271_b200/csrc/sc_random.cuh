@@ -41,7 +41,7 @@ randk_scatter_kernel(Layout L, const uint64_t* __restrict__ seeds, uint32_t* __r
 __global__ void __launch_bounds__(THREADS)
 randblock_kernel(Layout L, const float* __restrict__ grads, float* __restrict__ residuals,
                  const uint64_t* __restrict__ seeds, float* __restrict__ out_vals,
-                 uint32_t* __restrict__ out_idx, uint32_t total_items) {
+                 uint32_t* __restrict__ out_idx, uint32_t total_items, uint32_t wrap) {
     __shared__ uint32_t s_dec[4];
     const uint32_t group_step = (gridDim.x - 1u) * STREAM_GROUP + 1u;
     for (uint32_t item = blockIdx.x * STREAM_GROUP, ig = 0; item < total_items;
@@ -52,17 +52,22 @@ randblock_kernel(Layout L, const float* __restrict__ grads, float* __restrict__ 
             uint32_t s = find_by_tile(L, lt);
             const SegEntry sg = L.segs[s];
             s_dec[0] = w; s_dec[1] = s; s_dec[2] = lt - sg.tile_begin;
-            s_dec[3] = block_start(mix64(seeds[w], s), sg.n, sg.k);
+            s_dec[3] = wrap ? block_start_wrap(mix64(seeds[w], s), sg.n) : block_start(mix64(seeds[w], s), sg.n, sg.k);
         }
         __syncthreads();
         const uint32_t w = s_dec[0], s = s_dec[1], t = s_dec[2], a = s_dec[3];
         const SegEntry seg = L.segs[s];
+        const uint32_t head = (wrap && (uint64_t)a + seg.k > seg.n) ? (uint32_t)((uint64_t)a + seg.k - seg.n) : 0u;   // wrapped entries
         const size_t row = (size_t)w * L.n_total + seg.offset;
         const float* g = grads + row;
         float* e = residuals + row;
         const uint32_t mis = misalign_of(e);
         float* ovals = out_vals + (size_t)w * L.K_total + seg.msg_off;
         uint32_t* oidx = out_idx + (size_t)w * L.K_total + seg.msg_off;
+        // most tiles lie outside the kept block: they only stream p = gamma g + e back
+        const long long tlo = (long long)t * TILE - mis, thi = tlo + TILE;
+        const long long a_end = min((long long)a + (long long)seg.k, (long long)seg.n);
+        const bool touches = seg.k != 0u && ((tlo < a_end && thi > (long long)a) || tlo < (long long)head);
 #pragma unroll
         for (int j = 0; j < QUADS; ++j) {
             const long long base = (long long)t * TILE + (long long)(j * THREADS + threadIdx.x) * 4 - mis;
@@ -71,14 +76,20 @@ randblock_kernel(Layout L, const float* __restrict__ grads, float* __restrict__ 
             if (!m) continue;
             load_quad_stream(g, base, seg.n, gv);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                p[c] = gv[c] + p[c];
-                const long long i = base + c;
-                if (((m >> c) & 1u) && i >= (long long)a && i < (long long)a + seg.k) {
-                    const uint32_t slot = (uint32_t)(i - a);
-                    ovals[slot] = p[c];
-                    oidx[slot] = (uint32_t)(seg.offset + (uint64_t)i);
-                    p[c] = 0.0f;
+            for (int c = 0; c < 4; ++c) p[c] = accumulate(L.gamma, gv[c], p[c]);
+            if (touches) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const long long i = base + c;
+                    // distance from the block's start, cyclically when the block wraps: kept iff < k.  A wrapped
+                    // block's head [0, a + k - n) comes first in the ascending message, its tail [a, n) after it.
+                    const long long d = i >= (long long)a ? i - a : (wrap ? i + seg.n - a : (long long)seg.k);
+                    if (((m >> c) & 1u) && d < (long long)seg.k) {
+                        const uint32_t slot = i >= (long long)a ? head + (uint32_t)(i - a) : (uint32_t)i;
+                        ovals[slot] = p[c];
+                        oidx[slot] = (uint32_t)(seg.offset + (uint64_t)i);
+                        p[c] = 0.0f;
+                    }
                 }
             }
             store_quad(e, base, m, p);
@@ -235,7 +246,7 @@ randk_pack_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
             for (int j = 0; j < QUADS; ++j) {
                 const float4 ev = __ldcs(reinterpret_cast<const float4*>(e + mine + 128 * j));
                 const float4 gv = __ldcs(reinterpret_cast<const float4*>(g + mine + 128 * j));
-                qv[j] = make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w);
+                qv[j] = accumulate(L.gamma, gv, ev);
             }
             if (bits) {
 #pragma unroll
@@ -270,7 +281,7 @@ randk_pack_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
                 uint32_t rank = wbase + rowbase[j] + ((ex4 >> (8 * j)) & 0xFFu);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    p[c] = gv[c] + p[c];
+                    p[c] = accumulate(L.gamma, gv[c], p[c]);
                     if ((bits >> (4 * j + c)) & 1u) {
                         if (rank < seg.k) {
                             ovals[rank] = p[c];

@@ -69,7 +69,7 @@ topk_hist0_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
                 float gv[4];
                 load_quad_stream(g, base, seg.n, gv);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) p[c] = gv[c] + p[c];
+                for (int c = 0; c < 4; ++c) p[c] = accumulate(L.gamma, gv[c], p[c]);
                 if (m) store_quad(e, base, m, p);
             }
 #pragma unroll

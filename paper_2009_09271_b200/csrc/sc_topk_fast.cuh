@@ -120,8 +120,9 @@ topk_sample_kernel(FastParams P) {
     const float4 e0 = *reinterpret_cast<const float4*>(e + at), e1 = *reinterpret_cast<const float4*>(e + at + 4);
     const float4 g0 = *reinterpret_cast<const float4*>(g + at), g1 = *reinterpret_cast<const float4*>(g + at + 4);
     uint4 k0, k1;
-    k0.x = key_of(g0.x + e0.x); k0.y = key_of(g0.y + e0.y); k0.z = key_of(g0.z + e0.z); k0.w = key_of(g0.w + e0.w);
-    k1.x = key_of(g1.x + e1.x); k1.y = key_of(g1.y + e1.y); k1.z = key_of(g1.z + e1.z); k1.w = key_of(g1.w + e1.w);
+    const float4 p0 = accumulate(L.gamma, g0, e0), p1 = accumulate(L.gamma, g1, e1);
+    k0.x = key_of(p0.x); k0.y = key_of(p0.y); k0.z = key_of(p0.z); k0.w = key_of(p0.w);
+    k1.x = key_of(p1.x); k1.y = key_of(p1.y); k1.z = key_of(p1.z); k1.w = key_of(p1.w);
     uint4* out = reinterpret_cast<uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin + (size_t)c * 8u);
     out[0] = k0; out[1] = k1;
 }
@@ -300,6 +301,7 @@ topk_main_kernel(FastParams P) {
     uint32_t slot3 = 0;                                                // counter pair of the current tile
     uint32_t pend_item = 0xFFFFFFFFu, pend_slot = 0, pend_room = 0;    // tile whose counts are not written yet
     bool pend_accumulates = false;
+    const float gamma = L.gamma;
     const uint32_t group_step = (gridDim.x - 1u) * MAIN_GROUP + 1u;    // from a group's last tile to the next group's first
     for (uint32_t item = blockIdx.x * MAIN_GROUP, ig = 0; ;
          item += (ig + 1u == MAIN_GROUP ? group_step : 1u), ig = (ig + 1u == MAIN_GROUP ? 0u : ig + 1u)) {
@@ -356,7 +358,7 @@ topk_main_kernel(FastParams P) {
             }
 #pragma unroll
             for (int j = 0; j < QUADS; ++j) {
-                const float4 p = make_float4(gv[j].x + ev[j].x, gv[j].y + ev[j].y, gv[j].z + ev[j].z, gv[j].w + ev[j].w);
+                const float4 p = accumulate(gamma, gv[j], ev[j]);
                 *reinterpret_cast<float4*>(e + mine + 128 * j) = p;
                 *reinterpret_cast<float4*>(sp + off0 + 128 * j) = p;
                 flag16 |= ((uint32_t)(key_of(p.x) >= lo) | (uint32_t)(key_of(p.y) >= lo) << 1 |
@@ -371,7 +373,7 @@ topk_main_kernel(FastParams P) {
                 load_quad_stream(T.g, base, seg.n, gq);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    p[c] = gq[c] + p[c];
+                    p[c] = accumulate(gamma, gq[c], p[c]);
                     flag16 |= (((valid >> c) & 1u) & (uint32_t)(key_of(p[c]) >= lo)) << (4 * j + c);
                 }
                 if (valid) store_quad(e, base, valid, p);

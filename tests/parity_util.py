@@ -34,7 +34,7 @@ def segs_tuple(segs):
     return [(s.offset, s.n, s.k) if hasattr(s, "offset") else tuple(s) for s in segs]
 
 
-def run_step_both(ctx, scheme, grads_cpu, res_cpu, segs, seeds, check_status=True, use="step"):
+def run_step_both(ctx, scheme, grads_cpu, res_cpu, segs, seeds, check_status=True, use="step", gamma=1.0):
     """grads_cpu/res_cpu: [W, n] fp32 CPU tensors.  Runs one step on both sides,
     asserts bit equality of messages, residuals and the dense average, and
     returns the new residuals (CPU tensor) so that steps can be chained."""
@@ -47,6 +47,7 @@ def run_step_both(ctx, scheme, grads_cpu, res_cpu, segs, seeds, check_status=Tru
     vals = torch.full((W, max(K, 1)), float("nan"), device=dev)
     idx = torch.full((W, max(K, 1)), -1, device=dev, dtype=torch.int32)
     out = torch.full((n,), float("nan"), device=dev)
+    ctx.sc_set_gamma(gamma)
     if use == "step":
         ctx.sc_step(scheme, g, e, segs, seeds, vals, idx, out)
     elif use == "split":
@@ -56,12 +57,13 @@ def run_step_both(ctx, scheme, grads_cpu, res_cpu, segs, seeds, check_status=Tru
         h_out = torch.empty(n, dtype=torch.float32).pin_memory()
         ctx.sc_step_host(scheme, grads_cpu.contiguous().pin_memory(), e, segs, seeds, h_out)
         out = h_out
+    ctx.sc_set_gamma(1.0)
     if check_status:
         assert ctx.sc_sync_status() == 0
     torch.cuda.synchronize()
     gn = [grads_cpu[w].numpy() for w in range(W)]
     en = [res_cpu[w].numpy() for w in range(W)]
-    ov, oi, oe, oout = O.step(scheme, gn, en, segs, list(seeds))
+    ov, oi, oe, oout = O.step(scheme, gn, en, segs, list(seeds), gamma)
     for w in range(W):
         if use != "host":
             assert_bits_equal(idx[w, :K], oi[w], f"idx[w={w}]")

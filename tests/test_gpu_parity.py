@@ -10,7 +10,7 @@ from parity_util import assert_bits_equal, run_step_both
 
 pytestmark = pytest.mark.gpu
 
-SCHEMES = [sc.SC_TOPK, sc.SC_RANDK, sc.SC_RANDBLOCK]
+SCHEMES = [sc.SC_TOPK, sc.SC_RANDK, sc.SC_RANDBLOCK, sc.SC_RANDBLOCK_WRAP]
 TILE = 4096
 
 
@@ -264,6 +264,43 @@ def test_aggregate_private_coordinates_by_density(ctx, W, n, density, clumped):
     assert_bits_equal(out, O.aggregate(list(vals), list(idx), n), "aggregate by density")
     if own is not ctx:
         own.close()
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+@pytest.mark.parametrize("gamma", [0.1, -2.5, 3.0e-4])
+def test_step_size_is_one_fused_multiply_add(ctx, scheme, gamma):
+    """p = gamma g + e with a single rounding (Algorithm 1, accumulate line), on small and large
+    segments, over three steps so that the residual feeds back."""
+    W, n = 3, (1 << 17) + 4099
+    segs = [(0, 70_001, 701), (70_001, 5_000, 50), (75_001, n - 75_001, 4000)]
+    res = torch.zeros(W, n)
+    for t in range(3):
+        g = torch.stack([rand(n, 1000 * t + w, scale=1.0) for w in range(W)])
+        res = run_step_both(ctx, scheme, g, res, segs, [11 + t] * W, gamma=gamma)
+
+
+def test_step_size_halfway_cases(ctx):
+    """Inputs where rounding the product first would give another answer than the fused form."""
+    a = np.float32(1.0) + np.float32(2.0 ** -23)
+    n = 4096 + 64
+    g = torch.full((1, n), float(a))
+    e_vals = np.float32([2.0 ** -24, -(2.0 ** -24), 3 * 2.0 ** -24, 1.0, -1.0, 2.0 ** -47, 0.0, -0.0])
+    e = torch.from_numpy(np.resize(e_vals, n).copy()).view(1, n)
+    for scheme in SCHEMES:
+        run_step_both(ctx, scheme, g, e, [(0, n, 64)], [5], gamma=float(a))
+
+
+def test_wrap_block_that_wraps(ctx):
+    """Seeds are searched (on the CPU) until the block of the large and of a small segment wraps."""
+    W, n = 2, 200_000
+    segs = [(0, 150_000, 60_000), (150_000, 50_000, 49_999)]
+    seed = next(s for s in range(1000)
+                if O.block_start_wrap(O.segment_seed(s, 0), 150_000) + 60_000 > 150_000
+                and O.block_start_wrap(O.segment_seed(s, 1), 50_000) > 1)
+    g = torch.stack([rand(n, 77 + w) for w in range(W)])
+    res = torch.stack([rand(n, 99 + w, scale=1e-4) for w in range(W)])
+    run_step_both(ctx, sc.SC_RANDBLOCK_WRAP, g, res, segs, [seed] * W)
+    run_step_both(ctx, sc.SC_RANDBLOCK_WRAP, g, res, segs, [seed, seed + 1], use="split")
 
 
 def test_host_buffer_step(ctx):

@@ -70,3 +70,20 @@ def test_random_case(ctx, case):
     use = ["step", "split", "host"][int(rng.integers(0, 3))]
     e = run_step_both(ctx, scheme, g, e, segs, seeds, use=use)
     run_step_both(ctx, scheme, g, e, segs, [s + 1 for s in seeds], use="step")      # second step on the carried residual
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_case_wrap_block_and_step_size(ctx, case):
+    """The same generator of cases for the wrap-around block and for gamma != 1 (all schemes)."""
+    rng = np.random.default_rng(5000 + case)
+    scheme = [sc.SC_RANDBLOCK_WRAP, sc.SC_TOPK, sc.SC_RANDK, sc.SC_RANDBLOCK][case % 4] if case >= 4 else sc.SC_RANDBLOCK_WRAP
+    gamma = 1.0 if case < 4 else float(np.float32(10.0 ** rng.uniform(-3, 1) * (-1 if rng.random() < 0.3 else 1)))
+    segs, n = _table(rng, big=(case % 3 == 0))
+    W = int(rng.integers(1, 6))
+    g = torch.stack([_values(rng, n, int(rng.integers(0, 5))) for _ in range(W)])
+    e = torch.stack([_values(rng, n, int(rng.integers(0, 5))) * 0.1 for _ in range(W)])
+    shared = rng.random() < 0.5
+    seeds = [int(rng.integers(0, 2 ** 62))] * W if shared else [int(x) for x in rng.integers(0, 2 ** 62, W)]
+    use = ["step", "split", "host"][int(rng.integers(0, 3))]
+    e = run_step_both(ctx, scheme, g, e, segs, seeds, use=use, gamma=gamma)
+    run_step_both(ctx, scheme, g, e, segs, [s + 1 for s in seeds], use="step", gamma=gamma)
