@@ -308,11 +308,29 @@ inline uint32_t persistent_grid(const sc_ctx* c, int occ, uint64_t items) {
 // Compression of rows [0, W) of the given base pointers.  `mask_ready` tells the
 // random-k path that the membership mask of seed group 0 is already built (used
 // when one shared-seed step is issued worker by worker).
+// Exclusive scan of `rows` rows of `len` counts: clusters of ROW_SCAN_CTAS CTAs for long rows.
+int launch_row_scan(uint32_t* data, uint32_t rows, uint32_t len, cudaStream_t stream) {
+    if (rows == 0) return SC_OK;
+    if (len < 8192u) {
+        row_scan_kernel<1><<<rows, THREADS, 0, stream>>>(data, len);
+        return SC_OK;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(rows * ROW_SCAN_CTAS); cfg.blockDim = dim3(THREADS); cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = ROW_SCAN_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    SC_CUDA(cudaLaunchKernelEx(&cfg, row_scan_kernel<ROW_SCAN_CTAS>, data, len));
+    return SC_OK;
+}
+
 int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
                   const uint64_t* h_seeds, bool shared_seeds, bool mask_ready,
                   float* out_vals, uint32_t* out_idx, cudaStream_t stream) {
     Layout L = c->layout;
     L.gamma = c->gamma;
+    int rc_scan = SC_OK;
     if (n == 0 || L.tiles_per_worker == 0) return SC_OK;
     const uint64_t items64 = (uint64_t)W * L.tiles_per_worker;
     if (items64 > 0xFFFFFFF0ull) return SC_ERR_RANGE;
@@ -364,7 +382,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             { Launch l(c, KIND_TILECOUNT, stream);
               topk_tilecount_kernel<<<(uint32_t)(((uint64_t)items * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_ROW_SCAN, stream);
-              row_scan_kernel<<<W, THREADS, 0, stream>>>(c->d_offsets, L.tiles_per_worker); }
+              if ((rc_scan = launch_row_scan(c->d_offsets, (uint32_t)W, L.tiles_per_worker, stream)) != SC_OK) return rc_scan; }
             { Launch l(c, KIND_EMIT, stream);
               // flagged entries per tile, on average (the list holds the kept elements and a few per cent more)
               const double per_tile = 1.05 * (double)L.K_total * TILE / (double)std::max<size_t>(L.n_total, 1);
@@ -436,7 +454,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               mask_count_kernel<<<(uint32_t)((warps + WARPS - 1) / WARPS), THREADS, 0, stream>>>(
                   L, c->d_mask, groups, c->d_offsets); }
             { Launch l(c, KIND_ROW_SCAN, stream);
-              row_scan_kernel<<<groups, THREADS, 0, stream>>>(c->d_offsets, L.tiles_per_worker); }
+              if ((rc_scan = launch_row_scan(c->d_offsets, groups, L.tiles_per_worker, stream)) != SC_OK) return rc_scan; }
         }
         { Launch l(c, KIND_RANDK_PACK, stream);
           randk_pack_kernel<<<persistent_grid(c, c->occ_pack_mask, (items + STREAM_GROUP - 1) / STREAM_GROUP), THREADS, 0, stream>>>(

