@@ -373,14 +373,14 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             { Launch l(c, KIND_CANDBIN, stream);
               topk_candbin_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDFILTER, stream);
-              topk_candfilter_kernel<<<(uint32_t)(((uint64_t)items * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
+              topk_candfilter_kernel<<<(uint32_t)(((uint64_t)(items + TILES_PER_GROUP - 1) / TILES_PER_GROUP * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_FINAL, stream);
               topk_final_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_RESTORE, stream);
               const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
               topk_restore_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_TILECOUNT, stream);
-              topk_tilecount_kernel<<<(uint32_t)(((uint64_t)items * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
+              topk_tilecount_kernel<<<(uint32_t)(((uint64_t)(items + TILES_PER_GROUP - 1) / TILES_PER_GROUP * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_ROW_SCAN, stream);
               if ((rc_scan = launch_row_scan(c->d_offsets, (uint32_t)W, L.tiles_per_worker, stream)) != SC_OK) return rc_scan; }
             { Launch l(c, KIND_EMIT, stream);

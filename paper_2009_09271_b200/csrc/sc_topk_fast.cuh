@@ -528,31 +528,67 @@ topk_candbin_kernel(FastParams P) {
     }
 }
 
-// ---- filter: copy the candidates of the threshold's bin into the short list (8 lanes per tile) -------
+// ---- per-tile walks over the candidate slices ----------------------------------------------------
+// Eight lanes share TILES_PER_GROUP consecutive tiles.  The kernels below are bound by a chain of
+// dependent loads (slice length and base, then the slice), so a group first requests the placement
+// words of all its tiles, then the first eight candidates of every tile, and only then looks at
+// them: four tiles per group cut the number of such chains per launch by four.
+constexpr uint32_t TILES_PER_GROUP = 4;
+struct CandSlice {                 // one tile's slice as seen by a lane of its group
+    const uint2* list;             // nullptr: nothing to do for this tile
+    uint32_t cnt, prob, w, lt;
+    uint2 first;                   // entry `sub` of the slice (if sub < cnt)
+};
+template <bool NEED_FILTER>
+__device__ inline void cand_slices(const FastParams& P, uint32_t item0, uint32_t sub, CandSlice (&t)[TILES_PER_GROUP]) {
+    const Layout& L = P.L;
+    uint32_t base[TILES_PER_GROUP];
+#pragma unroll
+    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+        const uint32_t item = item0 + u;
+        t[u].list = nullptr; t[u].cnt = 0; base[u] = 0;
+        if (item < P.total_items) { t[u].cnt = __ldg(P.tile_ccnt + item); base[u] = __ldg(P.tile_cbase + item); }
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+        const uint32_t item = item0 + u;
+        t[u].first = make_uint2(0u, 0u);
+        if (item >= P.total_items) continue;
+        t[u].w = item / L.tiles_per_worker;
+        t[u].lt = item - t[u].w * L.tiles_per_worker;
+        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, t[u].lt);
+        const SegEntry& seg = L.segs[s];
+        t[u].prob = t[u].w * L.nseg + s;
+        if (!seg.fast) { t[u].cnt = 0; continue; }
+        const FastState* st = P.state + t[u].prob;
+        if (st->path != PATH_FAST || (NEED_FILTER && st->need2 == 0)) { t[u].cnt = 0; continue; }
+        t[u].list = P.cand + (size_t)t[u].w * L.cand_per_worker + seg.cand_begin + base[u];
+        if (sub < t[u].cnt) t[u].first = __ldg(t[u].list + sub);
+    }
+}
+
+// ---- filter: copy the candidates of the threshold's bin into the short list ----------------------
 __global__ void __launch_bounds__(THREADS)
 topk_candfilter_kernel(FastParams P) {
     const Layout& L = P.L;
     const uint32_t sub = threadIdx.x & 7u;
-    const uint32_t item = (blockIdx.x * THREADS + threadIdx.x) >> 3;
-    if (item >= P.total_items) return;
-    const uint32_t cnt = P.tile_ccnt[item];
-    if (cnt == 0u) return;
-    const uint32_t w = item / L.tiles_per_worker;
-    const uint32_t lt = item - w * L.tiles_per_worker;
-    const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-    const SegEntry seg = L.segs[s];
-    if (!seg.fast) return;
-    const size_t prob = (size_t)w * L.nseg + s;
-    const FastState* stp = P.state + prob;
-    if (stp->path != PATH_FAST || stp->need2 == 0) return;
-    const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
-    const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + P.tile_cbase[item];
-    uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
-    for (uint32_t i = sub; i < cnt; i += 8) {
-        const uint2 c = list[i];
-        if (c.x >= lo2 && c.x <= hi2) {
-            const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
-            if (pos < LIST2_CAP) out[pos] = c;
+    const uint32_t item0 = ((blockIdx.x * THREADS + threadIdx.x) >> 3) * TILES_PER_GROUP;
+    if (item0 >= P.total_items) return;
+    CandSlice t[TILES_PER_GROUP];
+    cand_slices<true>(P, item0, sub, t);
+#pragma unroll
+    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+        if (!t[u].list || t[u].cnt == 0u) continue;
+        const FastState* stp = P.state + t[u].prob;
+        const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
+        const uint32_t s = t[u].prob - t[u].w * L.nseg;
+        uint2* out = P.list2 + ((size_t)t[u].w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
+        for (uint32_t i = sub; i < t[u].cnt; i += 8) {
+            const uint2 c = i == sub ? t[u].first : t[u].list[i];
+            if (c.x >= lo2 && c.x <= hi2) {
+                const uint32_t pos = atomicAdd(&P.state[t[u].prob].cnt2, 1u);
+                if (pos < LIST2_CAP) out[pos] = c;
+            }
         }
     }
 }
@@ -607,37 +643,36 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
     return key > T || (key == T && coord < icut);
 }
 
-// ---- kept count per tile = sure elements + chosen candidates (8 lanes per tile) -----------------
+// ---- kept count per tile = sure elements + chosen candidates -------------------------------------
 __global__ void __launch_bounds__(THREADS)
 topk_tilecount_kernel(FastParams P) {
     const Layout& L = P.L;
     const uint32_t sub = threadIdx.x & 7u;
-    const uint32_t item = (blockIdx.x * THREADS + threadIdx.x) >> 3;
-    const bool live = item < P.total_items;
-    uint32_t kept = 0, w = 0, lt = 0;
-    if (live) {
-        w = item / L.tiles_per_worker;
-        lt = item - w * L.tiles_per_worker;
-        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-        const SegEntry seg = L.segs[s];
-        if (seg.fast) {
-            const FastState* st = P.state + (size_t)w * L.nseg + s;
-            if (st->path == PATH_FAST) {
-                const uint32_t T = st->T, icut = st->icut;
-                const uint32_t base = P.tile_cbase[item], cnt = P.tile_ccnt[item];
-                const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + base;
-                for (uint32_t i = sub; i < cnt; i += 8) {
-                    const uint2 c = list[i];
-                    kept += fast_kept(c.x, c.y, T, icut) ? 1u : 0u;
-                }
-                if (sub == 0) kept += P.tile_sure[item];
+    const uint32_t item0 = ((blockIdx.x * THREADS + threadIdx.x) >> 3) * TILES_PER_GROUP;
+    CandSlice t[TILES_PER_GROUP];
+    uint32_t sure[TILES_PER_GROUP];
+#pragma unroll
+    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u)
+        sure[u] = (sub == 0u && item0 + u < P.total_items) ? __ldg(P.tile_sure + item0 + u) : 0u;
+    cand_slices<false>(P, item0, sub, t);
+#pragma unroll
+    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+        uint32_t kept = 0;
+        if (t[u].list) {                                               // a tile of a segment on the one-pass path
+            const FastState* st = P.state + t[u].prob;
+            const uint32_t T = st->T, icut = st->icut;
+            for (uint32_t i = sub; i < t[u].cnt; i += 8) {
+                const uint2 c = i == sub ? t[u].first : t[u].list[i];
+                kept += fast_kept(c.x, c.y, T, icut) ? 1u : 0u;
             }
+            kept += sure[u];
         }
+        kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 1);
+        kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 2);
+        kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 4);
+        if (sub == 0u && item0 + u < P.total_items)
+            P.offsets[(size_t)t[u].w * (L.tiles_per_worker + 1) + t[u].lt] = kept;
     }
-    kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 1);
-    kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 2);
-    kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 4);
-    if (live && sub == 0) P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
 }
 
 // ---- emit: G lanes per tile walk the tile's slice of the flagged list ----------------------------

@@ -165,6 +165,35 @@ def test_topk_large_segment_all_densities(ctx, n):
         assert ctx.sc_topk_path_counts() == (0, 1, 0), k       # continuous values: the one-pass path serves it
 
 
+def test_topk_sample_large_enough_for_the_cluster_bracket(ctx):
+    """From 2^15 sample keys up the bracket kernel runs as a cluster of CTAs; the sample grows with the kept
+    fraction, so a quarter or a half kept on a million elements takes that path (and one per cent does not)."""
+    n = (1 << 20) + 13
+    W = 3
+    g = torch.stack([rand(n, 21 + w) for w in range(W)])
+    e = torch.stack([rand(n, 31 + w, scale=1e-4) for w in range(W)])
+    for k in (n // 100, n // 4, n // 2):
+        run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, k)], [3] * W)
+        assert ctx.sc_topk_path_counts() == (0, W, 0), k
+    # both kinds of sample in one call: a large and a small segment side by side
+    segs = [(0, 900_000, 300_000), (900_000, n - 900_000, 1000)]
+    run_step_both(ctx, sc.SC_TOPK, g, e, segs, [4] * W)
+    assert ctx.sc_topk_path_counts() == (0, 2 * W, 0)
+
+
+def test_row_of_more_than_8192_tiles():
+    """Rows of 8192 tiles and more have their per-tile counts scanned by a cluster of CTAs."""
+    n = 8200 * 4096 + 77
+    own = sc.Context(max_n=n, max_W=1, max_segments=2)
+    gen = torch.Generator().manual_seed(5)
+    g = (torch.randn(n, generator=gen) * 1e-3).view(1, n)
+    e = torch.zeros(1, n)
+    for scheme in (sc.SC_TOPK, sc.SC_RANDK):
+        run_step_both(own, scheme, g, e, [(0, n, n // 1000)], [8])
+    run_step_both(own, sc.SC_RANDK, g, e, [(0, 20_000_003, 20_000), (20_000_003, n - 20_000_003, 5)], [9])
+    own.close()
+
+
 def test_topk_large_segment_misaligned_rows_and_mixed_table(ctx):
     W, n = 3, BIG + 4099                       # odd row length: rows 1, 2 start misaligned
     g = torch.stack([rand(n, 900 + w) for w in range(W)])
