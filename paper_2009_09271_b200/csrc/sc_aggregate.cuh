@@ -146,24 +146,25 @@ constexpr uint32_t AWARP = 1024;                 // coordinates per warp
 constexpr uint32_t AWARP_BATCH = 8;              // workers whose slices are fetched together
 constexpr uint32_t AWARP_MAX_SLICE = 64;         // entries of one worker in one 4096-tile served by the fast loop
 
+template <uint32_t AW>
 __global__ void __launch_bounds__(THREADS)
 agg_warp_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
                 const uint32_t* __restrict__ bounds /* at ATILE granularity */, uint32_t W, uint32_t K, uint32_t n,
                 uint32_t ntiles, float* __restrict__ out, int* __restrict__ status) {
-    __shared__ __align__(16) float acc_all[WARPS][AWARP];
+    extern __shared__ __align__(16) float acc_dyn[];                   // WARPS x AW floats
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    float* acc = acc_all[warp];
+    float* acc = acc_dyn + warp * AW;
     const float fW = (float)W;
     const bool pow2 = (W & (W - 1u)) == 0u;
     const float rW = 1.0f / fW;
-    const uint32_t nq = (n + AWARP - 1) / AWARP;                       // quarter-tiles
+    const uint32_t nq = (n + AW - 1) / AW;                             // warp-owned parts of a tile
     const uint32_t warps_total = gridDim.x * WARPS;
     for (uint32_t q = blockIdx.x * WARPS + warp; q < nq; q += warps_total) {
-        const uint32_t t = q / (ATILE / AWARP);                          // enclosing tile of the bounds table
-        const uint32_t base = q * AWARP;
-        const uint32_t cnt_here = min(AWARP, n - base);
+        const uint32_t t = q / (ATILE / AW);                             // enclosing tile of the bounds table
+        const uint32_t base = q * AW;
+        const uint32_t cnt_here = min(AW, n - base);
 #pragma unroll
-        for (int i = 0; i < (int)(AWARP / 128); ++i)
+        for (int i = 0; i < (int)(AW / 128); ++i)
             reinterpret_cast<float4*>(acc)[i * 32 + lane] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         __syncwarp();
         for (uint32_t w0 = 0; w0 < W; w0 += AWARP_BATCH) {
@@ -206,9 +207,9 @@ agg_warp_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx
             }
         }
         float* o = out + base;
-        if (cnt_here == AWARP) {
+        if (cnt_here == AW) {
 #pragma unroll
-            for (int i = 0; i < (int)(AWARP / 128); ++i) {
+            for (int i = 0; i < (int)(AW / 128); ++i) {
                 float4 a = reinterpret_cast<const float4*>(acc)[i * 32 + lane];
                 if (pow2) { a.x *= rW; a.y *= rW; a.z *= rW; a.w *= rW; }
                 else { a.x = a.x / fW; a.y = a.y / fW; a.z = a.z / fW; a.w = a.w / fW; }
@@ -231,26 +232,26 @@ agg_warp_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx
 // the batch at once).  Then H rounds of 32 entries per worker are fetched for B workers together
 // and added in worker order; what exceeds 32 H entries is finished before the next worker.
 // ---------------------------------------------------------------------------------------------
-template <int H, int B>
+template <int H, int B, uint32_t AW>
 __global__ void __launch_bounds__(THREADS)
 agg_warp_fine_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx,
                      const uint32_t* __restrict__ bounds /* at ATILE granularity */, uint32_t W, uint32_t K, uint32_t n,
                      uint32_t ntiles, float* __restrict__ out, int* __restrict__ status) {
     static_assert(B <= 16, "a batch lies inside one group of 16 workers");
-    __shared__ __align__(16) float acc_all[WARPS][AWARP];
+    extern __shared__ __align__(16) float acc_dyn[];                   // WARPS x AW floats
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    float* acc = acc_all[warp];
+    float* acc = acc_dyn + warp * AW;
     const float fW = (float)W;
     const bool pow2 = (W & (W - 1u)) == 0u;
     const float rW = 1.0f / fW;
-    const uint32_t nq = (n + AWARP - 1) / AWARP;
+    const uint32_t nq = (n + AW - 1) / AW;
     const uint32_t warps_total = gridDim.x * WARPS;
     for (uint32_t q = blockIdx.x * WARPS + warp; q < nq; q += warps_total) {
-        const uint32_t t = q / (ATILE / AWARP);
-        const uint32_t base = q * AWARP;
-        const uint32_t cnt_here = min(AWARP, n - base);
+        const uint32_t t = q / (ATILE / AW);
+        const uint32_t base = q * AW;
+        const uint32_t cnt_here = min(AW, n - base);
 #pragma unroll
-        for (int i = 0; i < (int)(AWARP / 128); ++i)
+        for (int i = 0; i < (int)(AW / 128); ++i)
             reinterpret_cast<float4*>(acc)[i * 32 + lane] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         __syncwarp();
         for (uint32_t g0 = 0; g0 < W; g0 += 16) {
@@ -263,11 +264,11 @@ agg_warp_fine_kernel(const float* __restrict__ vals, const uint32_t* __restrict_
             if (g0 + u < W) {
                 const uint32_t* b = bounds + (size_t)(g0 + u) * (ntiles + 1) + t;
                 uint32_t a = __ldg(b), e = __ldg(b + 1);
-                const uint32_t target = base + (upper ? AWARP : 0u);
+                const uint32_t target = base + (upper ? AW : 0u);
                 const uint32_t* row = idx + (size_t)(g0 + u) * K;
-                const uint32_t qi = q % (ATILE / AWARP);
+                const uint32_t qi = q % (ATILE / AW);
                 if (!upper && qi == 0) e = a;                             // the tile's own first coordinate
-                else if (upper && qi == ATILE / AWARP - 1) a = e;         // the tile's end
+                else if (upper && qi == ATILE / AW - 1) a = e;         // the tile's end
                 while (a < e) {
                     const uint32_t len = e - a;
                     uint32_t c = 0;
@@ -322,9 +323,9 @@ agg_warp_fine_kernel(const float* __restrict__ vals, const uint32_t* __restrict_
         }
         }
         float* o = out + base;
-        if (cnt_here == AWARP) {
+        if (cnt_here == AW) {
 #pragma unroll
-            for (int i = 0; i < (int)(AWARP / 128); ++i) {
+            for (int i = 0; i < (int)(AW / 128); ++i) {
                 float4 a = reinterpret_cast<const float4*>(acc)[i * 32 + lane];
                 if (pow2) { a.x *= rW; a.y *= rW; a.z *= rW; a.w *= rW; }
                 else { a.x = a.x / fW; a.y = a.y / fW; a.z = a.z / fW; a.w = a.w / fW; }

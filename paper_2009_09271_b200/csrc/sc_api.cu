@@ -73,7 +73,7 @@ struct sc_ctx {
     uint64_t launches = 0;
 
     int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1, occ_agg_big = 1, occ_agg_warp = 1;
-    int occ_agg_fine[3] = {1, 1, 1};
+    int occ_agg_fine[5] = {1, 1, 1, 1, 1};
 
     // optional per-kernel timing (sc_profile)
     bool prof_on = false;
@@ -501,6 +501,12 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
 #define AGG_FINE_Q2 200.0
 #endif
 
+// Coordinates owned by one warp of agg_warp_kernel (a part of a 4096-tile).
+#ifndef SC_AGG_WARP_PART
+#define SC_AGG_WARP_PART 2048
+#endif
+constexpr uint32_t AGG_WARP_PART = SC_AGG_WARP_PART;
+
 inline uint32_t aggregate_tile(int W, size_t k, size_t n) {
     const double per_big_tile = (double)ATILE_BIG * (double)W * (double)k / (double)std::max<size_t>(n, 1);
     return per_big_tile <= 0.9 * AGG_STAGE ? ATILE_BIG : ATILE;
@@ -512,11 +518,12 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
     // sparse messages with private coordinates: warp-owned quarter tiles (slices of ~k/n*4096 entries)
     const double slice = (double)k * ATILE / (double)std::max<size_t>(n, 1);       // entries of one worker per 4096-tile
     const bool by_warp = !shared_idx && slice >= 8.0 && slice <= 0.75 * AWARP_MAX_SLICE;
-    // denser private coordinates: the same ownership with per-quarter boundaries; H rounds of 32 entries per
-    // worker cover the expected quarter slice with a 30 % margin
-    const double qslice = slice / (ATILE / AWARP);
+    // denser private coordinates: the same ownership with boundaries per warp-owned part; a part is half a tile
+    // while H rounds of 32 entries per worker cover its expected slice, a quarter beyond
+    const double half = slice / 2.0, quarter = slice / 4.0;
     const int fine = (shared_idx || by_warp || slice < 8.0) ? -1
-                     : qslice <= AGG_FINE_Q0 ? 0 : qslice <= AGG_FINE_Q1 ? 1 : qslice <= AGG_FINE_Q2 ? 2 : -1;
+                     : half <= AGG_FINE_Q0 ? 0 : half <= AGG_FINE_Q1 ? 1 : half <= 150.0 ? 2
+                     : quarter <= AGG_FINE_Q1 ? 3 : quarter <= AGG_FINE_Q2 ? 4 : -1;
     const uint32_t tile = (by_warp || fine >= 0) ? ATILE : aggregate_tile(shared_idx ? 1 : W, k, n);
     const uint32_t ntiles = (uint32_t)((n + tile - 1) / tile);
     const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
@@ -525,21 +532,26 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
       agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
           idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds); }
     { Launch l(c, KIND_AGG_TILES, stream);
-      const uint64_t nq = (n + AWARP - 1) / AWARP;
       if (by_warp) {
-          agg_warp_kernel<<<persistent_grid(c, c->occ_agg_warp, (nq + WARPS - 1) / WARPS), THREADS, 0, stream>>>(
+          const uint64_t nparts = (n + AGG_WARP_PART - 1) / AGG_WARP_PART;
+          agg_warp_kernel<AGG_WARP_PART><<<persistent_grid(c, c->occ_agg_warp, (nparts + WARPS - 1) / WARPS), THREADS,
+                                           WARPS * AGG_WARP_PART * sizeof(float), stream>>>(
               vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
       } else if (fine >= 0) {
-          const uint32_t grid = persistent_grid(c, c->occ_agg_fine[fine], (nq + WARPS - 1) / WARPS);
-          if (fine == 0)
-              agg_warp_fine_kernel<2, 8><<<grid, THREADS, 0, stream>>>(
-                  vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
-          else if (fine == 1)
-              agg_warp_fine_kernel<4, 4><<<grid, THREADS, 0, stream>>>(
-                  vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
-          else
-              agg_warp_fine_kernel<6, 3><<<grid, THREADS, 0, stream>>>(
-                  vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status);
+          const uint32_t part = fine <= 2 ? 2048u : 1024u;
+          const uint64_t nparts = (n + part - 1) / part;
+          const uint32_t grid = persistent_grid(c, c->occ_agg_fine[fine], (nparts + WARPS - 1) / WARPS);
+          const size_t smem = WARPS * part * sizeof(float);
+#define SC_FINE_LAUNCH(H, B, AW) agg_warp_fine_kernel<H, B, AW><<<grid, THREADS, smem, stream>>>( \
+              vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, out, c->d_status)
+          switch (fine) {
+              case 0: SC_FINE_LAUNCH(2, 8, 2048); break;
+              case 1: SC_FINE_LAUNCH(4, 4, 2048); break;
+              case 2: SC_FINE_LAUNCH(6, 3, 2048); break;
+              case 3: SC_FINE_LAUNCH(4, 4, 1024); break;
+              default: SC_FINE_LAUNCH(6, 3, 1024); break;
+          }
+#undef SC_FINE_LAUNCH
       } else {
           const uint32_t grid = persistent_grid(c, tile == ATILE_BIG ? c->occ_agg_big : c->occ_agg, ntiles);
           if (tile == ATILE_BIG)
@@ -648,10 +660,20 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_block, randblock_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel<ATILE>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_big, agg_tiles_kernel<ATILE_BIG>, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_warp, agg_warp_kernel, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_fine[0], agg_warp_fine_kernel<2, 8>, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_fine[1], agg_warp_fine_kernel<4, 4>, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_fine[2], agg_warp_fine_kernel<6, 3>, THREADS, 0);
+        cudaFuncSetAttribute(agg_warp_kernel<AGG_WARP_PART>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(WARPS * AGG_WARP_PART * sizeof(float)));
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_warp, agg_warp_kernel<AGG_WARP_PART>, THREADS,
+                                                      WARPS * AGG_WARP_PART * sizeof(float));
+        {
+#define SC_FINE_SETUP(I, H, B, AW)                                                                                         \
+    cudaFuncSetAttribute(agg_warp_fine_kernel<H, B, AW>, cudaFuncAttributeMaxDynamicSharedMemorySize,                      \
+                         (int)(WARPS * AW * sizeof(float)));                                                               \
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg_fine[I], agg_warp_fine_kernel<H, B, AW>, THREADS,           \
+                                                  WARPS * AW * sizeof(float))
+            SC_FINE_SETUP(0, 2, 8, 2048); SC_FINE_SETUP(1, 4, 4, 2048); SC_FINE_SETUP(2, 6, 3, 2048);
+            SC_FINE_SETUP(3, 4, 4, 1024); SC_FINE_SETUP(4, 6, 3, 1024);
+#undef SC_FINE_SETUP
+        }
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
         c->max_main_grid = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
     }
