@@ -304,28 +304,44 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     sampler = ClockSampler(str(torch.cuda.get_device_properties(dev).uuid))
     if not sampler.uuid.startswith("GPU-"):
         sampler.uuid = "GPU-" + sampler.uuid
-    barrier()
-    if rank == 0:
-        sampler.start()
-    ctx.sc_profile(not args.no_kernel_events)
-    launches0 = ctx.launch_count
-    marks = []
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    start.record()
-    for t in range(args.steps):
-        one_step(args.warmup + t, marks)
-    end.record()
-    barrier()
-    elapsed_ms = start.elapsed_time(end)
-    launches = ctx.launch_count - launches0
-    prof = ctx.sc_profile_read()
-    ctx.sc_profile(False)
-    clocks = sampler.stop() if rank == 0 else {}
-    status = ctx.sc_sync_status()
-    if status != 0:
-        raise RuntimeError(f"device status after the timed region: {sc.strerror(status)}")
-    elapsed_ms = ranks.max_ms(elapsed_ms)
+    # The timed region.  A measurement taken while the GPU reported a hardware or thermal slowdown, or with
+    # the SM clock far below its maximum for no stated reason, is thrown away and taken once more (every rank
+    # repeats, so that the collective calls stay matched); sw_power_cap is kept and reported.
+    remeasured = False
+    for attempt in range(2):
+        barrier()
+        if rank == 0:
+            sampler.start()
+        ctx.sc_profile(not args.no_kernel_events)
+        launches0 = ctx.launch_count
+        marks = []
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        start.record()
+        for t in range(args.steps):
+            one_step(args.warmup + t, marks)
+        end.record()
+        barrier()
+        elapsed_ms = start.elapsed_time(end)
+        launches = ctx.launch_count - launches0
+        prof = ctx.sc_profile_read()
+        ctx.sc_profile(False)
+        clocks = sampler.stop() if rank == 0 else {}
+        status = ctx.sc_sync_status()
+        if status != 0:
+            raise RuntimeError(f"device status after the timed region: {sc.strerror(status)}")
+        elapsed_ms = ranks.max_ms(elapsed_ms)
+        bad = 0.0
+        if rank == 0 and clocks.get("samples"):
+            slow = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(clocks["reasons"])
+            stuck = (not clocks["reasons"]) and clocks["sm_mhz"] < 0.8 * clocks["sm_max_mhz"]
+            bad = 1.0 if (slow or stuck) else 0.0
+        bad = ranks.max_ms(bad)                               # rank 0 decides for everyone
+        if bad == 0.0 or attempt == 1:
+            break
+        remeasured = True
+    if rank == 0 and clocks:
+        clocks["remeasured"] = remeasured
 
     # per-scheme device time from the marks
     per_scheme_ms = {s: 0.0 for s in schemes}
