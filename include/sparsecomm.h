@@ -94,7 +94,7 @@ int sc_profile_kinds(void);
 const char* sc_profile_name(int kind);
 int sc_profile_read(sc_ctx* ctx, double* h_ms, uint64_t* h_launches);
 
-/* Instrumentation (no counterpart in the paper).  Top-k of a segment of 2^20 or
+/* Instrumentation (no counterpart in the paper).  Top-k of a segment of 65,536 or
  * more elements first tries a one-pass path whose work depends on a sampled
  * bracket of the threshold; if the exact counts show the bracket missed, it redoes
  * the selection with a multi-pass radix select.  Both give the same bits.  After
@@ -105,7 +105,7 @@ int sc_topk_path_counts(sc_ctx* ctx, void* stream, uint32_t* h_counts);
 
 /* Algorithm 1, accumulate + compress + residual lines, one worker, global scope.
  * grad[n] read-only; residual[n] in/out (reads e, writes e'); out_vals[k],
- * out_idx[k] written.  k == 0 is allowed (residual <- g + e). */
+ * out_idx[k] written.  k == 0 is allowed (residual <- gamma g + e, see sc_set_gamma). */
 int sc_compress(sc_ctx* ctx, int scheme, const float* grad, float* residual, size_t n, size_t k,
                 uint64_t seed, float* out_vals, uint32_t* out_idx, void* stream);
 
