@@ -16,7 +16,7 @@ from parity_util import assert_bits_equal, run_step_both
 
 pytestmark = pytest.mark.gpu
 
-CODES = {"topk": sc.SC_TOPK, "randk": sc.SC_RANDK, "randblock": sc.SC_RANDBLOCK}
+CODES = {"topk": sc.SC_TOPK, "randk": sc.SC_RANDK, "randblock": sc.SC_RANDBLOCK, "randblock_wrap": sc.SC_RANDBLOCK_WRAP}
 
 
 def _noise(n, seed, scale):
@@ -77,7 +77,7 @@ def test_c4_lstm_shape_randblock_and_topk_one_percent_full():
 
 
 @pytest.mark.parametrize("scheme,density", [("topk", (1, 100)), ("randk", (1, 100)), ("randblock", (1, 100)),
-                                            ("topk", (1, 10000))])
+                                            ("topk", (1, 10000)), ("topk", (1, 10)), ("randblock_wrap", (1, 100))])
 def test_c5_full_size_in_the_benchmark_configuration(scheme, density):
     """n = 350,000,000, W = 16 in one sc_step call, as bench.py launches it."""
     w = wl.workload("c5")
