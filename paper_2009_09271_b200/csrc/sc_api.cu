@@ -15,6 +15,7 @@
 #include "sc_random.cuh"
 #include "sc_topk.cuh"
 #include "sc_topk_fast.cuh"
+#include "sc_topk_tiny.cuh"
 
 using namespace sc;
 
@@ -30,6 +31,9 @@ struct sc_ctx {
 
     SegEntry* d_segs = nullptr;
     uint32_t* d_fast_list = nullptr;
+    uint32_t* d_tiny_list = nullptr;      // [max_segments]: short segments, the <= TINY_SMALL_MAX ones first
+    uint32_t tiny_small = 0, tiny_large = 0, tiny_large_max_n = 0;
+    int occ_tiny_small = 1;
     uint32_t* d_lists = nullptr;     // slow tiles | fast tiles | slow pack groups | fast pack groups (each max_tiles long)
     uint32_t n_slow_tiles = 0, n_fast_tiles = 0, n_slow_groups = 0, n_fast_groups = 0;
     uint32_t* d_hist = nullptr;
@@ -92,6 +96,12 @@ struct sc_ctx {
     std::vector<cudaEvent_t> ev_worker;
 };
 
+// Top-k of segments below FAST_MIN_N elements runs with the segment in shared memory: one CTA per (worker,
+// segment) up to TINY_SMALL_MAX elements (the many very short tensors of a network keep several CTAs per SM),
+// a cluster of TINY_CTAS CTAs beyond.
+constexpr uint32_t TINY_SMALL_MAX = 4096;        // elements: 16 KB of shared memory
+constexpr uint32_t TINY_LARGE_MAX = FAST_MIN_N - 1;
+
 // Emit variants by the average number of flagged entries per tile: 8 or 16 lanes per tile for sparse slices
 // (4 or 2 tiles per warp side by side), the whole warp with 4 or 8 entries per lane for longer ones.
 constexpr double EMIT_MAX_8 = 12.0, EMIT_MAX_16 = 80.0, EMIT_MAX_32 = 200.0;
@@ -125,12 +135,12 @@ class DeviceGuard {
 
 enum { KIND_HIST0 = 0, KIND_RESOLVE, KIND_REFINE, KIND_PACK_TOPK, KIND_SCATTER, KIND_MASK_COUNT, KIND_ROW_SCAN,
        KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES, KIND_SAMPLE, KIND_BRACKET, KIND_MAIN,
-       KIND_CANDBIN, KIND_CANDFILTER, KIND_FINAL, KIND_TILECOUNT, KIND_EMIT, KIND_RESTORE, KIND_AGG_APPLY, KIND_COUNT };
+       KIND_CANDBIN, KIND_CANDFILTER, KIND_FINAL, KIND_TILECOUNT, KIND_EMIT, KIND_RESTORE, KIND_AGG_APPLY, KIND_TINY, KIND_COUNT };
 const char* const kKindNames[KIND_COUNT] = {"topk_hist0", "topk_resolve", "topk_refine", "pack_topk", "randk_scatter",
                                             "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
                                             "agg_tiles", "topk_sample", "topk_bracket", "topk_main", "topk_candbin",
                                             "topk_candfilter", "topk_final", "topk_tilecount", "topk_emit", "topk_restore",
-                                            "agg_apply"};
+                                            "agg_apply", "topk_tiny"};
 
 // Counts a kernel launch and, when profiling is on, brackets it with two events.
 class Launch {
@@ -166,7 +176,8 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         std::memcmp(c->cached_segs.data(), segs, sizeof(sc_segment) * nseg) == 0)
         return SC_OK;
     std::vector<SegEntry> h(nseg + 1);
-    std::vector<uint32_t> fast_list, lists[4];
+    std::vector<uint32_t> fast_list, lists[4], tiny_a, tiny_b;
+    uint32_t tiny_max_n = 0;
     uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0, cand = 0, flag = 0, smp = 0;
     uint32_t fast_count = 0, slow_count = 0, max_m = 0, max_cap = 0;
     for (int s = 0; s < nseg; ++s) {
@@ -214,13 +225,17 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             cand += cand_region * regions;
             flag += flag_region * regions;
             max_m = std::max(max_m, e.sample_m);
+        } else if (g.n <= TINY_LARGE_MAX) {
+            (g.n <= TINY_SMALL_MAX ? tiny_a : tiny_b).push_back((uint32_t)s);
+            tiny_max_n = std::max<uint32_t>(tiny_max_n, g.n <= TINY_SMALL_MAX ? 0u : (uint32_t)g.n);
         } else {
             ++slow_count;
         }
         h[s] = e;
         const int which = e.fast ? 1 : 0;
-        for (uint64_t t = 0; t < seg_tiles; ++t) lists[which].push_back((uint32_t)(tiles + t));
-        for (uint64_t t = 0; t < (seg_tiles + PACK_GROUP - 1) / PACK_GROUP; ++t) lists[2 + which].push_back((uint32_t)(groups + t));
+        const bool listed = e.fast || g.n > TINY_LARGE_MAX;            // short segments are served outside the tile lists
+        for (uint64_t t = 0; listed && t < seg_tiles; ++t) lists[which].push_back((uint32_t)(tiles + t));
+        for (uint64_t t = 0; listed && t < (seg_tiles + PACK_GROUP - 1) / PACK_GROUP; ++t) lists[2 + which].push_back((uint32_t)(groups + t));
         tiles += seg_tiles;
         groups += (seg_tiles + PACK_GROUP - 1) / PACK_GROUP;
         scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
@@ -267,6 +282,10 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
                                     sizeof(uint32_t) * lists[i].size(), cudaMemcpyHostToDevice, stream));
     c->n_slow_tiles = (uint32_t)lists[0].size(); c->n_fast_tiles = (uint32_t)lists[1].size();
     c->n_slow_groups = (uint32_t)lists[2].size(); c->n_fast_groups = (uint32_t)lists[3].size();
+    c->tiny_small = (uint32_t)tiny_a.size(); c->tiny_large = (uint32_t)tiny_b.size(); c->tiny_large_max_n = tiny_max_n;
+    tiny_a.insert(tiny_a.end(), tiny_b.begin(), tiny_b.end());
+    if (!tiny_a.empty())
+        SC_CUDA(cudaMemcpyAsync(c->d_tiny_list, tiny_a.data(), sizeof(uint32_t) * tiny_a.size(), cudaMemcpyHostToDevice, stream));
     if (!fast_list.empty())
         SC_CUDA(cudaMemcpyAsync(c->d_fast_list, fast_list.data(), sizeof(uint32_t) * fast_list.size(),
                                 cudaMemcpyHostToDevice, stream));
@@ -344,6 +363,29 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
         const uint32_t n_slow0 = (uint32_t)W * c->slow_segments;
         const uint32_t counters[2] = {n_slow0, 0u};
         SC_CUDA(cudaMemcpyAsync(c->d_nslow, counters, sizeof(counters), cudaMemcpyHostToDevice, stream));
+        if (c->tiny_small || c->tiny_large) {                          // short segments: one CTA each, in shared memory
+            TinyParams tp{};
+            tp.L = L; tp.grads = grads; tp.residuals = residuals; tp.out_vals = out_vals; tp.out_idx = out_idx;
+            tp.state = c->d_fstate; tp.W = (uint32_t)W; tp.status = c->d_status;
+            Launch l(c, KIND_TINY, stream);
+            if (c->tiny_small) {
+                tp.list = c->d_tiny_list; tp.count = c->tiny_small;
+                const uint32_t grid = persistent_grid(c, c->occ_tiny_small, (uint64_t)W * c->tiny_small);
+                topk_tiny_kernel<1><<<grid, THREADS, TINY_SMALL_MAX * sizeof(float), stream>>>(tp);
+            }
+            if (c->tiny_large) {
+                tp.list = c->d_tiny_list + c->tiny_small; tp.count = c->tiny_large;
+                const uint32_t per = (((c->tiny_large_max_n + TINY_CTAS - 1) / TINY_CTAS) + 3u) & ~3u;
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3((uint32_t)W * c->tiny_large * TINY_CTAS); cfg.blockDim = dim3(THREADS);
+                cfg.dynamicSmemBytes = (size_t)per * sizeof(float); cfg.stream = stream;
+                cudaLaunchAttribute attr;
+                attr.id = cudaLaunchAttributeClusterDimension;
+                attr.val.clusterDim.x = TINY_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+                cfg.attrs = &attr; cfg.numAttrs = 1;
+                SC_CUDA(cudaLaunchKernelEx(&cfg, topk_tiny_kernel<TINY_CTAS>, tp));
+            }
+        }
         if (L.fast_per_worker) {
             const uint32_t PF = (uint32_t)W * L.fast_per_worker;       // fast (worker, segment) pairs
             FastParams fp{};
@@ -621,6 +663,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     int rc = SC_OK;
     if ((rc = dev_alloc(c, &c->d_segs, (size_t)max_segments + 1)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_fast_list, (size_t)max_segments)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tiny_list, (size_t)max_segments)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_lists, 4 * c->max_tiles_per_worker)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_hist, P * HIST_WORDS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_state, P)) == SC_OK &&
@@ -649,6 +692,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     if (rc == SC_OK) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main, topk_main_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_tiny_small, topk_tiny_kernel<1>, THREADS, TINY_SMALL_MAX * sizeof(float));
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit, topk_restore_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[0], topk_emit_kernel<8, 4>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[1], topk_emit_kernel<16, 4>, THREADS, 0);
@@ -685,7 +729,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
 void sc_destroy(sc_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
-    cudaFree(c->d_segs); cudaFree(c->d_fast_list); cudaFree(c->d_lists); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
+    cudaFree(c->d_segs); cudaFree(c->d_fast_list); cudaFree(c->d_tiny_list); cudaFree(c->d_lists); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
     cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate);
     cudaFree(c->d_cand_hist); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_cbase);
     cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt);
@@ -755,7 +799,10 @@ int sc_topk_path_counts(sc_ctx* c, void* stream, uint32_t* h_counts) {
     if (h.empty()) return SC_OK;
     SC_CUDA(cudaMemcpyAsync(h.data(), c->d_fstate, h.size() * sizeof(FastState), cudaMemcpyDeviceToHost, st));
     SC_CUDA(cudaStreamSynchronize(st));
-    for (const FastState& f : h) if (f.path < 3) ++h_counts[f.path];
+    for (const FastState& f : h) {
+        if (f.path < 3) ++h_counts[f.path];
+        else if (f.path == PATH_TINY) ++h_counts[0];                   // a short segment: radix select in shared memory
+    }
     return SC_OK;
 }
 

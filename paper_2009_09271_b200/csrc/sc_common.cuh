@@ -80,7 +80,8 @@ struct TopkState {
 // Top-k of a large segment: state of the sampled-bracket path.
 enum { PATH_SLOW = 0,     // small segment: multi-pass radix select
        PATH_FAST = 1,     // bracket holds: single streaming pass + sparse emit
-       PATH_FAILED = 2 }; // bracket missed or a list overflowed: radix select on the parked p
+       PATH_FAILED = 2,   // bracket missed or a list overflowed: radix select on the parked p
+       PATH_TINY = 3 };   // short segment: one CTA, everything in shared memory
 struct FastState {
     uint32_t path;
     uint32_t lo, hi;       // bracket: key > hi is surely kept, key < lo surely dropped

@@ -173,7 +173,8 @@ pack_kernel(PackParams P) {
         const uint32_t item = s_dec[0];
         if (item == 0xFFFFFFFFu) break;
         const uint32_t w = s_dec[1], s = s_dec[2], gi = s_dec[3], ntl = s_dec[4];
-        if (P.fstate[(size_t)w * L.nseg + s].path == PATH_FAST) { __syncthreads(); continue; }
+        { const uint32_t path = P.fstate[(size_t)w * L.nseg + s].path;
+          if (path == PATH_FAST || path == PATH_TINY) { __syncthreads(); continue; } }
         const SegEntry seg = L.segs[s];
         const size_t row = (size_t)w * L.n_total + seg.offset;
         float* e = P.residuals + row;

@@ -48,7 +48,7 @@ topk_hist0_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
         }
         __syncthreads();
         const uint32_t w = s_dec[0], s = s_dec[1], t = s_dec[2], path = s_dec[3];
-        if (path == PATH_FAST) { __syncthreads(); continue; }
+        if (path == PATH_FAST || path == PATH_TINY) { __syncthreads(); continue; }
         const bool FUSE_ADD = path == PATH_SLOW;
         const long long prob = (long long)w * L.nseg + s;
         if (prob != cur_prob) {
@@ -116,7 +116,7 @@ topk_refine_kernel(Layout L, const float* __restrict__ residuals, uint32_t* __re
         const uint32_t w = s_dec[0], s = s_dec[1], t = s_dec[2];
         const long long prob = (long long)w * L.nseg + s;
         const TopkState st = state[prob];
-        if (st.active && fstate[prob].path != PATH_FAST) {   // uniform over the CTA
+        if (st.active && fstate[prob].path != PATH_FAST && fstate[prob].path != PATH_TINY) {   // uniform over the CTA
             if (prob != cur_prob) {
                 if (cur_prob >= 0) flush_hist<1024>(sh, hist + (size_t)cur_prob * HIST_WORDS + HOFF);
                 cur_prob = prob;
@@ -166,7 +166,7 @@ topk_resolve_kernel(Layout L, const uint32_t* __restrict__ hist, TopkState* __re
     __shared__ uint32_t s_found;
     const uint32_t prob = blockIdx.x;
     const uint32_t s = prob % L.nseg;
-    if (*n_slow == 0u || fstate[prob].path == PATH_FAST) return;
+    if (*n_slow == 0u || fstate[prob].path == PATH_FAST || fstate[prob].path == PATH_TINY) return;
     uint32_t need, prefix;
     if (LEVEL == 0) {
         need = L.segs[s].k;

@@ -36,6 +36,37 @@ def test_single_worker_sizes(ctx, scheme, n):
         run_step_both(ctx, scheme, g, e, [(0, n, k)], [1234 + k])
 
 
+@pytest.mark.parametrize("n", [4095, 4096, 4097, 36_864, 40_959, 40_960, 40_961, 50_000, 65_535])
+def test_topk_segment_size_classes(ctx, n):
+    """Short segments (one CTA, shared memory; two size classes) against the sizes just above them, which
+    take the multi-pass radix select: k from 1 to n, with ties across the threshold."""
+    W = 2
+    g = torch.stack([rand(n, 300 + w) for w in range(W)])
+    g[:, ::7] = g[:, 3:4]                                   # every seventh element equal: ties at many thresholds
+    e = torch.stack([rand(n, 310 + w, scale=1e-4) for w in range(W)])
+    e[:, ::7] = 0.0
+    for k in (1, n // 100, n // 7 + 3, n // 2, n - 1, n):
+        run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, k)], [0] * W)
+        assert ctx.sc_topk_path_counts() == (W, 0, 0)
+
+
+def test_topk_short_and_long_segments_in_one_table(ctx):
+    """All four size classes side by side in one call (short x 2, multi-pass, one-pass), several steps."""
+    sizes = [17, 4096, 1, 30_000, 45_000, 70_000, 2_000, 40_960, 131_072 + 5, 300]
+    segs, off = [], 0
+    for i, n_s in enumerate(sizes):
+        off += i % 3                                        # gaps: elements outside every segment stay untouched
+        segs.append((off, n_s, max(1, n_s // (3 + i))))
+        off += n_s
+    n, W = off + 2, 3
+    res = torch.stack([rand(n, 400 + w, scale=1e-4) for w in range(W)])
+    for t in range(3):
+        g = torch.stack([rand(n, 410 + 10 * t + w) for w in range(W)])
+        res = run_step_both(ctx, sc.SC_TOPK, g, res, segs, [t] * W, use=["step", "split", "host"][t])
+        workers_last_call = 1 if t == 2 else W              # the host-buffer step compresses worker by worker
+        assert ctx.sc_topk_path_counts() == (8 * workers_last_call, 2 * workers_last_call, 0)
+
+
 def test_topk_massive_ties_and_special_values(ctx):
     n = 3 * TILE + 17
     g = torch.zeros(1, n)
