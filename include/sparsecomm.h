@@ -113,7 +113,7 @@ int sc_compress(sc_ctx* ctx, int scheme, const float* grad, float* residual, siz
  * W rows of n elements (row w at +w*n); segs is a HOST array of nseg segments,
  * ascending and non-overlapping inside [0,n); elements outside every segment
  * are left alone.  h_seeds is a HOST array of W seeds; equal seeds give equal
- * coordinates (the paper's "same seed state").  Messages: row w of out_vals /
+ * coordinates (workers sharing their seed state, Methodology).  Messages: row w of out_vals /
  * out_idx has K = sum k_s entries (row w at +w*K). */
 int sc_compress_batch(sc_ctx* ctx, int scheme, int W, const float* grads, float* residuals, size_t n,
                       const sc_segment* segs, int nseg, const uint64_t* h_seeds,

@@ -15,15 +15,16 @@ agree bit for bit, so the oracle does NOT widen to fp64.
 Readings of the paper where it is silent or garbled (all restated in the
 project's design notes):
  * Algorithm 1, residual line: printed with the aggregate q_t; read as the
-   worker's own message, e' = p - q^w, as the Methodology prose says ("the
-   difference between the actual and the sparsified gradient is stored
-   locally"; "gradients of the current iteration that were not sent").
+   worker's own message, e' = p - q^w, as the Methodology prose says: what a
+   worker keeps is its own accumulated gradient minus what it sent, and the
+   residual collects the entries that were left out of the message.
  * Algorithm 1, accumulate line: gamma*g + e.  The caller passes gamma*g as the
    gradient; one fp32 add happens here.
  * Aggregate: Algorithm 1 prints a sum, the abstract and introduction say the
    workers use the average.  The oracle sums in worker order 0..W-1 starting
    from +0.0 and then divides by float(W).
- * "Top k ... according to their values": largest magnitude, compared on the
+ * Top-k (Methodology item; the paper does not say how values are ranked):
+   largest magnitude, compared on the
    bit pattern of |p| (so NaN > inf > finite, +0 == -0); ties go to the lowest
    index.
  * Message order: ascending coordinate, for every scheme.
@@ -37,7 +38,8 @@ project's design notes):
  * Step size: with gamma != 1 the accumulate line is evaluated as ONE fused
    multiply-add, p = round(gamma * g + e) (a single fp32 rounding); gamma = 1
    gives the plain add bit for bit.
- * "Same seed state": the seed is an argument; equal seeds give equal
+ * Workers that share their seed state (Methodology, on reduce against gather):
+   the seed is an argument; equal seeds give equal
    coordinates on every worker.
  * Scope (layer-wise or global): a segment table; segment s of a call uses the
    seed mix64(seed, s); global scope is a single segment (s = 0).
@@ -67,7 +69,7 @@ _M32 = (1 << 32) - 1
 
 # ---------------------------------------------------------------------------
 # Seed arithmetic (integer only).  This is the project's own specification of
-# "randomly selected" (Methodology, Random-k and Block-random-k items).
+# the random choice that the Methodology items Random-k and Block-random-k ask for.
 # ---------------------------------------------------------------------------
 def mix64(a: int, b: int) -> int:
     """64-bit finaliser of the SplitMix generator applied to a + (b+1)*phi."""
