@@ -54,7 +54,9 @@ struct sc_ctx {
     uint32_t* d_tile_ccnt = nullptr;
     uint32_t* d_tile_fbase = nullptr;
     uint32_t* d_tile_fcnt = nullptr;
-    size_t max_main_grid = 0;
+    size_t max_main_grid = 0;            // CTAs of the top-k pass in the build chosen for the current table
+    size_t main_grid_v[2] = {0, 0};      // [0]: three CTAs per SM, [1]: the two-CTA build
+    int main_wide = 0;                   // 1: the current table uses the two-CTA build
     uint2* d_flagged = nullptr;      // grown on demand: its size depends on k
     size_t flagged_slots = 0;
     uint32_t* d_nslow = nullptr;     // [0]: segments for the radix select, [1]: segments whose bracket missed
@@ -64,7 +66,7 @@ struct sc_ctx {
     uint32_t max_sample_m = 0, fast_big = 0;
     float gamma = 1.0f;                  // step size of the accumulate line (sc_set_gamma)
     uint32_t max_flag_cap = 0, max_cand_cap = 0;
-    int occ_main = 1, occ_emit = 1, occ_emit_v[4] = {1, 1, 1, 1};
+    int occ_main = 1, occ_main_wide = 1, occ_emit = 1, occ_emit_v[4] = {1, 1, 1, 1};
     uint64_t* d_seeds = nullptr;
     int* d_status = nullptr;
 
@@ -180,6 +182,19 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     uint32_t tiny_max_n = 0;
     uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0, cand = 0, flag = 0, smp = 0;
     uint32_t fast_count = 0, slow_count = 0, max_m = 0, max_cap = 0;
+    // Which build of the top-k streaming pass serves this table: the two-CTA build when every large segment is
+    // long (more tiles than the three-CTA build has CTAs) and the lists are sparse (at most 3 % flagged).
+    {
+        uint64_t big_n = 0, big_k = 0;
+        bool all_long = true;
+        for (int s = 0; s < nseg; ++s) {
+            if (segs[s].n < FAST_MIN_N) continue;
+            big_n += segs[s].n; big_k += segs[s].k;
+            if ((segs[s].n + 31 + TILE - 1) / TILE <= c->main_grid_v[0]) all_long = false;
+        }
+        c->main_wide = (big_n > 0 && all_long && 1.05 * (double)big_k <= 0.03 * (double)big_n) ? 1 : 0;
+        c->max_main_grid = c->main_grid_v[c->main_wide];
+    }
     for (int s = 0; s < nseg; ++s) {
         const sc_segment& g = segs[s];
         if (g.offset < end_prev || g.offset > n || g.n > n - g.offset) return SC_ERR_INVALID;
@@ -411,7 +426,9 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               }
               if (small) topk_bracket_kernel<1><<<small * (uint32_t)W, THREADS, 0, stream>>>(fp, big, small); }
             { Launch l(c, KIND_MAIN, stream);
-              topk_main_kernel<<<persistent_grid(c, c->occ_main, (items + MAIN_GROUP - 1) / MAIN_GROUP), THREADS, 0, stream>>>(fp); }
+              const uint64_t groups_of_tiles = (items + MAIN_GROUP - 1) / MAIN_GROUP;
+              if (c->main_wide) topk_main_kernel<1><<<persistent_grid(c, c->occ_main_wide, groups_of_tiles), THREADS, 0, stream>>>(fp);
+              else topk_main_kernel<3><<<persistent_grid(c, c->occ_main, groups_of_tiles), THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDBIN, stream);
               topk_candbin_kernel<<<PF, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_CANDFILTER, stream);
@@ -691,7 +708,8 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     }
     if (rc == SC_OK) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main, topk_main_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main, topk_main_kernel<3>, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main_wide, topk_main_kernel<1>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_tiny_small, topk_tiny_kernel<1>, THREADS, TINY_SMALL_MAX * sizeof(float));
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit, topk_restore_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[0], topk_emit_kernel<8, 4>, THREADS, 0);
@@ -719,7 +737,9 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
 #undef SC_FINE_SETUP
         }
         if (cudaGetLastError() != cudaSuccess) rc = SC_ERR_CUDA;
-        c->max_main_grid = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
+        c->main_grid_v[0] = (size_t)c->sm_count * (size_t)std::max(c->occ_main, 1);
+        c->main_grid_v[1] = (size_t)c->sm_count * (size_t)std::max(c->occ_main_wide, 1);
+        c->max_main_grid = c->main_grid_v[0];
     }
     if (rc != SC_OK) { sc_destroy(c); return rc; }
     *out = c;

@@ -274,7 +274,12 @@ __device__ inline MainTile main_decode(const FastParams& P, uint32_t item) {
     t.full = t.first >= 0 && t.first + TILE <= (long long)t.seg.n;
     return t;
 }
-__global__ void __launch_bounds__(THREADS)
+// Two builds of the same code: MINB = 3 holds the kernel to 80 registers (three CTAs per SM), which is what
+// many short segments and dense lists want; MINB = 1 lets it take 97 (two CTAs per SM), which streams long
+// segments with sparse lists 1.4 % faster (350 M x 16 at 1 %: 10.45 against 10.65 ms; at 10 %: 12.1 against
+// 11.6 ms the other way round).  The host picks one per segment table.
+template <int MINB>
+__global__ void __launch_bounds__(THREADS, MINB)
 topk_main_kernel(FastParams P) {
     __shared__ uint32_t sh[CAND_BINS];                                 // candidate histogram
     __shared__ __align__(16) float s_p[TILE];                          // the tile's p values, for the per-element work
@@ -303,9 +308,20 @@ topk_main_kernel(FastParams P) {
     bool pend_accumulates = false;
     const float gamma = L.gamma;
     const uint32_t group_step = (gridDim.x - 1u) * MAIN_GROUP + 1u;    // from a group's last tile to the next group's first
+    MainTile T{};
+    uint32_t seg_tile_end = 0;                                         // first tile after T's segment
     for (uint32_t item = blockIdx.x * MAIN_GROUP, ig = 0; ;
          item += (ig + 1u == MAIN_GROUP ? group_step : 1u), ig = (ig + 1u == MAIN_GROUP ? 0u : ig + 1u)) {
-        const MainTile T = main_decode(P, item);
+        // inside a group the next tile usually belongs to the same (worker, segment): then only its position
+        // changes, and the lookup of the segment (a search over the table) is skipped
+        if (ig != 0u && T.have && T.lt + 1u < seg_tile_end) {
+            T.lt += 1u;
+            T.first += TILE;
+            T.full = T.first >= 0 && T.first + TILE <= (long long)T.seg.n;
+        } else {
+            T = main_decode(P, item);
+            seg_tile_end = T.have ? L.segs[T.s + 1].tile_begin : 0u;
+        }
         // ---- flush the per-segment accumulators when the segment changes ---------------------------
         const long long prob = T.have ? (long long)T.w * L.nseg + T.s : -2;
         if (prob != cur_prob && cur_prob >= 0) {                       // uniform over the CTA
@@ -384,7 +400,7 @@ topk_main_kernel(FastParams P) {
         // during the per-element work below (measured on 350 M x 16 at 1 %: 12.3 -> 10.85 ms)
         if (SC_PREFETCH_DIST) {
             const uint32_t ahead = ig + 1u == MAIN_GROUP ? group_step : 1u;    // distance to this CTA's next tile
-            if (T.full && T.lt + ahead + 1u < L.segs[T.s + 1].tile_begin) {
+            if (T.full && T.lt + ahead + 1u < seg_tile_end) {
                 prefetch_tile_l2(T.g, e, T.first + (long long)ahead * TILE);
             } else {                                                   // the next tile lies in another segment: locate it
                 const MainTile N = main_decode(P, item + ahead);
