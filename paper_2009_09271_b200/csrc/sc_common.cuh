@@ -257,11 +257,12 @@ __device__ inline uint32_t key_of(float p) { return __float_as_uint(p) & 0x7FFFF
 
 // Tiles are laid on the 128-byte grid of the row, so that a warp's 512-byte access covers four
 // whole cache lines: elements of the segment before its first 128-byte boundary (0..31).
-// A persistent kernel knows which tile it takes next.  While the top-k pass works on a
-// tile's flagged elements its CTA has no loads in flight, so each thread asks L2 for one 128-byte line of
-// the tile that comes next (g by the lower half of the CTA, e by the upper half) and the next round of
-// loads finds its data in L2.  Only that kernel uses it: the random-k and block-random-k streams, which
-// have no such phase and run more CTAs per SM, were 15-25 % slower with the same prefetch.
+// A persistent kernel knows which tile it takes next.  While a CTA works on a tile (ranking, list and
+// message writes) it has no loads in flight, so once the tile's loads have landed each thread asks L2 for
+// one 128-byte line of the next tile (g by the lower half of the CTA, e by the upper half) and the next
+// round of loads finds its data in L2.  The request must come AFTER the current loads: issued before them
+// it made the random-k and block-random-k streams 15-25 % slower, after them it gains 12 % in the top-k
+// pass and 1.3 % in the random-k pass (the block-random-k stream already runs at the copy rate).
 #ifndef SC_PREFETCH_DIST
 #define SC_PREFETCH_DIST 1
 #endif

@@ -271,6 +271,10 @@ randk_pack_kernel(Layout L, const float* __restrict__ grads, float* __restrict__
                 const float4 gv = __ldcs(reinterpret_cast<const float4*>(g + mine + 128 * j));
                 qv[j] = accumulate(L.gamma, gv, ev);
             }
+            if (SC_PREFETCH_DIST) {   // this tile's loads have landed: ask L2 for the tile the CTA takes next
+                const uint32_t ahead = ig + 1u == STREAM_GROUP ? group_step : 1u;
+                if (lt + ahead + 1u < L.segs[s + 1].tile_begin) prefetch_tile_l2(g, e, first + (long long)ahead * TILE);
+            }
             if (bits) {
 #pragma unroll
                 for (int j = 0; j < QUADS; ++j) {
