@@ -346,8 +346,14 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     # per-scheme device time from the marks
     per_scheme_ms = {s: 0.0 for s in schemes}
     prev = start
+    step_ms, acc = [], 0.0
     for i, ev in enumerate(marks):
-        per_scheme_ms[schemes[i % len(schemes)]] += prev.elapsed_time(ev)
+        dt = prev.elapsed_time(ev)
+        per_scheme_ms[schemes[i % len(schemes)]] += dt
+        acc += dt
+        if (i + 1) % len(schemes) == 0:                        # the last scheme of a step
+            step_ms.append(acc)
+            acc = 0.0
         prev = ev
 
     peak, peak_src = measured_peak()
@@ -383,7 +389,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": elapsed_ms / args.steps,
+        "ms_per_step_median": round(statistics.median(step_ms), 4) if step_ms else None,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w.name}: flat n={n} x W={W} simulated workers per GPU, {w.values} values, "
                                f"density {num}/{den} (k={K}), schemes {','.join(schemes)}, shared seed per step, "
