@@ -750,9 +750,8 @@ topk_emit_kernel(FastParams P) {
             }
         }
         const uint32_t maxcnt = __reduce_max_sync(0xFFFFFFFFu, cnt);
-        // entry i of the slice belongs to lane i % G of the group; message pointers advance with the running rank
-        float* ov = ovals + running;
-        uint32_t* oi = oidx + running;
+        // entry i of the slice belongs to lane i % G of the group; the message position advances with the running rank
+        uint32_t pos = running;
         const uint2* fl = flist0 + base + gl;
         for (uint32_t b = 0; b < maxcnt; b += G * D) {                  // D independent loads in flight per lane
             uint2 a[D];
@@ -760,20 +759,18 @@ topk_emit_kernel(FastParams P) {
             for (int u = 0; u < D; ++u) a[u] = (b + G * u + gl < cnt) ? __ldg(fl + b + G * u) : make_uint2(0u, 0xFFFFFFFFu);
 #pragma unroll
             for (int u = 0; u < D; ++u) {
-                // a padding entry has key 0 and coordinate 2^32-1: kept only if T == 0 and icut == 2^32-1, which
-                // cannot happen (coordinates are < n < 2^32, so icut <= n); a group without a tile has cnt == 0 and
-                // T, icut from its last tile or 0, so its padding entries are never kept either
+                // a padding entry has key 0 and coordinate 2^32-1: it would be kept only if T == 0 and icut > 2^32-1,
+                // which cannot be (a group without a tile has T and icut of its last tile, or 0 and 0)
                 const uint32_t key = a[u].x & 0x7FFFFFFFu;
-                const bool sel = (b + G * u + gl < cnt) && (key > T || (key == T && a[u].y < icut));
+                const bool sel = key > T || (key == T && a[u].y < icut);
                 const uint32_t bal = (__ballot_sync(0xFFFFFFFFu, sel) >> gshift) & gmask;
                 if (sel) {
-                    const uint32_t r = __popc(bal & lt_mask);
-                    ov[r] = __uint_as_float(a[u].x);
-                    oi[r] = idx0 + a[u].y;
+                    const uint32_t r = pos + __popc(bal & lt_mask);
+                    ovals[r] = __uint_as_float(a[u].x);
+                    oidx[r] = idx0 + a[u].y;
                     if (key <= hi) e[a[u].y] = 0.0f;                    // a kept candidate: the main pass left p there
                 }
-                const uint32_t adv = __popc(bal);
-                ov += adv; oi += adv;
+                pos += __popc(bal);
             }
         }
     }
