@@ -50,6 +50,7 @@ struct sc_ctx {
     uint2* d_cand = nullptr;
     uint2* d_list2 = nullptr;
     uint32_t* d_tile_sure = nullptr;
+    uint32_t* d_tile_csum = nullptr;
     uint32_t* d_tile_cbase = nullptr;
     uint32_t* d_tile_ccnt = nullptr;
     uint32_t* d_tile_fbase = nullptr;
@@ -406,7 +407,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             FastParams fp{};
             fp.L = L; fp.grads = grads; fp.residuals = residuals; fp.out_vals = out_vals; fp.out_idx = out_idx;
             fp.state = c->d_fstate; fp.sample = c->d_sample; fp.cand_hist = c->d_cand_hist;
-            fp.list2 = c->d_list2; fp.cand = c->d_cand; fp.tile_sure = c->d_tile_sure; fp.tile_cbase = c->d_tile_cbase;
+            fp.list2 = c->d_list2; fp.cand = c->d_cand; fp.tile_sure = c->d_tile_sure; fp.tile_csum = c->d_tile_csum; fp.tile_cbase = c->d_tile_cbase;
             fp.tile_ccnt = c->d_tile_ccnt; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
             fp.flagged = c->d_flagged; fp.offsets = c->d_offsets;
             fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
@@ -439,7 +440,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
               topk_restore_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_TILECOUNT, stream);
-              topk_tilecount_kernel<<<(uint32_t)(((uint64_t)(items + TILES_PER_GROUP - 1) / TILES_PER_GROUP * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
+              topk_tilecount_kernel<<<(items + THREADS - 1) / THREADS, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_ROW_SCAN, stream);
               if ((rc_scan = launch_row_scan(c->d_offsets, (uint32_t)W, L.tiles_per_worker, stream)) != SC_OK) return rc_scan; }
             { Launch l(c, KIND_EMIT, stream);
@@ -693,6 +694,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_cand_hist, fastP * CAND_BINS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_list2, fastP * LIST2_CAP)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_sure, items_max)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tile_csum, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_cbase, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_ccnt, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_fbase, items_max)) == SC_OK &&
@@ -751,7 +753,7 @@ void sc_destroy(sc_ctx* c) {
     DeviceGuard guard(c->device);
     cudaFree(c->d_segs); cudaFree(c->d_fast_list); cudaFree(c->d_tiny_list); cudaFree(c->d_lists); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
     cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate);
-    cudaFree(c->d_cand_hist); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_cbase);
+    cudaFree(c->d_cand_hist); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_csum); cudaFree(c->d_tile_cbase);
     cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt);
     cudaFree(c->d_flagged); cudaFree(c->d_nslow); cudaFree(c->d_seeds); cudaFree(c->d_status);
     cudaFree(c->d_stage_grads); cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); cudaFree(c->d_stage_out);

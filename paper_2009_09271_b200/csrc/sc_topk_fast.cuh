@@ -44,6 +44,7 @@ struct FastParams {
     uint32_t* tile_sure;       // [W * tiles_per_worker] sure elements of the tile (zeroed before the pass)
     uint32_t* tile_cbase;      // first candidate slot of the tile
     uint32_t* tile_ccnt;       // candidates of the tile
+    uint32_t* tile_csum;       // candidates above the threshold's bin (low half) and inside it (high half)
     uint32_t* tile_fbase;      // first flagged slot of the tile (0xFFFFFFFF: the list was full, nothing written)
     uint32_t* tile_fcnt;       // flagged elements of the tile
     uint32_t* n_failed;        // segments whose bracket missed
@@ -589,23 +590,34 @@ topk_candfilter_kernel(FastParams P) {
     const Layout& L = P.L;
     const uint32_t sub = threadIdx.x & 7u;
     const uint32_t item0 = ((blockIdx.x * THREADS + threadIdx.x) >> 3) * TILES_PER_GROUP;
-    if (item0 >= P.total_items) return;
     CandSlice t[TILES_PER_GROUP];
     cand_slices<true>(P, item0, sub, t);
 #pragma unroll
     for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-        if (!t[u].list || t[u].cnt == 0u) continue;
-        const FastState* stp = P.state + t[u].prob;
-        const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
-        const uint32_t s = t[u].prob - t[u].w * L.nseg;
-        uint2* out = P.list2 + ((size_t)t[u].w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
-        for (uint32_t i = sub; i < t[u].cnt; i += 8) {
-            const uint2 c = i == sub ? t[u].first : t[u].list[i];
-            if (c.x >= lo2 && c.x <= hi2) {
-                const uint32_t pos = atomicAdd(&P.state[t[u].prob].cnt2, 1u);
-                if (pos < LIST2_CAP) out[pos] = c;
+        // candidates above the threshold's bin are kept whatever the exact threshold turns out to be; those
+        // inside the bin go to the short list.  Both counts are left for the per-tile kept count, which then
+        // reads a tile's candidates again only if some of them lie inside the bin (a few thousand tiles at most).
+        uint32_t above = 0, inbin = 0;
+        if (t[u].list && t[u].cnt) {
+            const FastState* stp = P.state + t[u].prob;
+            const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
+            const uint32_t s = t[u].prob - t[u].w * L.nseg;
+            uint2* out = P.list2 + ((size_t)t[u].w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
+            for (uint32_t i = sub; i < t[u].cnt; i += 8) {
+                const uint2 c = i == sub ? t[u].first : t[u].list[i];
+                if (c.x > hi2) ++above;
+                else if (c.x >= lo2) {
+                    ++inbin;
+                    const uint32_t pos = atomicAdd(&P.state[t[u].prob].cnt2, 1u);
+                    if (pos < LIST2_CAP) out[pos] = c;
+                }
             }
         }
+        uint32_t both = above | (inbin << 16);                         // a tile holds at most 4096 candidates
+        both += __shfl_xor_sync(0xFFFFFFFFu, both, 1);
+        both += __shfl_xor_sync(0xFFFFFFFFu, both, 2);
+        both += __shfl_xor_sync(0xFFFFFFFFu, both, 4);
+        if (sub == 0u && item0 + u < P.total_items) P.tile_csum[item0 + u] = both;
     }
 }
 
@@ -661,34 +673,32 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
 
 // ---- kept count per tile = sure elements + chosen candidates -------------------------------------
 __global__ void __launch_bounds__(THREADS)
-topk_tilecount_kernel(FastParams P) {
+topk_tilecount_kernel(FastParams P) {                                 // one thread per tile
     const Layout& L = P.L;
-    const uint32_t sub = threadIdx.x & 7u;
-    const uint32_t item0 = ((blockIdx.x * THREADS + threadIdx.x) >> 3) * TILES_PER_GROUP;
-    CandSlice t[TILES_PER_GROUP];
-    uint32_t sure[TILES_PER_GROUP];
-#pragma unroll
-    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u)
-        sure[u] = (sub == 0u && item0 + u < P.total_items) ? __ldg(P.tile_sure + item0 + u) : 0u;
-    cand_slices<false>(P, item0, sub, t);
-#pragma unroll
-    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-        uint32_t kept = 0;
-        if (t[u].list) {                                               // a tile of a segment on the one-pass path
-            const FastState* st = P.state + t[u].prob;
-            const uint32_t T = st->T, icut = st->icut;
-            for (uint32_t i = sub; i < t[u].cnt; i += 8) {
-                const uint2 c = i == sub ? t[u].first : t[u].list[i];
-                kept += fast_kept(c.x, c.y, T, icut) ? 1u : 0u;
+    const uint32_t item = blockIdx.x * THREADS + threadIdx.x;
+    if (item >= P.total_items) return;
+    const uint32_t sure = __ldg(P.tile_sure + item), both = __ldg(P.tile_csum + item);
+    const uint32_t w = item / L.tiles_per_worker;
+    const uint32_t lt = item - w * L.tiles_per_worker;
+    const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+    const SegEntry& seg = L.segs[s];
+    uint32_t kept = 0;
+    if (seg.fast) {
+        const FastState* st = P.state + (size_t)w * L.nseg + s;
+        if (st->path == PATH_FAST) {
+            kept = sure + (both & 0xFFFFu);
+            if (both >> 16) {                                          // candidates inside the threshold's bin: the exact rule
+                const uint32_t T = st->T, icut = st->icut, lo2 = st->lo2, hi2 = st->hi2;
+                const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + P.tile_cbase[item];
+                const uint32_t cnt = P.tile_ccnt[item];
+                for (uint32_t i = 0; i < cnt; ++i) {
+                    const uint2 c = list[i];
+                    if (c.x >= lo2 && c.x <= hi2) kept += fast_kept(c.x, c.y, T, icut) ? 1u : 0u;
+                }
             }
-            kept += sure[u];
         }
-        kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 1);
-        kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 2);
-        kept += __shfl_xor_sync(0xFFFFFFFFu, kept, 4);
-        if (sub == 0u && item0 + u < P.total_items)
-            P.offsets[(size_t)t[u].w * (L.tiles_per_worker + 1) + t[u].lt] = kept;
     }
+    P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
 }
 
 // ---- emit: G lanes per tile walk the tile's slice of the flagged list ----------------------------
