@@ -21,7 +21,8 @@
 //            kept entries go to the message in ascending coordinate order, kept candidates
 //            are zeroed in the residual.  On a fall-back the sure values are first written
 //            back from the flagged list.
-// No CTA waits on another anywhere on this path.
+// No CTA polls for another anywhere on this path; the bracket and the row scan use thread-block
+// clusters, whose CTAs meet at hardware cluster barriers only.
 #pragma once
 #include <cooperative_groups.h>
 
