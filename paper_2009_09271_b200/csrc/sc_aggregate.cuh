@@ -417,8 +417,9 @@ agg_apply_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restric
             for (uint32_t i = threadIdx.x; i < tile_n; i += THREADS) {
                 const float a = acc[i];
                 if (a != 0.0f) {                                   // also true for NaN
-                    const float q = pow2 ? a * rW : a / fW;
-                    x[tile_lo + i] = x[tile_lo + i] - q;
+                    // two roundings, as in "average, then subtract": never contracted into one fused multiply-add
+                    const float q = pow2 ? __fmul_rn(a, rW) : __fdiv_rn(a, fW);
+                    x[tile_lo + i] = __fsub_rn(x[tile_lo + i], q);
                 }
             }
         }
@@ -438,7 +439,7 @@ agg_apply_shared_kernel(const float* __restrict__ vals, const uint32_t* __restri
         float sum = 0.0f;
         for (uint32_t w = 0; w < W; ++w) sum = sum + vals[(size_t)w * K + j];
         if (i >= n) { atomicMin(status, ST_DEVICE_CHECK); continue; }
-        if (sum != 0.0f) x[i] = x[i] - (pow2 ? sum * rW : sum / fW);
+        if (sum != 0.0f) x[i] = __fsub_rn(x[i], pow2 ? __fmul_rn(sum, rW) : __fdiv_rn(sum, fW));   // never one fused multiply-add
     }
 }
 

@@ -178,6 +178,12 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     if (c->layout_valid && c->cached_n == n && (int)c->cached_segs.size() == nseg &&
         std::memcmp(c->cached_segs.data(), segs, sizeof(sc_segment) * nseg) == 0)
         return SC_OK;
+    // From here on the cached table no longer describes the scratch: a failure below must not let a later
+    // call with the old table take the early-out above.  Nothing of the context changes before the new
+    // table has been validated.
+    c->layout_valid = false;
+    int main_wide = 0;
+    size_t max_main_grid = 0;
     std::vector<SegEntry> h(nseg + 1);
     std::vector<uint32_t> fast_list, lists[4], tiny_a, tiny_b;
     uint32_t tiny_max_n = 0;
@@ -193,8 +199,8 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             big_n += segs[s].n; big_k += segs[s].k;
             if ((segs[s].n + 31 + TILE - 1) / TILE <= c->main_grid_v[0]) all_long = false;
         }
-        c->main_wide = (big_n > 0 && all_long && 1.05 * (double)big_k <= 0.03 * (double)big_n) ? 1 : 0;
-        c->max_main_grid = c->main_grid_v[c->main_wide];
+        main_wide = (big_n > 0 && all_long && 1.05 * (double)big_k <= 0.03 * (double)big_n) ? 1 : 0;
+        max_main_grid = c->main_grid_v[main_wide];
     }
     for (int s = 0; s < nseg; ++s) {
         const sc_segment& g = segs[s];
@@ -224,9 +230,9 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             // one region per tile when the segment has no more tiles than the pass has CTAs, else one
             // per CTA (which sees at most ceil(tiles / CTAs) tiles of the segment).  A region holds its
             // tiles' share of (k + slack) resp. slack entries plus a little room per tile.
-            const bool per_tile = seg_tiles <= c->max_main_grid;
+            const bool per_tile = seg_tiles <= max_main_grid;
             const uint64_t slack = per_tile ? g.n / 16 + 1024 : g.n / 32 + 16384;
-            const uint64_t regions = per_tile ? seg_tiles : c->max_main_grid;
+            const uint64_t regions = per_tile ? seg_tiles : max_main_grid;
             // (a CTA takes groups of MAIN_GROUP consecutive tiles, every regions-th group: the segment overlaps at
             // most seg_tiles / MAIN_GROUP + 2 groups)
             const uint64_t tiles_per_region = per_tile ? 1 : MAIN_GROUP * ((seg_tiles / MAIN_GROUP + 2 + regions - 1) / regions);
@@ -277,7 +283,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     const size_t smp_slots = ((size_t)c->max_W * smp + 1) / 2 + 1;  // sample keys are 4 bytes, list entries 8; +1 to align
     if ((size_t)c->max_W * (flag + cand) + smp_slots > c->flagged_slots) {   // the lists follow k: grow them (synchronous, rare)
         SC_CUDA(cudaStreamSynchronize(stream));
-        cudaFree(c->d_flagged); c->d_flagged = nullptr;
+        cudaFree(c->d_flagged); c->d_flagged = nullptr; c->d_cand = nullptr; c->d_sample = nullptr;
         c->scratch_bytes -= c->flagged_slots * sizeof(uint2);
         c->flagged_slots = 0;
         const size_t want = (size_t)c->max_W * (flag + cand) + smp_slots;
@@ -310,6 +316,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     L.scat_per_group = (uint32_t)scat; L.K_total = (uint32_t)msg; L.n_total = n; L.mask_words_per_group = maskw;
     L.cand_per_worker = cand; L.flag_per_worker = flag; L.sample_per_worker = smp; L.fast_per_worker = fast_count;
     c->layout = L;
+    c->main_wide = main_wide; c->max_main_grid = max_main_grid;
     c->slow_segments = slow_count; c->fast_big = big_count; c->max_sample_m = max_m; c->max_flag_cap = max_cap;
     c->cached_segs.assign(segs, segs + nseg);
     c->cached_n = n;

@@ -1,4 +1,6 @@
 """GPU parity: the CUDA library against the CPU oracle, bit for bit, through the C ABI."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -429,4 +431,58 @@ def test_aggregate_apply_matches_dense_update(W):
     c.sc_aggregate_apply(W, d_vals, d_idx[0].contiguous(), k, n, xs, shared=True)
     assert c.sc_sync_status() == 0
     assert_bits_equal(xs, O.aggregate_apply(x0, list(vals), [idx[0]] * W), "apply shared")
+    c.close()
+
+
+def test_rejected_table_does_not_poison_the_cached_layout():
+    """A segment table that fails validation after another one was accepted must leave the context able to
+    serve the earlier table again (the cached layout is dropped, not half-updated)."""
+    n = (1 << 20) + 4099
+    own = sc.Context(max_n=n, max_W=2, max_segments=4)
+    g = torch.stack([rand(n, 1200 + w) for w in range(2)])
+    e = torch.stack([rand(n, 1210 + w, scale=1e-4) for w in range(2)])
+    good = [(0, n, n // 100)]
+    e1 = run_step_both(own, sc.SC_TOPK, g, e, good, [0, 0])
+    lib, h = sc.load_library(), own._h
+    gd, ed = g.cuda(), e1.cuda()
+    ed0 = ed.clone()
+    vals = torch.zeros(2, n // 2, device="cuda"); idx = torch.zeros(2, n // 2, device="cuda", dtype=torch.int32)
+    seeds = (ctypes.c_uint64 * 2)(0, 0)
+    # overlapping segments; a table whose dense lists want the other build of the streaming pass, then fails
+    for bad in ([(0, n // 2 + 10, 5), (n // 2, n - n // 2, 5)],
+                [(0, n // 2, n // 4), (n // 2 - 1, n // 2, 7)]):
+        arr = (sc.binding.ScSegment * len(bad))(*[sc.binding.ScSegment(*b) for b in bad])
+        rc = lib.sc_compress_batch(h, sc.SC_TOPK, 2, gd.data_ptr(), ed.data_ptr(), n, arr, len(bad), seeds,
+                                   vals.data_ptr(), idx.data_ptr(), None)
+        assert rc == -1
+        torch.cuda.synchronize()
+        assert torch.equal(ed, ed0) and not vals.any()
+        run_step_both(own, sc.SC_TOPK, g, e1, good, [0, 0])              # the earlier table still gives the oracle's bits
+        assert own.sc_topk_path_counts() == (0, 2, 0)
+    own.close()
+
+
+@pytest.mark.parametrize("W", [2, 4, 3])
+def test_aggregate_apply_denormal_sums(W):
+    """Sums and model values in the denormal range: average-then-subtract is two roundings, which a fused
+    multiply-add would merge into one."""
+    rng = np.random.default_rng(90 + W)
+    n, k = 20_000, 3000
+    c = sc.Context(max_n=n, max_W=4, max_segments=1)
+    idx = np.stack([np.sort(rng.choice(n, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+    vals = rng.integers(1, 1 << 12, (W, k)).astype(np.uint32)            # denormals: tiny odd multiples of 2^-149
+    vals |= rng.integers(0, 2, (W, k)).astype(np.uint32) << 31
+    vals = vals.view(np.float32)
+    x0 = rng.integers(1, 1 << 14, n).astype(np.uint32)
+    x0 |= rng.integers(0, 2, n).astype(np.uint32) << 31
+    x0 = x0.view(np.float32)
+    d_idx, d_vals = torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(vals.copy()).cuda()
+    x = torch.from_numpy(x0.copy()).cuda()
+    c.sc_aggregate_apply(W, d_vals, d_idx, k, n, x)
+    assert c.sc_sync_status() == 0
+    assert_bits_equal(x, O.aggregate_apply(x0, list(vals), list(idx)), "apply, denormals")
+    xs = torch.from_numpy(x0.copy()).cuda()
+    c.sc_aggregate_apply(W, d_vals, d_idx[0].contiguous(), k, n, xs, shared=True)
+    assert c.sc_sync_status() == 0
+    assert_bits_equal(xs, O.aggregate_apply(x0, list(vals), [idx[0]] * W), "apply shared, denormals")
     c.close()
