@@ -52,6 +52,11 @@ def parse_args():
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="do not bracket every kernel with events in the timed region (no roofline object)")
     ap.add_argument("--cpu-sample-div", type=int, default=1, help="oracle sample = n / this of one worker")
+    ap.add_argument("--scope", default="layerwise", choices=["layerwise", "flat"],
+                    help="one k per tensor of the workload, or one segment over the whole vector")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the sweep over the other densities and workloads that follows the default run")
+    ap.add_argument("--sweep-steps", type=int, default=10)
     ap.add_argument("--selftest-dist", action="store_true",
                     help="CPU-only check of the multi-rank plumbing (gloo): barrier, max over ranks, aggregate value")
     return ap.parse_args()
@@ -121,16 +126,13 @@ def algorithmic_bytes(kind: str, n: int, W: int, K: int, shared: bool) -> float:
     """Bytes one launch of a kernel must move by the definition of its step
     (operands read once, results written once)."""
     return {
-        "topk_hist0": 12.0 * n * W,                      # read g, read e, write p
-        "topk_refine": 4.0 * n * W,                      # read p
-        "pack_topk": 4.0 * n * W + 12.0 * K * W,         # read p; write vals, idx and the kept zeros
         "randk_pack": 12.0 * n * W + n / 8.0 * W + 8.0 * K * W,  # read g, e, mask; write e', vals, idx
         "mask_count": n / 8.0, "row_scan": 8.0 * (n / 4096.0),
         "randblock": 12.0 * n * W + 8.0 * K * W,
         "randk_scatter": 4.0 * K,
         "agg_tiles": 4.0 * n + (4.0 * K * W + 4.0 * K if shared else 8.0 * K * W),
+        "agg_warp": 4.0 * n + 8.0 * K * W, "agg_fine": 4.0 * n + 8.0 * K * W,     # private coordinates (top-k)
         "agg_bounds": 4.0 * (n / 4096.0) * (1 if shared else W),
-        "topk_resolve": 0.0,
         "topk_main": 12.0 * n * W + 8.0 * K * W,          # read g, e; write e' and the flagged (value, coordinate) list
         "topk_emit": 16.0 * K * W,                        # read the flagged list, write vals and idx
     }.get(kind, 0.0)
@@ -199,8 +201,96 @@ def build_problem(args):
         sizes = [args.n]
     W = args.workers or w.W
     schemes = [s for s in (args.schemes.split(",") if args.schemes else w.schemes) if s]
-    segs = wl.segment_table(sizes, num, den)
+    segs = wl.flat_table(sum(sizes), num, den) if args.scope == "flat" else wl.segment_table(sizes, num, den)
     return w, sizes, W, schemes, segs, (num, den)
+
+
+
+# The other configurations of the metric: every (workload, scope, density) below is timed like the
+# headline (W workers per step, CUDA events around `steps` whole steps of one scheme, a fresh gradient
+# set every step out of `pool`, residuals carried, clocks sampled), without per-kernel events.
+SWEEP_PLAN = (
+    ("c5", "flat", ((1, 10000), (1, 1000), (1, 10))),          # 1/100 is the headline itself
+    ("c1", "flat", ((1, 100),)),
+    ("c2", "layerwise", ((1, 100),)),
+    ("c3", "layerwise", ((1, 1000),)),
+    ("c4", "layerwise", ((1, 1000), (1, 100), (1, 10))),
+    ("c4", "flat", ((1, 1000), (1, 100), (1, 10))),
+)
+
+
+def time_schemes(torch, sc, ctx, wl, w, W, n, schemes, seg_t, K, grads, res, vals, idx, out, steps, warmup, peak, uuid):
+    """One sweep entry: per scheme `warmup` untimed steps, then `steps` timed ones."""
+    pool = len(grads)
+    sampler = ClockSampler(uuid)
+    sampler.start()
+    per, paths = {}, None
+    for s in schemes:
+        code = sc.SCHEMES[s]
+        for t in range(warmup):
+            ctx.sc_step(code, grads[t % pool], res[s], seg_t, [wl.step_seed(w.base_seed, t)] * W, vals, idx, out)
+        if s == "topk":
+            paths = dict(zip(("radix_small", "one_pass", "radix_after_missed_bracket"), ctx.sc_topk_path_counts()))
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for t in range(steps):
+            ctx.sc_step(code, grads[(warmup + t) % pool], res[s], seg_t,
+                        [wl.step_seed(w.base_seed, warmup + t)] * W, vals, idx, out)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / steps
+        bmin = step_min_bytes(s, n, W, K, shared=True)
+        per[s] = {"ms": round(ms, 4), "elements_per_s": W * n / (ms * 1e-3), "min_GB": round(bmin / 1e9, 4),
+                  "frac_of_8000": round(bmin / (ms * 1e-3) / 1e9 / CONTRACT_PEAK_GBS, 4),
+                  "frac_of_measured": round(bmin / (ms * 1e-3) / 1e9 / peak, 4)}
+    status = ctx.sc_sync_status()
+    if status != 0:
+        raise RuntimeError(f"device status in the sweep: {sc.strerror(status)}")
+    return per, paths, sampler.stop()
+
+
+def run_sweep(args, torch, sc, wl, dev, peak, uuid, c5_state):
+    """Returns the list of sweep entries.  c5_state = (ctx, grads, res, out) of the headline run, reused for
+    the other densities of the largest workload; the smaller workloads get buffers of their own."""
+    entries = []
+    for name, scope, densities in SWEEP_PLAN:
+        w = wl.workload(name)
+        n, W = w.n, w.W
+        if name == "c5":
+            ctx, grads, res, out = c5_state
+            own = False
+        else:
+            ctx = sc.Context(max_n=n, max_W=W, max_segments=len(w.sizes))
+            grads = []
+            for t in range(max(1, args.pool)):
+                g = torch.empty(W, n, device=dev)
+                for ww in range(W):
+                    g[ww] = wl.generate(w, ww, t, dev)
+                grads.append(g)
+            res = {s: torch.zeros(W, n, device=dev) for s in w.schemes}
+            out = torch.empty(n, device=dev)
+            own = True
+        for num, den in densities:
+            segs = wl.flat_table(n, num, den) if scope == "flat" else wl.segment_table(w.sizes, num, den)
+            seg_t = [(s.offset, s.n, s.k) for s in segs]
+            K = sum(s.k for s in segs)
+            vals = torch.empty(W, max(K, 1), device=dev)
+            idx = torch.empty(W, max(K, 1), device=dev, dtype=torch.int32)
+            for s in w.schemes:
+                res[s].zero_()
+            per, paths, clocks = time_schemes(torch, sc, ctx, wl, w, W, n, w.schemes, seg_t, K, grads, res, vals, idx,
+                                              out, args.sweep_steps, max(3, args.warmup), peak, uuid)
+            entries.append({"config": name, "scope": scope, "density": f"{num}/{den}", "n": n, "W": W,
+                            "segments": len(segs), "k": K, "steps": args.sweep_steps,
+                            "l2": "working set fits L2" if 8.0 * n * W < 100e6 else "inputs larger than L2",
+                            "schemes": per, "topk_paths": paths, "clocks": clocks})
+            del vals, idx
+        if own:
+            ctx.close()
+            del grads, res, out
+            torch.cuda.empty_cache()
+    return entries
 
 
 def run_reference(args, rank: int):
@@ -377,7 +467,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         if per_elem is not None:
             roofline["traffic"] = per_elem * n * W
             roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum per element from one ncu capture "
-                                        "at n=1e8, W=2 (profiles/streaming_kernels_n100M_W2.md), scaled by n*W")
+                                        "of this kernel at n=1e8, W=2, scaled by n*W (traffic grows with n*W)")
+        else:
+            roofline["traffic_note"] = (f"no ncu capture of {dom} is on record: DRAM traffic per element was captured "
+                                        "for the streaming kernels only (" + ", ".join(NCU_DRAM_BYTES_PER_ELEMENT) + ")")
     step_roof = {}
     for s in schemes:
         t_s = per_scheme_ms[s] / args.steps * 1e-3
@@ -442,6 +535,13 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         line["next_rows"] = tim
         del xmodel
 
+    # ---- the other densities and workloads of the metric (not part of `value`) ------------------
+    default_run = (args.workload == "c5" and args.density == "1/100" and not args.n and not args.workers
+                   and not args.schemes and args.scope == "layerwise")
+    if rank == 0 and world == 1 and default_run and not args.no_sweep:
+        del vals, idx
+        line["sweep"] = run_sweep(args, torch, sc, wl, dev, peak, sampler.uuid, (ctx, grads, res, out))
+
     # ---- end to end through the C ABI with host buffers ------------------------------------
     if not args.no_e2e and rank == 0:
         line["e2e"] = run_e2e(args, ctx, sc, wl, w, sizes, W, schemes, codes, seg_t, res, n, dev)
@@ -484,11 +584,14 @@ def run_e2e(args, ctx, sc, wl, w, sizes, W, schemes, codes, seg_t, res, n, dev):
     status = ctx.sc_sync_status()
     if status != 0:
         raise RuntimeError(f"device status after the end-to-end run: {sc.strerror(status)}")
+    h2d, d2h = 4 * n * W * len(schemes), 4 * n * len(schemes)
     return {"value": W * n * len(schemes) * steps / dt, "unit": UNIT, "steps": steps,
             "ms_per_step": 1e3 * dt / steps,
-            "h2d_bytes_per_step": 4 * n * W * len(schemes), "d2h_bytes_per_step": 4 * n * len(schemes),
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "host_link_GBps": round((h2d + d2h) * steps / dt / 1e9, 2),
             "note": "sc_step_host: pinned host gradients copied per worker, overlapped with compression; "
-                    "dense average copied back"}
+                    "dense average copied back.  Every step uploads W*n fresh floats, so this number is the rate "
+                    "of the host link (host_link_GBps = bytes copied / time), not of the kernels"}
 
 
 def run_cpu_baseline(args, wl, w, sizes, schemes, num, den, grads0):
@@ -508,9 +611,37 @@ def run_cpu_baseline(args, wl, w, sizes, schemes, num, den, grads0):
         v, i, _ = O.compress_segments(O.SCHEMES[s], g, e, segs, wl.step_seed(w.base_seed, 0))
         O.aggregate([v], [i], n)
     dt = time.perf_counter() - t0
-    return {"value": n * len(schemes) / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 2),
+    base = {"value": n * len(schemes) / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": round(dt, 2),
             "sample": f"worker 0, first {n} of {n_full} elements, schemes {','.join(schemes)}, density {num}/{den}, "
                       f"compress + aggregate of that one message"}
+    # the same oracle with one thread per worker (workers are independent), on a quarter of each row
+    try:
+        from concurrent.futures import ThreadPoolExecutor
+        cores = len(os.sched_getaffinity(0))
+        Wt = max(1, min(grads0.shape[0], cores))
+        nq = max(1, n // 4)
+        segq = [(s.offset, s.n, s.k) for s in wl.segment_table([nq], num, den)] if len(sizes_s) == 1 else segs
+        nq = sum(s[1] for s in segq)
+        rows = [grads0[ww, :nq].cpu().numpy() for ww in range(Wt)]
+        seed = wl.step_seed(w.base_seed, 0)
+
+        def one_worker(g_row):
+            e_row = np.zeros(nq, np.float32)
+            return [O.compress_segments(O.SCHEMES[s], g_row, e_row, segq, seed)[:2] for s in schemes]
+
+        t0 = time.perf_counter()
+        with ThreadPoolExecutor(max_workers=Wt) as ex:
+            msgs = list(ex.map(one_worker, rows))
+        for si in range(len(schemes)):
+            O.aggregate([m[si][0] for m in msgs], [m[si][1] for m in msgs], nq)
+        dtq = time.perf_counter() - t0
+        base["threads"] = {"value": Wt * nq * len(schemes) / dtq, "unit": UNIT, "cores": Wt, "kind": "oracle",
+                           "seconds": round(dtq, 2),
+                           "sample": f"{Wt} workers in {Wt} threads (host has {cores} cores), first {nq} elements "
+                                     f"of each, then one aggregate of the {Wt} messages per scheme"}
+    except Exception as ex_:                                    # the single-core figure stands on its own
+        base["threads"] = {"value": None, "note": f"not timed: {ex_}"}
+    return base
 
 
 def main():

@@ -99,9 +99,31 @@ int sc_profile_read(sc_ctx* ctx, double* h_ms, uint64_t* h_launches);
  * bracket of the threshold; if the exact counts show the bracket missed, it redoes
  * the selection with a multi-pass radix select.  Both give the same bits.  After
  * synchronising `stream` this fills h_counts[3] for the most recent top-k call:
- * (worker, segment) pairs served by [0] the radix select because the segment is
- * small, [1] the one-pass path, [2] the radix select after a missed bracket. */
+ * (worker, segment) pairs served by [0] the radix select in shared memory because the
+ * segment is short, [1] the one-pass path, [2] the radix select after a missed bracket. */
 int sc_topk_path_counts(sc_ctx* ctx, void* stream, uint32_t* h_counts);
+
+/* Instrumentation (no counterpart in the paper).  More about the most recent top-k call, after
+ * synchronising `stream`: h_counts[8] (HOST) = (worker, segment) pairs [0] served in shared memory
+ * (short segments), [1] served by the one-pass path, [2] redone by the radix select; of the large
+ * segments: [3] those for which the sample showed one massive key value (a "tie key": exact zeros of a
+ * sparse tensor, a constant tensor) whose elements are counted instead of listed, [4] those whose
+ * threshold turned out to BE that key (tie-key elements admitted by coordinate order); reasons for
+ * [2]: [5] a list overflowed, [6] the exact counts disproved the bracket, [7] too many candidates share
+ * the threshold's histogram bin. */
+int sc_topk_path_detail(sc_ctx* ctx, void* stream, uint32_t* h_counts);
+
+/* Instrumentation for tests of the bounded device-side waits (no counterpart in the paper).  The
+ * fall-back radix select is one kernel whose CTAs meet at grid-wide barriers and whose pack phase looks
+ * back at its predecessors' counts; both waits give up after a number of polls, record
+ * SC_ERR_TIMEOUT in the status word and let the kernel return.  sc_debug_set_poll_limits changes the
+ * two limits for later calls of this context (0 restores the default).  sc_debug_wait_probe launches a
+ * small kernel that runs one of the waits where what it waits for never arrives: which = 0, a barrier
+ * that expects one CTA more than the launch has; which = 1, a look-back at a count nobody publishes.
+ * The kernel returns when the limit is reached (set a small one first); sc_sync_status then reports
+ * SC_ERR_TIMEOUT. */
+int sc_debug_set_poll_limits(sc_ctx* ctx, uint32_t lookback_polls, uint32_t barrier_polls);
+int sc_debug_wait_probe(sc_ctx* ctx, int which, void* stream);
 
 /* Algorithm 1, accumulate + compress + residual lines, one worker, global scope.
  * grad[n] read-only; residual[n] in/out (reads e, writes e'); out_vals[k],

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsparsecomm.so")
 
 EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_set_gamma", "sc_scratch_bytes", "sc_launch_count",
-           "sc_topk_path_counts", "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
+           "sc_topk_path_counts", "sc_topk_path_detail", "sc_debug_set_poll_limits", "sc_debug_wait_probe", "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
            "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_aggregate_static", "sc_aggregate_apply",
            "sc_aggregate_apply_shared", "sc_step", "sc_step_host"]
 
@@ -63,6 +63,12 @@ def load_library() -> ctypes.CDLL:
     lib.sc_launch_count.restype = u64
     lib.sc_topk_path_counts.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sc_topk_path_counts.restype = ci
+    lib.sc_topk_path_detail.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.sc_topk_path_detail.restype = ci
+    lib.sc_debug_set_poll_limits.argtypes = [vp, ctypes.c_uint32, ctypes.c_uint32]
+    lib.sc_debug_set_poll_limits.restype = ci
+    lib.sc_debug_wait_probe.argtypes = [vp, ci, vp]
+    lib.sc_debug_wait_probe.restype = ci
     lib.sc_profile.argtypes = [vp, ci]
     lib.sc_profile.restype = ci
     lib.sc_profile_kinds.argtypes = []
@@ -184,6 +190,20 @@ class Context:
         out = (ctypes.c_uint32 * 3)()
         _check(self._lib.sc_topk_path_counts(self._h, _stream(stream), out), "sc_topk_path_counts")
         return tuple(out)
+
+    PATH_DETAIL = ("short", "one_pass", "radix_after_failure", "tie_key_seen", "ties_admitted",
+                   "failed_list_overflow", "failed_bracket", "failed_short_list")
+
+    def sc_topk_path_detail(self, stream=None) -> dict:
+        out = (ctypes.c_uint32 * 8)()
+        _check(self._lib.sc_topk_path_detail(self._h, _stream(stream), out), "sc_topk_path_detail")
+        return dict(zip(self.PATH_DETAIL, out))
+
+    def sc_debug_set_poll_limits(self, lookback_polls: int = 0, barrier_polls: int = 0) -> None:
+        _check(self._lib.sc_debug_set_poll_limits(self._h, lookback_polls, barrier_polls), "sc_debug_set_poll_limits")
+
+    def sc_debug_wait_probe(self, which: int, stream=None) -> None:
+        _check(self._lib.sc_debug_wait_probe(self._h, which, _stream(stream)), "sc_debug_wait_probe")
 
     def sc_profile(self, enable: bool) -> None:
         _check(self._lib.sc_profile(self._h, 1 if enable else 0), "sc_profile")

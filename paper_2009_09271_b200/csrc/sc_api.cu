@@ -11,10 +11,8 @@
 #include "../../include/sparsecomm.h"
 #include "sc_aggregate.cuh"
 #include "sc_common.cuh"
-#include "sc_pack.cuh"
 #include "sc_random.cuh"
-#include "sc_topk.cuh"
-#include "sc_topk_fast.cuh"
+#include "sc_topk_fallback.cuh"
 #include "sc_topk_tiny.cuh"
 
 using namespace sc;
@@ -34,19 +32,21 @@ struct sc_ctx {
     uint32_t* d_tiny_list = nullptr;      // [max_segments]: short segments, the <= TINY_SMALL_MAX ones first
     uint32_t tiny_small = 0, tiny_large = 0, tiny_large_max_n = 0;
     int occ_tiny_small = 1;
-    uint32_t* d_lists = nullptr;     // slow tiles | fast tiles | slow pack groups | fast pack groups (each max_tiles long)
-    uint32_t n_slow_tiles = 0, n_fast_tiles = 0, n_slow_groups = 0, n_fast_groups = 0;
-    uint32_t* d_hist = nullptr;
+    uint32_t* d_lists = nullptr;     // tiles of the large segments | their pack groups (each max_tiles long)
+    uint32_t n_fast_tiles = 0, n_fast_groups = 0;
+    uint32_t* d_hist = nullptr;      // radix histograms of the fall-back (cleared by the fall-back kernel itself)
     TopkState* d_state = nullptr;
     unsigned long long* d_desc = nullptr;
     unsigned long long* d_ticket = nullptr;
     uint32_t* d_mask = nullptr;
     uint32_t* d_bounds = nullptr;
     uint32_t* d_offsets = nullptr;   // per seed group / worker: exclusive kept-count prefix over tiles
-    // sampled-bracket top-k path
-    FastState* d_fstate = nullptr;
+    // sampled-bracket top-k path.  Everything that must start at zero in a top-k call lies in one block
+    // (one memset): counters and the barrier word, then the per-problem states, then the candidate histograms.
+    unsigned char* d_zero = nullptr;
+    size_t zero_bytes = 0;
+    FastState* d_fstate = nullptr;   // inside d_zero
     uint32_t* d_sample = nullptr;
-    uint32_t* d_cand_hist = nullptr;
     uint2* d_cand = nullptr;
     uint2* d_list2 = nullptr;
     uint32_t* d_tile_sure = nullptr;
@@ -55,19 +55,18 @@ struct sc_ctx {
     uint32_t* d_tile_ccnt = nullptr;
     uint32_t* d_tile_fbase = nullptr;
     uint32_t* d_tile_fcnt = nullptr;
+    uint32_t* d_tile_tie = nullptr;
     size_t max_main_grid = 0;            // CTAs of the top-k pass in the build chosen for the current table
     size_t main_grid_v[2] = {0, 0};      // [0]: three CTAs per SM, [1]: the two-CTA build
     int main_wide = 0;                   // 1: the current table uses the two-CTA build
     uint2* d_flagged = nullptr;      // grown on demand: its size depends on k
     size_t flagged_slots = 0;
-    uint32_t* d_nslow = nullptr;     // [0]: segments for the radix select, [1]: segments whose bracket missed
     size_t max_fast_per_worker = 0, max_cand_per_worker = 0;
     uint32_t last_topk_problems = 0; // (worker, segment) pairs of the most recent top-k call
-    uint32_t slow_segments = 0;      // segments of the cached table that take the radix-select path
     uint32_t max_sample_m = 0, fast_big = 0;
     float gamma = 1.0f;                  // step size of the accumulate line (sc_set_gamma)
-    uint32_t max_flag_cap = 0, max_cand_cap = 0;
-    int occ_main = 1, occ_main_wide = 1, occ_emit = 1, occ_emit_v[4] = {1, 1, 1, 1};
+    int occ_main = 1, occ_main_wide = 1, occ_emit_v[4] = {1, 1, 1, 1}, occ_fallback = 1;
+    uint32_t lookback_poll_limit = LOOKBACK_POLL_LIMIT, barrier_poll_limit = BARRIER_POLL_LIMIT;
     uint64_t* d_seeds = nullptr;
     int* d_status = nullptr;
 
@@ -79,7 +78,7 @@ struct sc_ctx {
     uint32_t epoch = 0;
     uint64_t launches = 0;
 
-    int occ_hist = 1, occ_refine = 1, occ_pack_topk = 1, occ_pack_mask = 1, occ_block = 1, occ_agg = 1, occ_agg_big = 1, occ_agg_warp = 1;
+    int occ_pack_mask = 1, occ_block = 1, occ_agg = 1, occ_agg_big = 1, occ_agg_warp = 1;
     int occ_agg_fine[5] = {1, 1, 1, 1, 1};
 
     // optional per-kernel timing (sc_profile)
@@ -103,7 +102,6 @@ struct sc_ctx {
 // segment) up to TINY_SMALL_MAX elements (the many very short tensors of a network keep several CTAs per SM),
 // a cluster of TINY_CTAS CTAs beyond.
 constexpr uint32_t TINY_SMALL_MAX = 4096;        // elements: 16 KB of shared memory
-constexpr uint32_t TINY_LARGE_MAX = FAST_MIN_N - 1;
 
 // Emit variants by the average number of flagged entries per tile: 8 or 16 lanes per tile for sparse slices
 // (4 or 2 tiles per warp side by side), the whole warp with 4 or 8 entries per lane for longer ones.
@@ -136,14 +134,12 @@ class DeviceGuard {
     bool set_ = false;
 };
 
-enum { KIND_HIST0 = 0, KIND_RESOLVE, KIND_REFINE, KIND_PACK_TOPK, KIND_SCATTER, KIND_MASK_COUNT, KIND_ROW_SCAN,
-       KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES, KIND_SAMPLE, KIND_BRACKET, KIND_MAIN,
-       KIND_CANDBIN, KIND_CANDFILTER, KIND_FINAL, KIND_TILECOUNT, KIND_EMIT, KIND_RESTORE, KIND_AGG_APPLY, KIND_TINY, KIND_COUNT };
-const char* const kKindNames[KIND_COUNT] = {"topk_hist0", "topk_resolve", "topk_refine", "pack_topk", "randk_scatter",
-                                            "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
-                                            "agg_tiles", "topk_sample", "topk_bracket", "topk_main", "topk_candbin",
-                                            "topk_candfilter", "topk_final", "topk_tilecount", "topk_emit", "topk_restore",
-                                            "agg_apply", "topk_tiny"};
+enum { KIND_SCATTER = 0, KIND_MASK_COUNT, KIND_ROW_SCAN, KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES,
+       KIND_AGG_WARP, KIND_AGG_FINE, KIND_AGG_APPLY, KIND_TINY, KIND_BRACKET, KIND_MAIN, KIND_RESOLVE, KIND_EMIT,
+       KIND_FALLBACK, KIND_COUNT };
+const char* const kKindNames[KIND_COUNT] = {"randk_scatter", "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
+                                            "agg_tiles", "agg_warp", "agg_fine", "agg_apply", "topk_tiny", "topk_bracket",
+                                            "topk_main", "topk_resolve", "topk_emit", "topk_fallback"};
 
 // Counts a kernel launch and, when profiling is on, brackets it with two events.
 class Launch {
@@ -185,10 +181,10 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     int main_wide = 0;
     size_t max_main_grid = 0;
     std::vector<SegEntry> h(nseg + 1);
-    std::vector<uint32_t> fast_list, lists[4], tiny_a, tiny_b;
+    std::vector<uint32_t> fast_list, lists[2], tiny_a, tiny_b;
     uint32_t tiny_max_n = 0;
     uint64_t tiles = 0, scat = 0, maskw = 0, msg = 0, end_prev = 0, groups = 0, cand = 0, flag = 0, smp = 0;
-    uint32_t fast_count = 0, slow_count = 0, max_m = 0, max_cap = 0;
+    uint32_t fast_count = 0, max_m = 0;
     // Which build of the top-k streaming pass serves this table: the two-CTA build when every large segment is
     // long (more tiles than the three-CTA build has CTAs) and the lists are sparse (at most 3 % flagged).
     {
@@ -238,26 +234,33 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             const uint64_t tiles_per_region = per_tile ? 1 : MAIN_GROUP * ((seg_tiles / MAIN_GROUP + 2 + regions - 1) / regions);
             const uint64_t cand_region = tiles_per_region * ((slack + seg_tiles - 1) / seg_tiles + 16);
             const uint64_t flag_region = tiles_per_region * ((g.k + slack + seg_tiles - 1) / seg_tiles + 16);
-            if (flag_region * regions > 0xFFFFFFFFull) return SC_ERR_RANGE;
+            // Behind the regions lies a pool from which a full region continues (elements above the bracket
+            // may crowd in a part of the segment: the dense tensors of a flat vector that is mostly zero rows).
+            // Its size covers any distribution of k flagged elements over the tiles; a CTA takes it in chunks.
+            const uint64_t chunk = per_tile ? 0 : std::min<uint64_t>(8192, std::max<uint64_t>(1024, 8 * ((g.k + slack) / seg_tiles)));
+            const uint64_t pool = g.k + g.n / 64 + 4096 + regions * chunk;
+            if (flag_region * regions + pool > 0xFFFFFFF0ull) return SC_ERR_RANGE;
             e.region_per_tile = per_tile ? 1u : 0u;
             e.cand_cap = (uint32_t)cand_region;
             e.flag_cap = (uint32_t)flag_region;
+            e.ext_begin = (uint32_t)(flag_region * regions);
+            e.ext_cap = (uint32_t)pool;
+            e.ext_chunk = (uint32_t)chunk;
             e.cand_begin = cand;
             e.flag_begin = flag;
-            cand += cand_region * regions;
-            flag += flag_region * regions;
+            e.cov_begin = cand + cand_region * regions;
+            e.cov_cap = (uint32_t)(slack / 2 + 4096);
+            cand += cand_region * regions + e.cov_cap;
+            flag += flag_region * regions + pool;
             max_m = std::max(max_m, e.sample_m);
-        } else if (g.n <= TINY_LARGE_MAX) {
+        } else {                                                       // short: served in shared memory
             (g.n <= TINY_SMALL_MAX ? tiny_a : tiny_b).push_back((uint32_t)s);
             tiny_max_n = std::max<uint32_t>(tiny_max_n, g.n <= TINY_SMALL_MAX ? 0u : (uint32_t)g.n);
-        } else {
-            ++slow_count;
         }
         h[s] = e;
-        const int which = e.fast ? 1 : 0;
-        const bool listed = e.fast || g.n > TINY_LARGE_MAX;            // short segments are served outside the tile lists
-        for (uint64_t t = 0; listed && t < seg_tiles; ++t) lists[which].push_back((uint32_t)(tiles + t));
-        for (uint64_t t = 0; listed && t < (seg_tiles + PACK_GROUP - 1) / PACK_GROUP; ++t) lists[2 + which].push_back((uint32_t)(groups + t));
+        // the fall-back walks the tiles (and pack groups) of the large segments only
+        for (uint64_t t = 0; e.fast && t < seg_tiles; ++t) lists[0].push_back((uint32_t)(tiles + t));
+        for (uint64_t t = 0; e.fast && t < (seg_tiles + PACK_GROUP - 1) / PACK_GROUP; ++t) lists[1].push_back((uint32_t)(groups + t));
         tiles += seg_tiles;
         groups += (seg_tiles + PACK_GROUP - 1) / PACK_GROUP;
         scat += (g.k + SCAT_CHUNK - 1) / SCAT_CHUNK;
@@ -298,12 +301,11 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     sentinel.scat_begin = (uint32_t)scat; sentinel.mask_word_begin = maskw; sentinel.grp_begin = (uint32_t)groups;
     h[nseg] = sentinel;
     SC_CUDA(cudaMemcpyAsync(c->d_segs, h.data(), sizeof(SegEntry) * (nseg + 1), cudaMemcpyHostToDevice, stream));
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 2; ++i)
         if (!lists[i].empty())
             SC_CUDA(cudaMemcpyAsync(c->d_lists + (size_t)i * c->max_tiles_per_worker, lists[i].data(),
                                     sizeof(uint32_t) * lists[i].size(), cudaMemcpyHostToDevice, stream));
-    c->n_slow_tiles = (uint32_t)lists[0].size(); c->n_fast_tiles = (uint32_t)lists[1].size();
-    c->n_slow_groups = (uint32_t)lists[2].size(); c->n_fast_groups = (uint32_t)lists[3].size();
+    c->n_fast_tiles = (uint32_t)lists[0].size(); c->n_fast_groups = (uint32_t)lists[1].size();
     c->tiny_small = (uint32_t)tiny_a.size(); c->tiny_large = (uint32_t)tiny_b.size(); c->tiny_large_max_n = tiny_max_n;
     tiny_a.insert(tiny_a.end(), tiny_b.begin(), tiny_b.end());
     if (!tiny_a.empty())
@@ -317,7 +319,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     L.cand_per_worker = cand; L.flag_per_worker = flag; L.sample_per_worker = smp; L.fast_per_worker = fast_count;
     c->layout = L;
     c->main_wide = main_wide; c->max_main_grid = max_main_grid;
-    c->slow_segments = slow_count; c->fast_big = big_count; c->max_sample_m = max_m; c->max_flag_cap = max_cap;
+    c->fast_big = big_count; c->max_sample_m = max_m;
     c->cached_segs.assign(segs, segs + nseg);
     c->cached_n = n;
     c->layout_valid = true;
@@ -380,16 +382,20 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
     const uint32_t P = (uint32_t)W * L.nseg;
 
     if (scheme == SC_TOPK) {
-        SC_CUDA(cudaMemsetAsync(c->d_hist, 0, (size_t)P * HIST_WORDS * sizeof(uint32_t), stream));
-        SC_CUDA(cudaMemsetAsync(c->d_fstate, 0, (size_t)P * sizeof(FastState), stream));
+        // one memset for everything that starts at zero: counters, barrier word, problem states, candidate histograms
+        const uint32_t PF = (uint32_t)W * L.fast_per_worker;           // fast (worker, segment) pairs
+        const size_t state_bytes = ((size_t)P * sizeof(FastState) + 15) & ~(size_t)15;
+        uint32_t* counters = reinterpret_cast<uint32_t*>(c->d_zero);
+        unsigned int* barrier = reinterpret_cast<unsigned int*>(c->d_zero + 16);
+        FastState* fstate = reinterpret_cast<FastState*>(c->d_zero + 64);
+        uint32_t* cand_hist = reinterpret_cast<uint32_t*>(c->d_zero + 64 + state_bytes);
+        SC_CUDA(cudaMemsetAsync(c->d_zero, 0, 64 + state_bytes + (size_t)PF * CAND_BINS * sizeof(uint32_t), stream));
+        c->d_fstate = fstate;
         c->last_topk_problems = P;
-        const uint32_t n_slow0 = (uint32_t)W * c->slow_segments;
-        const uint32_t counters[2] = {n_slow0, 0u};
-        SC_CUDA(cudaMemcpyAsync(c->d_nslow, counters, sizeof(counters), cudaMemcpyHostToDevice, stream));
         if (c->tiny_small || c->tiny_large) {                          // short segments: one CTA each, in shared memory
             TinyParams tp{};
             tp.L = L; tp.grads = grads; tp.residuals = residuals; tp.out_vals = out_vals; tp.out_idx = out_idx;
-            tp.state = c->d_fstate; tp.W = (uint32_t)W; tp.status = c->d_status;
+            tp.state = fstate; tp.W = (uint32_t)W; tp.status = c->d_status;
             Launch l(c, KIND_TINY, stream);
             if (c->tiny_small) {
                 tp.list = c->d_tiny_list; tp.count = c->tiny_small;
@@ -410,17 +416,13 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
             }
         }
         if (L.fast_per_worker) {
-            const uint32_t PF = (uint32_t)W * L.fast_per_worker;       // fast (worker, segment) pairs
             FastParams fp{};
             fp.L = L; fp.grads = grads; fp.residuals = residuals; fp.out_vals = out_vals; fp.out_idx = out_idx;
-            fp.state = c->d_fstate; fp.sample = c->d_sample; fp.cand_hist = c->d_cand_hist;
+            fp.state = fstate; fp.sample = c->d_sample; fp.cand_hist = cand_hist;
             fp.list2 = c->d_list2; fp.cand = c->d_cand; fp.tile_sure = c->d_tile_sure; fp.tile_csum = c->d_tile_csum; fp.tile_cbase = c->d_tile_cbase;
-            fp.tile_ccnt = c->d_tile_ccnt; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt;
+            fp.tile_ccnt = c->d_tile_ccnt; fp.tile_fbase = c->d_tile_fbase; fp.tile_fcnt = c->d_tile_fcnt; fp.tile_tie = c->d_tile_tie;
             fp.flagged = c->d_flagged; fp.offsets = c->d_offsets;
-            fp.n_slow = c->d_nslow; fp.n_failed = c->d_nslow + 1; fp.status = c->d_status; fp.total_items = items;
-            SC_CUDA(cudaMemsetAsync(c->d_cand_hist, 0, (size_t)W * L.fast_per_worker * CAND_BINS * sizeof(uint32_t), stream));
-            { Launch l(c, KIND_SAMPLE, stream);
-              topk_sample_kernel<<<dim3((uint32_t)((L.sample_per_worker / 8 + THREADS - 1) / THREADS), W), THREADS, 0, stream>>>(fp); }
+            fp.counters = counters; fp.status = c->d_status; fp.total_items = items;
             { Launch l(c, KIND_BRACKET, stream);
               const uint32_t big = c->fast_big, small = L.fast_per_worker - big;
               if (big) {                                               // clusters of BRACKET_CTAS CTAs, one per problem
@@ -437,19 +439,8 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               const uint64_t groups_of_tiles = (items + MAIN_GROUP - 1) / MAIN_GROUP;
               if (c->main_wide) topk_main_kernel<1><<<persistent_grid(c, c->occ_main_wide, groups_of_tiles), THREADS, 0, stream>>>(fp);
               else topk_main_kernel<3><<<persistent_grid(c, c->occ_main, groups_of_tiles), THREADS, 0, stream>>>(fp); }
-            { Launch l(c, KIND_CANDBIN, stream);
-              topk_candbin_kernel<<<PF, THREADS, 0, stream>>>(fp); }
-            { Launch l(c, KIND_CANDFILTER, stream);
-              topk_candfilter_kernel<<<(uint32_t)(((uint64_t)(items + TILES_PER_GROUP - 1) / TILES_PER_GROUP * 8 + THREADS - 1) / THREADS), THREADS, 0, stream>>>(fp); }
-            { Launch l(c, KIND_FINAL, stream);
-              topk_final_kernel<<<PF, THREADS, 0, stream>>>(fp); }
-            { Launch l(c, KIND_RESTORE, stream);
-              const uint32_t blocks = persistent_grid(c, c->occ_emit, (items + WARPS - 1) / WARPS);
-              topk_restore_kernel<<<blocks, THREADS, 0, stream>>>(fp); }
-            { Launch l(c, KIND_TILECOUNT, stream);
-              topk_tilecount_kernel<<<(items + THREADS - 1) / THREADS, THREADS, 0, stream>>>(fp); }
-            { Launch l(c, KIND_ROW_SCAN, stream);
-              if ((rc_scan = launch_row_scan(c->d_offsets, (uint32_t)W, L.tiles_per_worker, stream)) != SC_OK) return rc_scan; }
+            { Launch l(c, KIND_RESOLVE, stream);
+              topk_resolve_kernel<<<(items + FILTER_TILES_PER_CTA - 1) / FILTER_TILES_PER_CTA, THREADS, 0, stream>>>(fp); }
             { Launch l(c, KIND_EMIT, stream);
               // flagged entries per tile, on average (the list holds the kept elements and a few per cent more)
               const double per_tile = 1.05 * (double)L.K_total * TILE / (double)std::max<size_t>(L.n_total, 1);
@@ -461,42 +452,30 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               else if (v == 1) topk_emit_kernel<16, 4><<<blocks, THREADS, 0, stream>>>(fp);
               else if (v == 2) topk_emit_kernel<32, 4><<<blocks, THREADS, 0, stream>>>(fp);
               else topk_emit_kernel<32, 8><<<blocks, THREADS, 0, stream>>>(fp); }
+            // The fall-back: one cooperative launch, which returns at once unless some segment's bracket missed.
+            FallbackParams fb{};
+            fb.F = fp;
+            fb.K.L = L; fb.K.residuals = residuals; fb.K.out_vals = out_vals; fb.K.out_idx = out_idx;
+            fb.K.state = c->d_state; fb.K.fstate = fstate;
+            fb.K.wl = WorkList{c->d_lists + c->max_tiles_per_worker, counters, c->n_fast_groups, 0u};
+            if (++c->epoch >= (1u << 28)) {        // tags wrapped: forget every old word
+                SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), stream));
+                c->epoch = 1;
+            }
+            fb.K.epoch = c->epoch; fb.K.total_items = (uint32_t)W * c->n_fast_groups; fb.K.poll_limit = c->lookback_poll_limit;
+            fb.K.ticket = c->d_ticket; fb.K.desc = c->d_desc; fb.K.status = c->d_status;
+            fb.hist = c->d_hist; fb.rstate = c->d_state;
+            fb.tiles = WorkList{c->d_lists, counters, c->n_fast_tiles, 0u};
+            fb.W = (uint32_t)W; fb.poll_limit = c->barrier_poll_limit; fb.barrier = barrier;
+            { Launch l(c, KIND_FALLBACK, stream);
+              void* args[] = {&fb};
+              const uint32_t grid = (uint32_t)c->sm_count * (uint32_t)std::max(c->occ_fallback, 1);
+              SC_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(topk_fallback_kernel), dim3(grid), dim3(THREADS), args, 0, stream)); }
         }
-        // Radix select: once over the small segments (if any), once over the large ones, where the
-        // launch returns at once unless some segment's bracket missed.
-        WorkList lists[2];
-        lists[0] = WorkList{c->d_lists, c->d_nslow, c->n_slow_tiles, 0u};
-        lists[1] = WorkList{c->d_lists + c->max_tiles_per_worker, c->d_nslow + 1, c->n_fast_tiles, 0u};
-        for (int pass = 0; pass < 2; ++pass) {
-            if (!lists[pass].len) continue;
-            const uint32_t n_it = (uint32_t)W * lists[pass].len;
-            Launch l(c, KIND_HIST0, stream);
-            topk_hist0_kernel<<<persistent_grid(c, c->occ_hist, n_it), THREADS, 0, stream>>>(
-                L, grads, residuals, c->d_hist, c->d_fstate, lists[pass], n_it);
-        }
-        { Launch l(c, KIND_RESOLVE, stream);
-          topk_resolve_kernel<0><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
-        for (int pass = 0; pass < 2; ++pass) {
-            if (!lists[pass].len) continue;
-            const uint32_t n_it = (uint32_t)W * lists[pass].len;
-            Launch l(c, KIND_REFINE, stream);
-            topk_refine_kernel<1><<<persistent_grid(c, c->occ_refine, n_it), THREADS, 0, stream>>>(
-                L, residuals, c->d_hist, c->d_state, c->d_fstate, lists[pass], n_it);
-        }
-        { Launch l(c, KIND_RESOLVE, stream);
-          topk_resolve_kernel<1><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
-        for (int pass = 0; pass < 2; ++pass) {
-            if (!lists[pass].len) continue;
-            const uint32_t n_it = (uint32_t)W * lists[pass].len;
-            Launch l(c, KIND_REFINE, stream);
-            topk_refine_kernel<2><<<persistent_grid(c, c->occ_refine, n_it), THREADS, 0, stream>>>(
-                L, residuals, c->d_hist, c->d_state, c->d_fstate, lists[pass], n_it);
-        }
-        { Launch l(c, KIND_RESOLVE, stream);
-          topk_resolve_kernel<2><<<P, THREADS, 0, stream>>>(L, c->d_hist, c->d_state, c->d_fstate, c->d_nslow, c->d_status); }
-    } else {
-        SC_CUDA(cudaMemcpyAsync(c->d_seeds, h_seeds, sizeof(uint64_t) * W, cudaMemcpyHostToDevice, stream));
+        SC_CUDA(cudaGetLastError());
+        return SC_OK;
     }
+    SC_CUDA(cudaMemcpyAsync(c->d_seeds, h_seeds, sizeof(uint64_t) * W, cudaMemcpyHostToDevice, stream));
 
     if (scheme == SC_RANDBLOCK || scheme == SC_RANDBLOCK_WRAP) {
         { Launch l(c, KIND_RANDBLOCK, stream);
@@ -531,27 +510,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
         return SC_OK;
     }
 
-    PackParams pp{};
-    pp.L = L; pp.grads = grads; pp.residuals = residuals; pp.out_vals = out_vals; pp.out_idx = out_idx;
-    pp.state = c->d_state; pp.mask = c->d_mask; pp.mask_per_worker = 0u;
-    pp.fstate = c->d_fstate;
-    pp.ticket = c->d_ticket; pp.desc = c->d_desc; pp.status = c->d_status;
-    for (int pass = 0; pass < 2; ++pass) {
-        const uint32_t len = pass == 0 ? c->n_slow_groups : c->n_fast_groups;
-        if (!len) continue;
-        pp.wl = WorkList{c->d_lists + (size_t)(2 + pass) * c->max_tiles_per_worker, c->d_nslow + pass, len, 0u};
-        SC_CUDA(cudaMemsetAsync(c->d_ticket, 0, sizeof(unsigned long long), stream));
-        if (++c->epoch >= (1u << 28)) {        // tags wrapped: forget every old word
-            SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), stream));
-            c->epoch = 1;
-        }
-        const uint32_t gitems = (uint32_t)W * len;
-        pp.epoch = c->epoch; pp.total_items = gitems;
-        Launch l(c, KIND_PACK_TOPK, stream);
-        pack_kernel<PACK_TOPK><<<persistent_grid(c, c->occ_pack_topk, gitems), THREADS, 0, stream>>>(pp);
-    }
-    SC_CUDA(cudaGetLastError());
-    return SC_OK;
+    return SC_ERR_INVALID;
 }
 
 // Tile of the dense output: the larger one halves the per-tile overhead, but only pays while all
@@ -598,7 +557,7 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
     { Launch l(c, KIND_AGG_BOUNDS, stream);
       agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
           idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds); }
-    { Launch l(c, KIND_AGG_TILES, stream);
+    { Launch l(c, by_warp ? KIND_AGG_WARP : fine >= 0 ? KIND_AGG_FINE : KIND_AGG_TILES, stream);
       if (by_warp) {
           const uint64_t nparts = (n + AGG_WARP_PART - 1) / AGG_WARP_PART;
           agg_warp_kernel<AGG_WARP_PART><<<persistent_grid(c, c->occ_agg_warp, (nparts + WARPS - 1) / WARPS), THREADS,
@@ -685,11 +644,12 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
     c->max_cand_per_worker = max_n / 32 + c->max_fast_per_worker * 16384;
     const size_t items_max = (size_t)max_W * c->max_tiles_per_worker;
     const size_t fastP = (size_t)max_W * c->max_fast_per_worker;
+    c->zero_bytes = 64 + ((P * sizeof(FastState) + 15) & ~(size_t)15) + fastP * CAND_BINS * sizeof(uint32_t);
     int rc = SC_OK;
     if ((rc = dev_alloc(c, &c->d_segs, (size_t)max_segments + 1)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_fast_list, (size_t)max_segments)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tiny_list, (size_t)max_segments)) == SC_OK &&
-        (rc = dev_alloc(c, &c->d_lists, 4 * c->max_tiles_per_worker)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_lists, 2 * c->max_tiles_per_worker)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_hist, P * HIST_WORDS)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_state, P)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_desc, (size_t)max_W * c->max_tiles_per_worker * 2)) == SC_OK &&
@@ -697,8 +657,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_mask, (size_t)max_W * c->max_mask_words)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_bounds, (size_t)max_W * (c->max_atiles + 1))) == SC_OK &&
         (rc = dev_alloc(c, &c->d_offsets, (size_t)max_W * (c->max_tiles_per_worker + 1))) == SC_OK &&
-        (rc = dev_alloc(c, &c->d_fstate, P)) == SC_OK &&
-        (rc = dev_alloc(c, &c->d_cand_hist, fastP * CAND_BINS)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_zero, c->zero_bytes)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_list2, fastP * LIST2_CAP)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_sure, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_csum, items_max)) == SC_OK &&
@@ -706,7 +665,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         (rc = dev_alloc(c, &c->d_tile_ccnt, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_fbase, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_tile_fcnt, items_max)) == SC_OK &&
-        (rc = dev_alloc(c, &c->d_nslow, 2)) == SC_OK &&
+        (rc = dev_alloc(c, &c->d_tile_tie, items_max)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_seeds, (size_t)max_W)) == SC_OK &&
         (rc = dev_alloc(c, &c->d_status, 1)) == SC_OK) {
         bool ok = cudaMemset(c->d_desc, 0, (size_t)max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long)) == cudaSuccess &&
@@ -716,17 +675,14 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         if (!ok) rc = SC_ERR_CUDA;
     }
     if (rc == SC_OK) {
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_hist, topk_hist0_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main, topk_main_kernel<3>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main_wide, topk_main_kernel<1>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_tiny_small, topk_tiny_kernel<1>, THREADS, TINY_SMALL_MAX * sizeof(float));
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit, topk_restore_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_fallback, topk_fallback_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[0], topk_emit_kernel<8, 4>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[1], topk_emit_kernel<16, 4>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[2], topk_emit_kernel<32, 4>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[3], topk_emit_kernel<32, 8>, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_refine, topk_refine_kernel<1>, THREADS, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_topk, pack_kernel<PACK_TOPK>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack_mask, randk_pack_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_block, randblock_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_agg, agg_tiles_kernel<ATILE>, THREADS, 0);
@@ -759,10 +715,10 @@ void sc_destroy(sc_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
     cudaFree(c->d_segs); cudaFree(c->d_fast_list); cudaFree(c->d_tiny_list); cudaFree(c->d_lists); cudaFree(c->d_hist); cudaFree(c->d_state); cudaFree(c->d_desc);
-    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_fstate);
-    cudaFree(c->d_cand_hist); cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_csum); cudaFree(c->d_tile_cbase);
-    cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt);
-    cudaFree(c->d_flagged); cudaFree(c->d_nslow); cudaFree(c->d_seeds); cudaFree(c->d_status);
+    cudaFree(c->d_ticket); cudaFree(c->d_mask); cudaFree(c->d_bounds); cudaFree(c->d_offsets); cudaFree(c->d_zero);
+    cudaFree(c->d_list2); cudaFree(c->d_tile_sure); cudaFree(c->d_tile_csum); cudaFree(c->d_tile_cbase);
+    cudaFree(c->d_tile_ccnt); cudaFree(c->d_tile_fbase); cudaFree(c->d_tile_fcnt); cudaFree(c->d_tile_tie);
+    cudaFree(c->d_flagged); cudaFree(c->d_seeds); cudaFree(c->d_status);
     cudaFree(c->d_stage_grads); cudaFree(c->d_stage_vals); cudaFree(c->d_stage_idx); cudaFree(c->d_stage_out);
     for (cudaEvent_t e : c->ev_worker) cudaEventDestroy(e);
     for (auto& r : c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -825,13 +781,60 @@ int sc_topk_path_counts(sc_ctx* c, void* stream, uint32_t* h_counts) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     std::vector<FastState> h(c->last_topk_problems);
     h_counts[0] = h_counts[1] = h_counts[2] = 0;
-    if (h.empty()) return SC_OK;
+    if (h.empty() || !c->d_fstate) return SC_OK;
     SC_CUDA(cudaMemcpyAsync(h.data(), c->d_fstate, h.size() * sizeof(FastState), cudaMemcpyDeviceToHost, st));
     SC_CUDA(cudaStreamSynchronize(st));
     for (const FastState& f : h) {
         if (f.path < 3) ++h_counts[f.path];
         else if (f.path == PATH_TINY) ++h_counts[0];                   // a short segment: radix select in shared memory
     }
+    return SC_OK;
+}
+
+int sc_topk_path_detail(sc_ctx* c, void* stream, uint32_t* h_counts) {
+    if (!c || !h_counts) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::vector<FastState> h(c->last_topk_problems);
+    for (int i = 0; i < 8; ++i) h_counts[i] = 0;
+    if (h.empty() || !c->d_fstate) return SC_OK;
+    SC_CUDA(cudaMemcpyAsync(h.data(), c->d_fstate, h.size() * sizeof(FastState), cudaMemcpyDeviceToHost, st));
+    SC_CUDA(cudaStreamSynchronize(st));
+    for (const FastState& f : h) {
+        if (f.path == PATH_TINY) ++h_counts[0];
+        else if (f.path == PATH_FAST) ++h_counts[1];
+        else if (f.path == PATH_FAILED) ++h_counts[2];
+        if (f.path == PATH_FAST || f.path == PATH_FAILED) {
+            if (f.tie_key != TIE_NONE) ++h_counts[3];
+            if (f.path == PATH_FAST && f.need_ties) ++h_counts[4];
+            if (f.path == PATH_FAILED && f.fail >= FAIL_OVERFLOW && f.fail <= FAIL_SHORT_LIST) ++h_counts[4 + f.fail];
+        }
+    }
+    return SC_OK;
+}
+
+int sc_debug_set_poll_limits(sc_ctx* c, uint32_t lookback_polls, uint32_t barrier_polls) {
+    if (!c) return SC_ERR_INVALID;
+    c->lookback_poll_limit = lookback_polls ? lookback_polls : LOOKBACK_POLL_LIMIT;
+    c->barrier_poll_limit = barrier_polls ? barrier_polls : BARRIER_POLL_LIMIT;
+    return SC_OK;
+}
+
+int sc_debug_wait_probe(sc_ctx* c, int which, void* stream) {
+    if (!c || (which != 0 && which != 1)) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PackParams k{};
+    if (++c->epoch >= (1u << 28)) {
+        SC_CUDA(cudaMemsetAsync(c->d_desc, 0, (size_t)c->max_W * c->max_tiles_per_worker * 2 * sizeof(unsigned long long), st));
+        c->epoch = 1;
+    }
+    k.epoch = c->epoch; k.poll_limit = c->lookback_poll_limit; k.desc = c->d_desc; k.status = c->d_status;
+    unsigned int* barrier = reinterpret_cast<unsigned int*>(c->d_zero + 16);
+    SC_CUDA(cudaMemsetAsync(barrier, 0, sizeof(unsigned int), st));
+    ++c->launches;
+    wait_probe_kernel<<<which == 0 ? 2 : 1, THREADS, 0, st>>>(k, barrier, which == 0 ? c->barrier_poll_limit : 0u, which);
+    SC_CUDA(cudaGetLastError());
     return SC_OK;
 }
 

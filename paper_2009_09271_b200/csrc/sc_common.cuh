@@ -38,6 +38,11 @@ struct SegEntry {
     uint32_t flag_cap;        // capacity of ONE region of the segment's flagged list
     uint32_t region_per_tile; // 1: one list region per tile (few tiles), 0: one per CTA of the main pass
     uint64_t sample_begin;    // first sample key of the segment inside a worker
+    uint32_t ext_begin;       // the regions are followed by a pool handed out on demand: its first slot ...
+    uint32_t ext_cap;         // ... and its size (a tile or CTA whose region is full continues there)
+    uint32_t ext_chunk;       // slots a CTA takes from the pool at a time (0: exactly what the tile needs)
+    uint32_t cov_cap;         // candidates that find their tile's slice full go, one by one, to an overflow list ...
+    uint64_t cov_begin;       // ... of this size, at this slot of the worker's candidate array
 };
 
 struct Layout {
@@ -82,6 +87,8 @@ enum { PATH_SLOW = 0,     // small segment: multi-pass radix select
        PATH_FAST = 1,     // bracket holds: single streaming pass + sparse emit
        PATH_FAILED = 2,   // bracket missed or a list overflowed: radix select on the parked p
        PATH_TINY = 3 };   // short segment: one CTA, everything in shared memory
+constexpr uint32_t TIE_NONE = 0xFFFFFFFFu;
+enum { FAIL_NONE = 0, FAIL_OVERFLOW = 1, FAIL_BRACKET = 2, FAIL_SHORT_LIST = 3 };
 struct FastState {
     uint32_t path;
     uint32_t lo, hi;       // bracket: key > hi is surely kept, key < lo surely dropped
@@ -93,7 +100,17 @@ struct FastState {
     uint32_t cnt2;         // candidates copied into the short list
     uint32_t T, icut;      // kept <=> key > T, or key == T and coordinate < icut
     uint32_t overflow;     // a list region was full during the main pass
-    uint32_t pad[3];
+    uint32_t tie_key;      // TIE_NONE, or lo - 1: a key value so frequent in the sample that its elements are
+                           // counted per tile instead of being listed (massive ties around the threshold)
+    uint32_t tie_total;    // elements with key == tie_key
+    uint32_t need_ties;    // how many of them are kept, lowest coordinates first (then T == tie_key)
+    uint32_t tiles_main;   // tiles of the segment the streaming pass has finished (the last CTA resolves the bin)
+    uint32_t tiles_filter; // tiles the candidate filter has finished (the last CTA finishes the problem)
+    uint32_t ext_used;     // slots handed out from the flagged list's extension pool
+    uint32_t fail;         // FAIL_*: why the one-pass path gave up
+    uint32_t expect2;      // entries the short list must hold (from the candidate histogram)
+    uint32_t cov_used;     // entries appended to the candidate overflow list (may exceed its capacity)
+    uint32_t pad[2];
 };
 
 constexpr uint32_t FAST_MIN_N = 1u << 16;

@@ -1,44 +1,37 @@
-// Stream-compaction pack + residual writeback (Algorithm 1: q^w = C(p), e' = p - q^w).
+// Fall-back stream-compaction pack + residual writeback (Algorithm 1: q^w = C(p), e' = p - q^w) for
+// segments whose sampled bracket missed; last phase of the fall-back kernel (sc_topk_fallback.cuh).
 //
-// One persistent kernel walks all (worker, segment, tile group) items in order, handing
+// The CTAs walk all (worker, segment, tile group) items of the failed segments in order, handing
 // out groups of PACK_GROUP tiles through an atomic ticket so that every group's
 // predecessors are already owned by running CTAs.
-//   phase 1  streams the group's tiles: forms or reads p, classifies every element, keeps
-//            only the 4-bit "kept" masks per quad (shared memory) and the per-warp counts;
+//   phase 1  streams the group's tiles: reads p (parked in the residual buffer), classifies every
+//            element against the threshold T, keeps only the 4-bit "kept" masks per quad (shared
+//            memory) and the per-warp counts;
 //   scan     block scan of the counts, then ONE chained-scan look-back per group (each
 //            group publishes its count, then sums its predecessors' words);
 //   phase 2  re-reads only the quads that hold kept elements (they are still in L2),
 //            writes values and coordinates at their ranks and zeroes them in the residual.
+// kept = key > T, plus the first r coordinates with key == T.
 // Grouping matters because a chained scan advances by at most 32 descriptors per L2 round
 // trip: with single 16 KB tiles that caps the pass near 1 TB/s, far below HBM.
 // Every wait on a predecessor is bounded; when it runs out the kernel records ST_TIMEOUT
 // in the status word and carries on with a zero prefix.
-//
-// PACK_TOPK: p is read from the residual buffer (parked there by the histogram pass);
-//            kept = key > T, plus the first r coordinates with key == T.
-// PACK_MASK: p = g + e is formed here and written to the residual buffer in phase 1;
-//            kept = membership bit of the coordinate.
 #pragma once
 #include "sc_common.cuh"
 
 namespace sc {
 
-enum { PACK_TOPK = 0, PACK_MASK = 1 };
-
 struct PackParams {
     Layout L;
-    const float* grads;
     float* residuals;
     float* out_vals;
     uint32_t* out_idx;
-    const TopkState* state;          // PACK_TOPK
-    const FastState* fstate;         // segments already served by the sampled-bracket path are skipped
+    const TopkState* state;
+    const FastState* fstate;         // only segments whose bracket missed are served
     WorkList wl;                     // the pack groups this launch walks
-    const uint32_t* mask;            // PACK_MASK
-    uint32_t mask_per_worker;        // 1: worker w uses mask group w, 0: all use group 0
     uint32_t epoch;                  // tag of this launch inside the descriptor words
     uint32_t total_items;            // groups over all workers
-    uint32_t pad;
+    uint32_t poll_limit;             // polls after which a look-back gives up
     unsigned long long* ticket;      // zeroed before the launch
     unsigned long long* desc;        // two words per group
     int* status;
@@ -46,7 +39,7 @@ struct PackParams {
 
 constexpr uint32_t DESC_AGG = 1u, DESC_INC = 2u;
 constexpr unsigned long long DESC_VAL_MASK = (1ull << 34) - 1ull;
-constexpr uint32_t LOOKBACK_POLL_LIMIT = 1u << 21;
+constexpr uint32_t LOOKBACK_POLL_LIMIT = 1u << 21;   // default of PackParams::poll_limit
 
 __device__ inline void desc_store(unsigned long long* p, uint32_t epoch, uint32_t st, unsigned long long v) {
     *reinterpret_cast<volatile unsigned long long*>(p) = ((unsigned long long)((epoch << 2) | st) << 34) | v;
@@ -100,7 +93,7 @@ __device__ inline void lookback(const PackParams& P, uint32_t item, uint32_t fir
                 }
             }
             if (__all_sync(0xFFFFFFFFu, ready)) break;
-            if (++polls > LOOKBACK_POLL_LIMIT) {           // give up: report and stop waiting
+            if (++polls > P.poll_limit) {           // give up: report and stop waiting
                 if (lane == 0) atomicMin(P.status, ST_TIMEOUT);
                 ex0 = 0; ex1 = 0;
                 return;
@@ -132,26 +125,22 @@ __device__ inline void lookback(const PackParams& P, uint32_t item, uint32_t fir
 // [16 t, 16 t + 16) (four float4 loads of one 64-byte run), so that the rank of a kept
 // element is (kept in lower lanes, one warp scan per tile) + (kept bits below it in the
 // thread's own 16-bit mask).
-template <int MODE>
-__global__ void __launch_bounds__(THREADS)
-pack_kernel(PackParams P) {
+__device__ inline void pack_failed_segments(const PackParams& P) {
     constexpr int G = PACK_GROUP;
     constexpr int NCNT = G * WARPS;                // one count per (tile, warp)
     constexpr int EPL = NCNT / 32;                 // count entries per lane in the warp scan
     constexpr int BATCH = 4;                       // quads re-read together in phase 2
     constexpr int EPT = QUADS * 4;                 // elements per thread per tile
     static_assert(NCNT % 32 == 0 && G * QUADS <= 32 && EPT == 16, "table layout");
-    constexpr bool TOPK = MODE == PACK_TOPK;
     __shared__ uint32_t s_dec[5];
     __shared__ uint16_t s_abits[G][THREADS];                   // kept / above-threshold bits of 16 elements
-    __shared__ uint16_t s_tbits[TOPK ? G : 1][THREADS];        // tie bits
+    __shared__ uint16_t s_tbits[G][THREADS];                   // tie bits
     __shared__ uint16_t s_arank[G][THREADS];                   // kept elements in lower lanes, same tile
-    __shared__ uint16_t s_trank[TOPK ? G : 1][THREADS];
+    __shared__ uint16_t s_trank[G][THREADS];
     __shared__ uint32_t s_cnt[2][NCNT];
     __shared__ uint32_t s_grp_excl[2];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const Layout& L = P.L;
-    if (*P.wl.gate == 0u) return;
 
     while (true) {
         if (threadIdx.x == 0) {
@@ -173,24 +162,14 @@ pack_kernel(PackParams P) {
         const uint32_t item = s_dec[0];
         if (item == 0xFFFFFFFFu) break;
         const uint32_t w = s_dec[1], s = s_dec[2], gi = s_dec[3], ntl = s_dec[4];
-        { const uint32_t path = P.fstate[(size_t)w * L.nseg + s].path;
-          if (path == PATH_FAST || path == PATH_TINY) { __syncthreads(); continue; } }
+        if (__ldcg(&P.fstate[(size_t)w * L.nseg + s].path) != PATH_FAILED) { __syncthreads(); continue; }
         const SegEntry seg = L.segs[s];
         const size_t row = (size_t)w * L.n_total + seg.offset;
         float* e = P.residuals + row;
-        const float* g = P.grads + row;
         const uint32_t mis = misalign_of(e);
         const long long t0 = (long long)gi * G;
-
-        uint32_t T = 0, r = 0;
-        bool dual = false;
-        const uint32_t* mask = nullptr;
-        if (TOPK) {
-            const TopkState st = P.state[(size_t)w * L.nseg + s];
-            T = st.T; r = st.r; dual = st.dual != 0;
-        } else {
-            mask = P.mask + (P.mask_per_worker ? (size_t)w * L.mask_words_per_group : 0) + seg.mask_word_begin;
-        }
+        const uint32_t T = __ldcg(&P.state[(size_t)w * L.nseg + s].T), r = __ldcg(&P.state[(size_t)w * L.nseg + s].r);
+        const bool dual = __ldcg(&P.state[(size_t)w * L.nseg + s].dual) != 0;
 
         // ---- phase 1: stream, classify, rank inside the warp, count -------------------------
         uint32_t pend = 0;                       // bit gl*QUADS+j: this thread's quad holds a candidate
@@ -200,72 +179,20 @@ pack_kernel(PackParams P) {
             if (gl < ntl) {
                 const long long first = (t0 + gl) * TILE - mis;          // local index of the tile's first element
                 const long long mine = first + (long long)threadIdx.x * EPT;
-                if (first >= 0 && first + TILE <= (long long)seg.n) {   // whole tile inside the segment
-                    float4 q[QUADS];
-                    const float4* pe = reinterpret_cast<const float4*>(e + mine);
 #pragma unroll
-                    for (int j = 0; j < QUADS; ++j) q[j] = pe[j];
-                    if (!TOPK) {
-                        const float4* pg = reinterpret_cast<const float4*>(g + mine);
+                for (int j = 0; j < QUADS; ++j) {
+                    const long long base = mine + 4 * j;
+                    float p[4];
+                    const uint32_t valid = load_quad(e, base, seg.n, p);
 #pragma unroll
-                        for (int j = 0; j < QUADS; ++j) {
-                            const float4 gv = __ldcs(pg + j);
-                            q[j].x = accumulate(P.L.gamma, gv.x, q[j].x); q[j].y = accumulate(P.L.gamma, gv.y, q[j].y);
-                            q[j].z = accumulate(P.L.gamma, gv.z, q[j].z); q[j].w = accumulate(P.L.gamma, gv.w, q[j].w);
-                        }
-                        float4* po = reinterpret_cast<float4*>(e + mine);
-#pragma unroll
-                        for (int j = 0; j < QUADS; ++j) po[j] = q[j];
-                        const uint32_t pos = (uint32_t)mine, a = pos >> 5, sh = pos & 31u;
-                        const uint32_t lo = __ldg(mask + a);
-                        const uint32_t hi = (sh > 16u) ? __ldg(mask + a + 1) : lo;
-                        ab16 = __funnelshift_r(lo, hi, sh) & 0xFFFFu;
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < QUADS; ++j) {
-                            const float v[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                const uint32_t key = key_of(v[c]);
-                                if (dual) {
-                                    ab16 |= (uint32_t)(key > T) << (4 * j + c);
-                                    tb16 |= (uint32_t)(key == T) << (4 * j + c);
-                                } else {
-                                    ab16 |= (uint32_t)(key >= T) << (4 * j + c);
-                                }
-                            }
-                        }
-                    }
-                } else {                                                   // ragged first / last tile
-#pragma unroll
-                    for (int j = 0; j < QUADS; ++j) {
-                        const long long base = mine + 4 * j;
-                        float p[4];
-                        const uint32_t valid = load_quad(e, base, seg.n, p);
-                        if (!TOPK) {
-                            float gv[4];
-                            load_quad_stream(g, base, seg.n, gv);
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) p[c] = accumulate(P.L.gamma, gv[c], p[c]);
-                            if (valid) store_quad(e, base, valid, p);
-#pragma unroll
-                            for (int c = 0; c < 4; ++c)
-                                if ((valid >> c) & 1u) {
-                                    const long long i = base + c;
-                                    ab16 |= ((__ldg(mask + (i >> 5)) >> (uint32_t)(i & 31)) & 1u) << (4 * j + c);
-                                }
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t key = key_of(p[c]);
+                        const uint32_t v = (valid >> c) & 1u;
+                        if (dual) {
+                            ab16 |= (v & (uint32_t)(key > T)) << (4 * j + c);
+                            tb16 |= (v & (uint32_t)(key == T)) << (4 * j + c);
                         } else {
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                const uint32_t key = key_of(p[c]);
-                                const uint32_t v = (valid >> c) & 1u;
-                                if (dual) {
-                                    ab16 |= (v & (uint32_t)(key > T)) << (4 * j + c);
-                                    tb16 |= (v & (uint32_t)(key == T)) << (4 * j + c);
-                                } else {
-                                    ab16 |= (v & (uint32_t)(key >= T)) << (4 * j + c);
-                                }
-                            }
+                            ab16 |= (v & (uint32_t)(key >= T)) << (4 * j + c);
                         }
                     }
                 }
@@ -283,14 +210,14 @@ pack_kernel(PackParams P) {
                 }
                 s_arank[gl][threadIdx.x] = (uint16_t)(inc - __popc(ab16));
                 if (lane == 31u) s_cnt[0][gl * WARPS + warp] = inc;
-                if (TOPK && dual) {
+                if (dual) {
                     uint32_t tinc = __popc(tb16);
 #pragma unroll
                     for (int d = 1; d < 32; d <<= 1) {
                         const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, tinc, d);
                         if (lane >= (uint32_t)d) tinc += t;
                     }
-                    s_trank[TOPK ? gl : 0][threadIdx.x] = (uint16_t)(tinc - __popc(tb16));
+                    s_trank[gl][threadIdx.x] = (uint16_t)(tinc - __popc(tb16));
                     if (lane == 31u) s_cnt[1][gl * WARPS + warp] = tinc;
                 }
             } else if (lane == 0) {
@@ -298,7 +225,7 @@ pack_kernel(PackParams P) {
                 s_cnt[1][gl * WARPS + warp] = 0;
             }
             s_abits[gl][threadIdx.x] = (uint16_t)ab16;
-            if (TOPK) s_tbits[gl][threadIdx.x] = (uint16_t)tb16;
+            s_tbits[gl][threadIdx.x] = (uint16_t)tb16;
         }
         __syncthreads();
 
@@ -376,12 +303,12 @@ pack_kernel(PackParams P) {
                 if (sl[b] < 0) continue;
                 const uint32_t gl = (uint32_t)sl[b] / QUADS, j = (uint32_t)sl[b] % QUADS;
                 const uint32_t ab16 = s_abits[gl][threadIdx.x];
-                const uint32_t tb16 = (TOPK && dual) ? s_tbits[gl][threadIdx.x] : 0u;
+                const uint32_t tb16 = dual ? s_tbits[gl][threadIdx.x] : 0u;
                 const uint32_t below = (1u << (4 * j)) - 1u;
                 uint32_t a_before = gex0 + s_cnt[0][gl * WARPS + warp] + s_arank[gl][threadIdx.x] + __popc(ab16 & below);
                 uint32_t t_before = 0;
-                if (TOPK && dual)
-                    t_before = gex1 + s_cnt[1][gl * WARPS + warp] + s_trank[TOPK ? gl : 0][threadIdx.x] + __popc(tb16 & below);
+                if (dual)
+                    t_before = gex1 + s_cnt[1][gl * WARPS + warp] + s_trank[gl][threadIdx.x] + __popc(tb16 & below);
                 const uint32_t ab = (ab16 >> (4 * j)) & 0xFu, tb = (tb16 >> (4 * j)) & 0xFu;
                 uint32_t kept = 0;
 #pragma unroll

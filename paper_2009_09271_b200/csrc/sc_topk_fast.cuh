@@ -3,26 +3,32 @@
 //
 // A radix select has to see every key before it knows the threshold, which costs extra
 // passes over HBM.  Here a small systematic sample of |g + e| brackets the threshold first:
-//   sample   m keys per (worker, segment); two order statistics of the sample, six standard
-//            deviations either side of rank k m / n, give [lo, hi] with
-//            count(key > hi) <= k <= count(key >= lo) except with negligible probability;
+//   bracket  m keys per (worker, segment) are read from evenly spaced 32-byte sectors; two order
+//            statistics of the sample, six standard deviations either side of rank k m / n, give
+//            [lo, hi] with count(key > hi) <= k <= count(key >= lo) except with negligible
+//            probability.  A key value that holds a large share of the sample at the lower order
+//            statistic (exact zeros of a sparse gradient, a constant tensor) becomes the "tie key":
+//            its elements are counted per tile instead of being listed;
 //   main     the streaming pass forms p = g + e and writes the residual at once: 0 for the
 //            "sure" elements (key > hi), p for the rest.  Every element with key >= lo is
 //            appended, in coordinate order inside its tile, to a "flagged" list (value,
 //            coordinate); the few candidates (lo <= key <= hi) also go to a candidate list
-//            and into a 2048-bin histogram;
-//   resolve  the candidate histogram pins the bin of the k-th key, the candidates of that
-//            bin are sorted in shared memory: exact threshold T and the coordinate cut for
-//            ties.  Every count is exact, so the result equals the plain definition; the
-//            sample only decides how much work that takes.  If the bracket is wrong (counts
-//            prove it) or a list overflows, the segment falls back to the radix select on
-//            the parked p;
-//   emit     per-tile kept counts -> exclusive scan -> a pass over the flagged list only:
-//            kept entries go to the message in ascending coordinate order, kept candidates
-//            are zeroed in the residual.  On a fall-back the sure values are first written
-//            back from the flagged list.
-// No CTA polls for another anywhere on this path; the bracket and the row scan use thread-block
-// clusters, whose CTAs meet at hardware cluster barriers only.
+//            and into a 2048-bin histogram.  The CTA that finishes a segment's last tile reads
+//            the histogram and pins the bin of the k-th key (exact counts decide whether the
+//            bracket held);
+//   resolve  the candidates of that bin are copied to a short list; the CTA that finishes a
+//            segment's last tile sorts it in shared memory (exact threshold T and the coordinate
+//            cut for ties), admits tie-key elements by coordinate order if the threshold is the
+//            tie key, and scans the per-tile kept counts into message offsets;
+//   emit     a pass over the flagged list only: kept entries go to the message in ascending
+//            coordinate order, kept candidates are zeroed in the residual; tiles that admit
+//            tie-key elements are re-read from the residual instead.
+// Every count is exact, so the result equals the plain definition; the sample only decides how
+// much work that takes.  If the bracket is wrong (counts prove it) or a list overflows, the
+// segment falls back to the radix select on the parked p.
+// No CTA polls for another anywhere on this path: the bracket uses a thread-block cluster, whose
+// CTAs meet at hardware cluster barriers only, and "the CTA that finishes last" is found with one
+// atomic counter per segment (nobody waits for it).
 #pragma once
 #include <cooperative_groups.h>
 
@@ -42,25 +48,40 @@ struct FastParams {
     uint2* list2;              // [W * fast_per_worker][LIST2_CAP]
     uint2* flagged;            // [W][flag_per_worker] (value bits, coordinate inside the segment)
     uint2* cand;               // [W][cand_per_worker] (key, coordinate) of the candidates, any order inside a tile
-    uint32_t* tile_sure;       // [W * tiles_per_worker] sure elements of the tile (zeroed before the pass)
+    uint32_t* tile_sure;       // [W * tiles_per_worker] sure elements of the tile
     uint32_t* tile_cbase;      // first candidate slot of the tile
     uint32_t* tile_ccnt;       // candidates of the tile
-    uint32_t* tile_csum;       // candidates above the threshold's bin (low half) and inside it (high half)
+    uint32_t* tile_csum;       // kept candidates of the tile (low half), candidates inside the threshold's bin (high
+                               // half); after the resolve step of a segment that admits ties: ties admitted in the tile
     uint32_t* tile_fbase;      // first flagged slot of the tile (0xFFFFFFFF: the list was full, nothing written)
     uint32_t* tile_fcnt;       // flagged elements of the tile
-    uint32_t* n_failed;        // segments whose bracket missed
-    uint32_t* offsets;         // [W][tiles_per_worker + 1]
-    uint32_t* n_slow;          // segments that need the radix-select path
+    uint32_t* tile_tie;        // elements equal to the tie key (written only for segments that have one)
+    uint32_t* counters;        // [0] segments whose bracket missed, [1] segments that admit tie-key elements
+    uint32_t* offsets;         // [W][tiles_per_worker + 1]: kept coordinates of the SEGMENT before the tile
     int* status;
     uint32_t total_items;
 };
 
-// The per-segment kernels of this path are launched over the fast segments only: block index
+// The per-segment launches of this path cover the fast segments only: problem index
 // f = w * fast_per_worker + fast_index, mapped to the segment through the layout's fast list.
 __device__ inline uint32_t fast_problem(const Layout& L, uint32_t f, uint32_t& w, uint32_t& s) {
     w = f / L.fast_per_worker;
     s = L.fast_list[f - w * L.fast_per_worker];
     return w * L.nseg + s;
+}
+
+// Reads that must see what other CTAs wrote or added with atomics: straight from L2.
+struct L2Words {
+    const uint32_t* p;
+    __device__ uint32_t operator[](uint32_t i) const { return __ldcg(p + i); }
+};
+__device__ inline FastState load_state_l2(const FastState* p) {
+    FastState st;
+    const uint4* src = reinterpret_cast<const uint4*>(p);
+    uint4* dst = reinterpret_cast<uint4*>(&st);
+#pragma unroll
+    for (int i = 0; i < (int)(sizeof(FastState) / 16); ++i) dst[i] = __ldcg(src + i);
+    return st;
 }
 
 // ---- shared helper: walk a histogram from its highest bin down to the bin that holds the
@@ -97,56 +118,33 @@ __device__ inline bool find_from_top(HistPtr h, uint32_t need, uint32_t* s_tmp /
     return bin != 0xFFFFFFFFu;
 }
 
-// ---- sample: one 32-byte sector (8 elements) of g and e per thread ----------------------
-__global__ void __launch_bounds__(THREADS)
-topk_sample_kernel(FastParams P) {
-    const Layout& L = P.L;
-    const uint32_t w = blockIdx.y;
-    const uint64_t pos = ((uint64_t)blockIdx.x * THREADS + threadIdx.x) * 8u;   // first key of this thread's sector
-    if (pos >= L.sample_per_worker) return;
-    // the samples of a worker's large segments lie one after the other, in fast-list order: find the segment
-    uint32_t f0 = 0, f1 = L.fast_per_worker - 1u;
-    while (f0 < f1) {
-        const uint32_t mid = (f0 + f1 + 1u) >> 1;
-        if (L.segs[L.fast_list[mid]].sample_begin <= pos) f0 = mid; else f1 = mid - 1u;
-    }
-    const SegEntry seg = L.segs[L.fast_list[f0]];
-    const uint32_t c = (uint32_t)((pos - seg.sample_begin) / 8u);      // sector of the segment's sample
-    const size_t row = (size_t)w * L.n_total + seg.offset;
-    const float* g = P.grads + row;
-    const float* e = P.residuals + row;
-    const uint32_t a0 = (8u - (uint32_t)((reinterpret_cast<uintptr_t>(e) >> 2) & 7u)) & 7u;   // first 32B-aligned element
-    const uint32_t sectors = (seg.n - a0) / 8u;
-    const uint32_t sidx = (uint32_t)(((uint64_t)c * sectors) / (seg.sample_m / 8u));
-    const size_t at = (size_t)a0 + (size_t)sidx * 8u;
-    const float4 e0 = *reinterpret_cast<const float4*>(e + at), e1 = *reinterpret_cast<const float4*>(e + at + 4);
-    const float4 g0 = *reinterpret_cast<const float4*>(g + at), g1 = *reinterpret_cast<const float4*>(g + at + 4);
-    uint4 k0, k1;
-    const float4 p0 = accumulate(L.gamma, g0, e0), p1 = accumulate(L.gamma, g1, e1);
-    k0.x = key_of(p0.x); k0.y = key_of(p0.y); k0.z = key_of(p0.z); k0.w = key_of(p0.w);
-    k1.x = key_of(p1.x); k1.y = key_of(p1.y); k1.z = key_of(p1.z); k1.w = key_of(p1.w);
-    uint4* out = reinterpret_cast<uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin + (size_t)c * 8u);
-    out[0] = k0; out[1] = k1;
-}
-
-// ---- bracket: two order statistics of the sample, to 21 bits -----------------------------------
-// One thread-block cluster of BRACKET_CTAS CTAs per problem: every CTA histograms its share of the
-// sample in its own shared memory, CTA 0 adds the shares up through distributed shared memory, walks
-// the total and hands the two bins back the same way; a second round refines them by ten more bits.
+// ---- bracket: sample the segment, take two order statistics of the sample ---------------------
+// One thread-block cluster of BRACKET_CTAS CTAs per problem (one CTA for small samples).  Every CTA
+// reads its share of the sample: one 32-byte sector (8 elements) of g and e per step and thread, from
+// evenly spaced positions; the keys are kept in global memory for the later rounds (each thread reads
+// back only what it wrote itself).  Round 1 histograms key bits 30..20 in shared memory, CTA 0 adds the
+// shares up through distributed shared memory, walks the total and hands the two bins back the same
+// way; round 2 refines them by ten more bits.  If the lower order statistic falls on a key prefix that
+// holds a large share of the sample, round 3 resolves the last ten bits: when ONE key value holds that
+// share it becomes the tie key (counted, not listed, by the streaming pass).
 // The cluster barriers are the hardware's; no CTA leaves before the last one (a peer's shared memory
-// must stay alive while it is read).
-// Segments with a small sample take one CTA each (C = 1: no cluster calls at all).  `first` and `count`
-// select a range of the fast list; the grid covers count problems of every worker.
+// must stay alive while it is read).  `first` and `count` select a range of the fast list; the grid
+// covers count problems of every worker.
 constexpr uint32_t BRACKET_CTAS = 8;
 constexpr uint32_t BRACKET_BIG_SAMPLE = 1u << 15;                      // samples from this size up take a cluster
+constexpr int SAMPLE_BATCH = 4;                                        // sectors of g and e in flight per thread
+// a key value is "massive" when it holds at least 1/256 of the sample (its elements would fill a good
+// part of the candidate list, which has room for n/32 entries) and at least 16 keys
+__device__ inline bool massive_in_sample(uint32_t cnt, uint32_t m) { return cnt >= 16u && (uint64_t)cnt * 256u >= m; }
+
 template <uint32_t C>
 __global__ void __launch_bounds__(THREADS)
 topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     namespace cg = cooperative_groups;
     __shared__ uint32_t h0[HIST0_BINS];
-    __shared__ uint32_t hA[1024], hB[1024];
+    __shared__ uint32_t hA[1024], hB[1024], hC[1024];
     __shared__ uint32_t s_tmp[WARPS + 4];
-    __shared__ uint32_t s_bins[4];                                     // binA, binB, needA, needB (valid in CTA 0)
+    __shared__ uint32_t s_bins[8];                                     // valid in CTA 0: binA, binB, needA, needB, round 3?, prefix B
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t rank = C > 1 ? cluster.block_rank() : 0u;
     const Layout& L = P.L;
@@ -155,10 +153,11 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     const uint32_t prob = fast_problem(L, (pidx / count) * L.fast_per_worker + first + pidx % count, w, s);
     const SegEntry seg = L.segs[s];
     const uint32_t m = seg.sample_m;
-    const uint4* smp = reinterpret_cast<const uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin);
-    // this CTA's share of the sample (in groups of four keys)
-    const uint32_t per = (m / 4u + C - 1u) / C;
-    const uint32_t i_begin = min(rank * per, m / 4u), i_end = min(i_begin + per, m / 4u);
+    uint4* smp = reinterpret_cast<uint4*>(P.sample + (size_t)w * L.sample_per_worker + seg.sample_begin);
+    // this CTA's share of the sample, in sectors of eight keys
+    const uint32_t S = m / 8u;
+    const uint32_t per = (S + C - 1u) / C;
+    const uint32_t c_begin = min(rank * per, S), c_end = min(c_begin + per, S);
     // ranks (from the top) that bracket the k-th largest of the segment
     const double q = (double)seg.k / (double)seg.n;
     const double centre = q * (double)m;
@@ -168,17 +167,48 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     const bool have_hi = j_hi >= 1, have_lo = j_lo <= (long long)m;
 
     for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) h0[b] = 0;
-    for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) { hA[b] = 0; hB[b] = 0; }
+    for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) { hA[b] = 0; hB[b] = 0; hC[b] = 0; }
     __syncthreads();
-    for (uint32_t i = i_begin + threadIdx.x; i < i_end; i += THREADS) {
-        const uint4 k = smp[i];
-        atomicAdd(&h0[k.x >> 20], 1u); atomicAdd(&h0[k.y >> 20], 1u);
-        atomicAdd(&h0[k.z >> 20], 1u); atomicAdd(&h0[k.w >> 20], 1u);
+    {   // ---- the sample: sector c of the sample is sector floor(c sectors / S) of the segment's aligned part
+        const size_t row = (size_t)w * L.n_total + seg.offset;
+        const float* g = P.grads + row;
+        const float* e = P.residuals + row;
+        const uint32_t a0 = (8u - (uint32_t)((reinterpret_cast<uintptr_t>(e) >> 2) & 7u)) & 7u;   // first 32-byte aligned element
+        const uint32_t sectors = (seg.n - a0) / 8u;
+        for (uint32_t c0 = c_begin + threadIdx.x; c0 < c_end; c0 += THREADS * SAMPLE_BATCH) {
+            float4 ev[SAMPLE_BATCH][2], gv[SAMPLE_BATCH][2];
+#pragma unroll
+            for (int u = 0; u < SAMPLE_BATCH; ++u) {
+                const uint32_t c = c0 + u * THREADS;
+                if (c < c_end) {
+                    const size_t at = (size_t)a0 + (size_t)(((uint64_t)c * sectors) / S) * 8u;
+                    ev[u][0] = *reinterpret_cast<const float4*>(e + at); ev[u][1] = *reinterpret_cast<const float4*>(e + at + 4);
+                    gv[u][0] = *reinterpret_cast<const float4*>(g + at); gv[u][1] = *reinterpret_cast<const float4*>(g + at + 4);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < SAMPLE_BATCH; ++u) {
+                const uint32_t c = c0 + u * THREADS;
+                if (c < c_end) {
+                    const float4 p0 = accumulate(L.gamma, gv[u][0], ev[u][0]), p1 = accumulate(L.gamma, gv[u][1], ev[u][1]);
+                    uint4 k0, k1;
+                    k0.x = key_of(p0.x); k0.y = key_of(p0.y); k0.z = key_of(p0.z); k0.w = key_of(p0.w);
+                    k1.x = key_of(p1.x); k1.y = key_of(p1.y); k1.z = key_of(p1.z); k1.w = key_of(p1.w);
+                    smp[2 * (size_t)c] = k0; smp[2 * (size_t)c + 1] = k1;
+                    atomicAdd(&h0[k0.x >> 20], 1u); atomicAdd(&h0[k0.y >> 20], 1u);
+                    atomicAdd(&h0[k0.z >> 20], 1u); atomicAdd(&h0[k0.w >> 20], 1u);
+                    atomicAdd(&h0[k1.x >> 20], 1u); atomicAdd(&h0[k1.y >> 20], 1u);
+                    atomicAdd(&h0[k1.z >> 20], 1u); atomicAdd(&h0[k1.w >> 20], 1u);
+                }
+            }
+        }
     }
-    if (C > 1) cluster.sync();
+    if (C > 1) cluster.sync(); else __syncthreads();
     // when k is so small that no sample rank lies safely above the threshold there is no "sure"
     // set (hi stays at the largest key); the candidate histogram then spans up to the largest
-    // sample key and everything above it shares the last bin
+    // sample key and everything above it shares the last bin.  The lower statistic is always
+    // located (the smallest sample key when no rank lies safely below the threshold): that is
+    // where a massive key value matters.
     if (rank == 0) {
         for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) {
             uint32_t v = h0[b];
@@ -186,26 +216,27 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
             h0[b] = v;
         }
         __syncthreads();
-        const uint32_t rankA = have_hi ? (uint32_t)j_hi : 1u;
+        const uint32_t rankA = have_hi ? (uint32_t)j_hi : 1u, rankB = have_lo ? (uint32_t)j_lo : m;
         uint32_t binA = 0, needA = 0, binB = 0, needB = 0, cnt = 0;
         find_from_top<HIST0_BINS>(h0, rankA, s_tmp, binA, needA, cnt);
-        if (have_lo) find_from_top<HIST0_BINS>(h0, (uint32_t)j_lo, s_tmp, binB, needB, cnt);
+        find_from_top<HIST0_BINS>(h0, rankB, s_tmp, binB, needB, cnt);
         if (threadIdx.x == 0) { s_bins[0] = binA; s_bins[1] = binB; s_bins[2] = needA; s_bins[3] = needB; }
     }
-    if (C > 1) cluster.sync();
-    if (C == 1) __syncthreads();
+    if (C > 1) cluster.sync(); else __syncthreads();
     const uint32_t* bins0 = C > 1 ? cluster.map_shared_rank(s_bins, 0) : s_bins;
     const uint32_t binA = bins0[0], binB = bins0[1];
-    for (uint32_t i = i_begin + threadIdx.x; i < i_end; i += THREADS) {
-        const uint4 k = smp[i];
-        const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
+    for (uint32_t c = c_begin + threadIdx.x; c < c_end; c += THREADS) {
+        const uint4 k0 = smp[2 * (size_t)c], k1 = smp[2 * (size_t)c + 1];
+        const uint32_t kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if ((kk[c] >> 20) == binA) atomicAdd(&hA[(kk[c] >> 10) & 1023u], 1u);
-            if (have_lo && (kk[c] >> 20) == binB) atomicAdd(&hB[(kk[c] >> 10) & 1023u], 1u);
+        for (int i = 0; i < 8; ++i) {
+            if ((kk[i] >> 20) == binA) atomicAdd(&hA[(kk[i] >> 10) & 1023u], 1u);
+            if ((kk[i] >> 20) == binB) atomicAdd(&hB[(kk[i] >> 10) & 1023u], 1u);
         }
     }
-    if (C > 1) cluster.sync();
+    if (C > 1) cluster.sync(); else __syncthreads();
+    uint32_t bin1A = 0, need2A = 0, bin1B = 0, need2B = 0;             // valid in CTA 0
+    bool okA = false, okB = false;
     if (rank == 0) {
         for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) {
             uint32_t va = hA[b], vb = hB[b];
@@ -216,21 +247,108 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
             hA[b] = va; hB[b] = vb;
         }
         __syncthreads();
-        const uint32_t needA = s_bins[2], needB = s_bins[3];
-        uint32_t top = 0x7FFFFFFFu, lo = 0u, bin1 = 0, need1 = 0, cnt = 0;
-        if (find_from_top<1024>(hA, needA, s_tmp, bin1, need1, cnt)) top = (binA << 20) | (bin1 << 10) | 1023u;
-        if (have_lo && find_from_top<1024>(hB, needB, s_tmp, bin1, need1, cnt)) lo = (binB << 20) | (bin1 << 10);
-        const uint32_t hi = have_hi ? top : 0x7FFFFFFFu;
-        if (lo > top) lo = top;                                        // (cannot happen; keeps the bracket sane)
+        uint32_t cntA = 0, cntB = 0;
+        okA = find_from_top<1024>(hA, s_bins[2], s_tmp, bin1A, need2A, cntA);
+        okB = find_from_top<1024>(hB, s_bins[3], s_tmp, bin1B, need2B, cntB);
         if (threadIdx.x == 0) {
-            const uint32_t width_m1 = top - lo;
+            s_bins[4] = (okB && massive_in_sample(cntB, m)) ? 1u : 0u;
+            s_bins[5] = (binB << 10) | bin1B;
+        }
+    }
+    if (C > 1) cluster.sync(); else __syncthreads();
+    const bool round3 = bins0[4] != 0u;                                // the same answer in every CTA of the cluster
+    if (round3) {
+        const uint32_t prefB = bins0[5];
+        for (uint32_t c = c_begin + threadIdx.x; c < c_end; c += THREADS) {
+            const uint4 k0 = smp[2 * (size_t)c], k1 = smp[2 * (size_t)c + 1];
+            const uint32_t kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if ((kk[i] >> 10) == prefB) atomicAdd(&hC[kk[i] & 1023u], 1u);
+        }
+        if (C > 1) cluster.sync(); else __syncthreads();
+    }
+    if (rank == 0) {
+        const uint32_t prefA = (binA << 10) | bin1A, prefB = (binB << 10) | bin1B;
+        uint32_t top = okA ? ((prefA << 10) | 1023u) : 0x7FFFFFFFu;
+        uint32_t lo = (have_lo && okB) ? (prefB << 10) : 0u;
+        uint32_t tie_key = TIE_NONE;
+        if (round3) {
+            for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) {
+                uint32_t v = hC[b];
+                for (uint32_t r = 1; r < C; ++r) v += cluster.map_shared_rank(hC, r)[b];
+                hC[b] = v;
+            }
+            __syncthreads();
+            uint32_t bin2 = 0, need3 = 0, mult = 0;
+            if (find_from_top<1024>(hC, need2B, s_tmp, bin2, need3, mult) && massive_in_sample(mult, m)) {
+                tie_key = (prefB << 10) | bin2;
+                lo = tie_key + 1u;                                     // listed: strictly above the tie key
+                uint32_t bin2a = 0, multa = 0;
+                if (okA && prefA == prefB && find_from_top<1024>(hC, need2A, s_tmp, bin2a, need3, multa))
+                    top = (prefA << 10) | bin2a;                       // the upper statistic, exactly (it may be the tie key itself)
+            }
+        }
+        const uint32_t hi = have_hi ? top : 0x7FFFFFFFu;
+        if (tie_key == TIE_NONE && lo > top) lo = top;                 // (cannot happen; keeps the bracket sane)
+        if (threadIdx.x == 0) {
+            const uint32_t width_m1 = top >= lo ? top - lo : 0u;
             const uint32_t bits = width_m1 ? 32u - (uint32_t)__clz((int)width_m1) : 0u;
             FastState st = {};
             st.path = PATH_FAST; st.lo = lo; st.hi = hi; st.shift = bits > 11u ? bits - 11u : 0u;
+            st.tie_key = tie_key;
             P.state[prob] = st;
         }
     }
     if (C > 1) cluster.sync();                                                    // peers stay until CTA 0 has read their histograms
+}
+
+// ---- the bin of the threshold (run by the CTA that finished the segment's last tile) ---------
+// Exact counts decide whether the bracket held: count(key > hi) <= k <= count(key >= lo) + ties.
+// Then either the k-th key lies among the candidates (its histogram bin is pinned here, the exact
+// key by the resolve step), or every candidate is kept and the rest are tie-key elements.
+__device__ __noinline__ void resolve_bin(const FastParams& P, uint32_t prob) {
+    __shared__ uint32_t s_tmp[WARPS + 4];
+    const Layout& L = P.L;
+    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    const SegEntry& seg = L.segs[s];
+    FastState st = load_state_l2(P.state + prob);
+    if (st.path != PATH_FAST) return;
+    const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
+    st.cand_total += min(st.cov_used, seg.cov_cap);                   // from here on: every listed candidate
+    const uint64_t listed = (uint64_t)st.sure_total + st.cand_total;
+    const uint64_t ties = st.tie_key != TIE_NONE ? st.tie_total : 0u;
+    uint32_t fail = FAIL_NONE;
+    if (st.overflow) fail = FAIL_OVERFLOW;
+    else if (st.sure_total > seg.k || (uint64_t)seg.k > listed + ties) fail = FAIL_BRACKET;
+    uint32_t bin = 0, need_in = 0, cnt = 0;
+    const uint32_t need = fail ? 0u : seg.k - st.sure_total;
+    const bool among_candidates = need != 0u && need <= st.cand_total;
+    if (!fail && among_candidates) {
+        const bool found = find_from_top<CAND_BINS>(L2Words{P.cand_hist + fidx * CAND_BINS}, need, s_tmp, bin, need_in, cnt);
+        if (!found) fail = FAIL_BRACKET;
+        else if (cnt > LIST2_CAP) fail = FAIL_SHORT_LIST;
+    }
+    if (threadIdx.x == 0) {
+        st.need2 = 0; st.need_ties = 0; st.cnt2 = 0; st.expect2 = 0; st.icut = 0;
+        if (fail) {
+            st.path = PATH_FAILED; st.fail = fail;
+            atomicAdd(P.counters, 1u);
+        } else if (need == 0) {
+            st.T = st.hi;                                              // exactly the sure elements are kept
+        } else if (among_candidates) {
+            st.lo2 = st.lo + (bin << st.shift);
+            const uint64_t top = (uint64_t)st.lo2 + (1ull << st.shift) - 1ull;
+            st.hi2 = bin == CAND_BINS - 1u ? st.hi : (uint32_t)min(top, (uint64_t)st.hi);
+            st.need2 = need_in;
+            st.expect2 = cnt;                                          // length of the short list (checked by the resolve step)
+        } else {                                                       // all candidates, and the first need_ties tie-key elements
+            st.T = st.tie_key;
+            st.need_ties = need - st.cand_total;
+            atomicAdd(P.counters + 1, 1u);
+        }
+        P.state[prob] = st;
+    }
 }
 
 // ---- main streaming pass ---------------------------------------------------------------
@@ -277,37 +395,43 @@ __device__ inline MainTile main_decode(const FastParams& P, uint32_t item) {
     return t;
 }
 // Two builds of the same code: MINB = 3 holds the kernel to 80 registers (three CTAs per SM), which is what
-// many short segments and dense lists want; MINB = 1 lets it take 97 (two CTAs per SM), which streams long
+// many short segments and dense lists want; MINB = 1 lets it take more (two CTAs per SM), which streams long
 // segments with sparse lists 1.4 % faster (350 M x 16 at 1 %: 10.45 against 10.65 ms; at 10 %: 12.1 against
 // 11.6 ms the other way round).  The host picks one per segment table.
 template <int MINB>
 __global__ void __launch_bounds__(THREADS, MINB)
-topk_main_kernel(FastParams P) {
+topk_main_kernel(const __grid_constant__ FastParams P) {
     __shared__ uint32_t sh[CAND_BINS];                                 // candidate histogram
     __shared__ __align__(16) float s_p[TILE];                          // the tile's p values, for the per-element work
     __shared__ uint16_t s_list[WARPS][512];                            // per warp: its flagged elements, in coordinate order
     __shared__ uint32_t s_wflag[2][WARPS];
-    __shared__ uint32_t s_cnt[3][2];                                   // per tile in flight: candidates appended, sure elements
+    __shared__ uint32_t s_cnt[3][4];                                   // per tile in flight: candidates appended, sure elements, tie-key elements
+    __shared__ uint32_t s_tot[6];                                      // of the current segment in this CTA: candidates, sure, ties, tiles; [4] its tile count
+    __shared__ uint32_t s_misc[3];                                     // broadcasts of thread 0
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t lt_mask = (1u << lane) - 1u;
     const uint32_t off0 = warp * 512u + lane * 4u;                     // this thread's quad of row 0 inside a tile
     // A segment's flagged and candidate lists are cut into regions: one per CTA of this kernel when the
     // segment has more tiles than CTAs (a tile's slots then follow from running counters), else one
-    // per tile.  Either way no CTA waits for another and the flagged list does not depend on scheduling.
+    // per tile.  A region that is full continues in a pool behind the regions, handed out in chunks through
+    // one atomic counter per segment (the only global atomic on the way, and only where elements of the
+    // bracket are much denser than on average).  Either way no CTA waits for another; where a tile's slice
+    // lies is recorded per tile, so the later steps do not depend on the order of the chunks.
     // Candidates are appended through a shared-memory counter, so their order inside a tile's slice is
     // arbitrary (all later uses count or sort them).  A tile's candidate and sure counts are final once
     // every warp has passed the next barrier; they are written out then ("pending" tile).
-    uint32_t run_flag = 0, run_cand = 0, tot_cand = 0, tot_sure = 0, fcap = 0, ccap = 0;
+    uint32_t cur_pos = 0, cur_end = 0, run_cand = 0, ccap = 0;
     for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) sh[b] = 0;
-    if (threadIdx.x < 6) s_cnt[threadIdx.x >> 1][threadIdx.x & 1] = 0;
+    if (threadIdx.x < 12) s_cnt[threadIdx.x >> 2][threadIdx.x & 3] = 0;
+    if (threadIdx.x < 6) s_tot[threadIdx.x] = 0;
     __syncthreads();
     long long cur_prob = -1;
     size_t cur_fidx = 0;
-    uint32_t lo = 0, hi = 0, shift = 0, parity = 0;
-    uint32_t slot3 = 0;                                                // counter pair of the current tile
+    uint32_t lo = 0, hi = 0, shift = 0, tie_key = TIE_NONE, parity = 0;
+    uint32_t slot3 = 0;                                                // counter triple of the current tile
     uint32_t pend_item = 0xFFFFFFFFu, pend_slot = 0, pend_room = 0;    // tile whose counts are not written yet
-    bool pend_accumulates = false;
+    bool pend_accumulates = false, pool_dry = false;
     const float gamma = L.gamma;
     const uint32_t group_step = (gridDim.x - 1u) * MAIN_GROUP + 1u;    // from a group's last tile to the next group's first
     MainTile T{};
@@ -328,24 +452,37 @@ topk_main_kernel(FastParams P) {
         const long long prob = T.have ? (long long)T.w * L.nseg + T.s : -2;
         if (prob != cur_prob && cur_prob >= 0) {                       // uniform over the CTA
             __syncthreads();                                           // the last tile's counts are final
-            if (pend_item != 0xFFFFFFFFu) {
-                const uint32_t c = min(s_cnt[pend_slot][0], pend_room), su = s_cnt[pend_slot][1];
-                if (threadIdx.x == 0) { P.tile_ccnt[pend_item] = c; P.tile_sure[pend_item] = su; }
-                tot_cand += c; tot_sure += su;
-                pend_item = 0xFFFFFFFFu;
+            if (threadIdx.x == 0 && pend_item != 0xFFFFFFFFu) {
+                const uint32_t c = min(s_cnt[pend_slot][0], pend_room), su = s_cnt[pend_slot][1], ti = s_cnt[pend_slot][2];
+                P.tile_ccnt[pend_item] = c; P.tile_sure[pend_item] = su;
+                if (tie_key != TIE_NONE) P.tile_tie[pend_item] = ti;
+                s_tot[0] += c; s_tot[1] += su; s_tot[2] += ti;
             }
-            if (threadIdx.x == 0) {
-                if (tot_sure) atomicAdd(&P.state[cur_prob].sure_total, tot_sure);
-                if (tot_cand) atomicAdd(&P.state[cur_prob].cand_total, tot_cand);
-            }
+            pend_item = 0xFFFFFFFFu;
             for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
                 const uint32_t c = sh[b];
                 if (c) { atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c); sh[b] = 0; }
             }
+            __threadfence();                                           // this thread's additions are in L2 before the count below
             __syncthreads();
-            if (threadIdx.x < 6) s_cnt[threadIdx.x >> 1][threadIdx.x & 1] = 0;
+            if (threadIdx.x == 0) {
+                FastState* st = P.state + cur_prob;
+                if (s_tot[1]) atomicAdd(&st->sure_total, s_tot[1]);
+                if (s_tot[0]) atomicAdd(&st->cand_total, s_tot[0]);
+                if (s_tot[2]) atomicAdd(&st->tie_total, s_tot[2]);
+                __threadfence();
+                const uint32_t before = atomicAdd(&st->tiles_main, s_tot[3]);
+                s_misc[0] = (before + s_tot[3] == s_tot[4]) ? 1u : 0u;  // this CTA finished the segment's last tile
+                s_tot[0] = 0; s_tot[1] = 0; s_tot[2] = 0; s_tot[3] = 0;
+            }
+            if (threadIdx.x < 12) s_cnt[threadIdx.x >> 2][threadIdx.x & 3] = 0;
             __syncthreads();
-            tot_sure = 0; run_flag = 0; run_cand = 0; tot_cand = 0;
+            if (s_misc[0]) {                                           // uniform: every other CTA's counts are in
+                __threadfence();
+                resolve_bin(P, (uint32_t)cur_prob);
+                __syncthreads();
+            }
+            run_cand = 0;
             cur_prob = -1;
         }
         if (!T.have) break;
@@ -355,8 +492,11 @@ topk_main_kernel(FastParams P) {
             cur_prob = prob;
             cur_fidx = (size_t)T.w * L.fast_per_worker + seg.fast_index;
             const FastState st = P.state[prob];
-            lo = st.lo; hi = st.hi; shift = st.shift;
-            fcap = seg.flag_cap; ccap = seg.cand_cap;                  // region sizes
+            lo = st.lo; hi = st.hi; shift = st.shift; tie_key = st.tie_key;
+            ccap = seg.cand_cap;                                       // region size
+            cur_pos = blockIdx.x * seg.flag_cap; cur_end = cur_pos + seg.flag_cap;
+            pool_dry = false;
+            if (threadIdx.x == 0) s_tot[4] = seg_tile_end - seg.tile_begin;
         }
         parity ^= 1u;
         slot3 = slot3 == 2u ? 0u : slot3 + 1u;
@@ -443,36 +583,68 @@ topk_main_kernel(FastParams P) {
         }
         // the previous tile's counts are final now (every warp has left its per-element loop)
         if (pend_item != 0xFFFFFFFFu) {
-            const uint32_t c = min(s_cnt[pend_slot][0], pend_room), su = s_cnt[pend_slot][1];
-            if (threadIdx.x == 0) { P.tile_ccnt[pend_item] = c; P.tile_sure[pend_item] = su; }
+            const uint32_t c = min(s_cnt[pend_slot][0], pend_room);
+            if (threadIdx.x == 0) {
+                const uint32_t su = s_cnt[pend_slot][1], ti = s_cnt[pend_slot][2];
+                P.tile_ccnt[pend_item] = c; P.tile_sure[pend_item] = su;
+                if (tie_key != TIE_NONE) P.tile_tie[pend_item] = ti;
+                s_tot[0] += c; s_tot[1] += su; s_tot[2] += ti;
+            }
             if (pend_accumulates) run_cand += c;
-            tot_cand += c; tot_sure += su;
         }
         // this CTA's regions of the two lists, and where this tile's entries go inside them
         const uint32_t tseg = T.lt - seg.tile_begin;                   // tile inside the segment
-        if (seg.region_per_tile) { run_flag = 0; run_cand = 0; }
+        if (seg.region_per_tile) { cur_pos = tseg * seg.flag_cap; cur_end = cur_pos + seg.flag_cap; run_cand = 0; }
+        bool fits = cur_pos + tflag <= cur_end;
+        if (!fits && !pool_dry) {                                      // uniform: the region is full, continue in the pool
+            if (threadIdx.x == 0) {
+                const uint32_t want = max(tflag, seg.ext_chunk);
+                const uint32_t got = atomicAdd(&P.state[prob].ext_used, want);
+                s_misc[1] = ((uint64_t)got + want <= seg.ext_cap) ? got : 0xFFFFFFFFu;
+                s_misc[2] = want;
+            }
+            __syncthreads();
+            const uint32_t got = s_misc[1];
+            if (got != 0xFFFFFFFFu) { cur_pos = seg.ext_begin + got; cur_end = cur_pos + s_misc[2]; fits = true; }
+            else pool_dry = true;
+        }
         const uint32_t region = seg.region_per_tile ? tseg : blockIdx.x;
-        const bool fits = run_flag + tflag <= fcap;
-        const uint32_t fbase = region * fcap + run_flag, cbase = region * ccap + run_cand;
+        const uint32_t fbase = cur_pos, cbase = region * ccap + run_cand;
         const uint32_t room = ccap - run_cand;                         // candidate slots left for this tile
         if (threadIdx.x == 0) {
             P.tile_fbase[item] = fits ? fbase : 0xFFFFFFFFu;
             P.tile_fcnt[item] = tflag;
             P.tile_cbase[item] = cbase;
-            if (!fits) P.state[prob].overflow = 1u;                    // a region is full: the segment falls back
+            if (!fits) P.state[prob].overflow = 1u;                    // the list is full: the segment falls back
             const uint32_t nxt = slot3 == 2u ? 0u : slot3 + 1u;        // counters of the tile after this one
-            s_cnt[nxt][0] = 0; s_cnt[nxt][1] = 0;
+            s_cnt[nxt][0] = 0; s_cnt[nxt][1] = 0; s_cnt[nxt][2] = 0;
+            s_tot[3] += 1u;
         }
         pend_item = item; pend_slot = slot3; pend_room = fits ? room : 0u; pend_accumulates = !seg.region_per_tile;
-        if (fits) run_flag += tflag;
+        if (fits) cur_pos += tflag;
+        if (tie_key != TIE_NONE) {                                     // uniform: count this thread's tie-key elements
+            uint32_t ties = 0;
+#pragma unroll
+            for (int j = 0; j < QUADS; ++j) {
+                const float4 p = *reinterpret_cast<const float4*>(sp + off0 + 128 * j);
+                const uint32_t c0 = (uint32_t)(mine + 128 * j);        // coordinates outside the segment wrap far beyond n
+                ties += (uint32_t)(key_of(p.x) == tie_key && c0 < seg.n) + (uint32_t)(key_of(p.y) == tie_key && c0 + 1u < seg.n) +
+                        (uint32_t)(key_of(p.z) == tie_key && c0 + 2u < seg.n) + (uint32_t)(key_of(p.w) == tie_key && c0 + 3u < seg.n);
+            }
+            ties = __reduce_add_sync(0xFFFFFFFFu, ties);
+            if (lane == 0 && ties) atomicAdd(&s_cnt[slot3][2], ties);
+        }
         if (fits && wflag) {
             // the tile's entries fit: write them (entry r of the warp's slice by lane r % 32: coalesced), zero
             // the sure ones in the residual (their values stay in the list, from where a fall-back restores
-            // them), append the candidates to the tile's slice and histogram them
+            // them; with a tie key the residual keeps p everywhere, so that the emit step can still tell a kept
+            // element from a tie), append the candidates to the tile's slice and histogram them
             uint2* flist = P.flagged + (size_t)T.w * L.flag_per_worker + seg.flag_begin + fbase + fwbase;
             uint2* clist = P.cand + (size_t)T.w * L.cand_per_worker + seg.cand_begin + cbase;
+            uint2* cover = P.cand + (size_t)T.w * L.cand_per_worker + seg.cov_begin;   // where candidates go when the slice is full
             const uint32_t first32 = (uint32_t)T.first + warp * 512u;
             const float* spw = sp + warp * 512u;
+            const bool zero_now = tie_key == TIE_NONE;
             uint32_t sure_w = 0;
             for (uint32_t r0 = 0; r0 < wflag; r0 += 32) {
                 const uint32_t r = r0 + lane;
@@ -484,7 +656,7 @@ topk_main_kernel(FastParams P) {
                 const bool sure = active && key > hi;
                 const bool cand = active && key <= hi;
                 if (active) flist[r] = make_uint2(__float_as_uint(v), coord);
-                if (sure) e[coord] = 0.0f;
+                if (sure && zero_now) e[coord] = 0.0f;
                 const uint32_t bs = __ballot_sync(0xFFFFFFFFu, sure);
                 const uint32_t bc = __ballot_sync(0xFFFFFFFFu, cand);
                 sure_w += __popc(bs);
@@ -496,10 +668,12 @@ topk_main_kernel(FastParams P) {
                         const uint32_t pos = base + __popc(bc & lt_mask);
                         if (pos < room) {
                             clist[pos] = make_uint2(key, coord);
-                            atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
-                        } else {
-                            P.state[prob].overflow = 1u;
+                        } else {                                       // rare: candidates crowd in this part of the segment
+                            const uint32_t gp = atomicAdd(&P.state[prob].cov_used, 1u);
+                            if (gp < seg.cov_cap) cover[gp] = make_uint2(key, coord);
+                            else P.state[prob].overflow = 1u;
                         }
+                        atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
                     }
                 }
             }
@@ -508,63 +682,26 @@ topk_main_kernel(FastParams P) {
     }
 }
 
-// ---- resolve 1: validity of the bracket, bin of the threshold (one CTA per problem) ------
-__global__ void __launch_bounds__(THREADS)
-topk_candbin_kernel(FastParams P) {
-    __shared__ uint32_t s_tmp[WARPS + 4];
-    const Layout& L = P.L;
-    uint32_t w, s;
-    const uint32_t prob = fast_problem(L, blockIdx.x, w, s);
-    const SegEntry seg = L.segs[s];
-    FastState st = P.state[prob];
-    if (st.path != PATH_FAST) return;
-    const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
-    bool ok = st.overflow == 0u && st.sure_total <= seg.k &&
-              (uint64_t)seg.k <= (uint64_t)st.sure_total + st.cand_total;
-    uint32_t bin = 0, need_in = 0, cnt = 0;
-    const uint32_t need = ok ? seg.k - st.sure_total : 0u;
-    if (ok && need) {
-        ok = find_from_top<CAND_BINS>(P.cand_hist + fidx * CAND_BINS, need, s_tmp, bin, need_in, cnt);
-        ok = ok && cnt <= LIST2_CAP;
-    }
-    if (threadIdx.x == 0) {
-        if (!ok) {
-            st.path = PATH_FAILED;
-            atomicAdd(P.n_slow, 1u);
-            atomicAdd(P.n_failed, 1u);
-        } else if (need == 0) {
-            st.need2 = 0; st.T = st.hi; st.icut = 0;                   // exactly the sure elements are kept
-        } else {
-            st.lo2 = st.lo + (bin << st.shift);
-            const uint64_t top = (uint64_t)st.lo2 + (1ull << st.shift) - 1ull;
-            st.hi2 = bin == CAND_BINS - 1u ? st.hi : (uint32_t)min(top, (uint64_t)st.hi);
-            st.need2 = need_in;
-            st.T = cnt;                                                // expected length of the short list (checked later)
-        }
-        st.cnt2 = 0;
-        P.state[prob] = st;
-    }
-}
-
 // ---- per-tile walks over the candidate slices ----------------------------------------------------
-// Eight lanes share TILES_PER_GROUP consecutive tiles.  The kernels below are bound by a chain of
+// Eight lanes share TILES_PER_GROUP consecutive tiles.  The filter below is bound by a chain of
 // dependent loads (slice length and base, then the slice), so a group first requests the placement
 // words of all its tiles, then the first eight candidates of every tile, and only then looks at
 // them: four tiles per group cut the number of such chains per launch by four.
 constexpr uint32_t TILES_PER_GROUP = 4;
+constexpr uint32_t FILTER_TILES_PER_CTA = (THREADS / 8) * TILES_PER_GROUP;
 struct CandSlice {                 // one tile's slice as seen by a lane of its group
     const uint2* list;             // nullptr: nothing to do for this tile
     uint32_t cnt, prob, w, lt;
+    bool counts;                   // the tile belongs to a segment on the one-pass path
     uint2 first;                   // entry `sub` of the slice (if sub < cnt)
 };
-template <bool NEED_FILTER>
 __device__ inline void cand_slices(const FastParams& P, uint32_t item0, uint32_t sub, CandSlice (&t)[TILES_PER_GROUP]) {
     const Layout& L = P.L;
     uint32_t base[TILES_PER_GROUP];
 #pragma unroll
     for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
         const uint32_t item = item0 + u;
-        t[u].list = nullptr; t[u].cnt = 0; base[u] = 0;
+        t[u].list = nullptr; t[u].cnt = 0; base[u] = 0; t[u].counts = false; t[u].prob = 0xFFFFFFFFu;
         if (item < P.total_items) { t[u].cnt = __ldg(P.tile_ccnt + item); base[u] = __ldg(P.tile_cbase + item); }
     }
 #pragma unroll
@@ -576,28 +713,176 @@ __device__ inline void cand_slices(const FastParams& P, uint32_t item0, uint32_t
         t[u].lt = item - t[u].w * L.tiles_per_worker;
         const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, t[u].lt);
         const SegEntry& seg = L.segs[s];
-        t[u].prob = t[u].w * L.nseg + s;
         if (!seg.fast) { t[u].cnt = 0; continue; }
+        t[u].prob = t[u].w * L.nseg + s;
         const FastState* st = P.state + t[u].prob;
-        if (st->path != PATH_FAST || (NEED_FILTER && st->need2 == 0)) { t[u].cnt = 0; continue; }
+        if (st->path != PATH_FAST) { t[u].cnt = 0; t[u].prob = 0xFFFFFFFFu; continue; }
+        t[u].counts = true;
+        if (st->need2 == 0) { t[u].cnt = 0; continue; }               // no candidate, or every candidate, is kept
         t[u].list = P.cand + (size_t)t[u].w * L.cand_per_worker + seg.cand_begin + base[u];
         if (sub < t[u].cnt) t[u].first = __ldg(t[u].list + sub);
     }
 }
 
-// ---- filter: copy the candidates of the threshold's bin into the short list ----------------------
+__device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint32_t icut) {
+    return key > T || (key == T && coord < icut);
+}
+
+// Last step of a segment (run by the CTA that filtered its last tile): exact threshold from the short
+// list, per-tile kept counts, message offsets.
+//   threshold among the candidates: the short list (the candidates of the threshold's histogram bin,
+//       at most LIST2_CAP) is sorted in shared memory, larger key first and lower coordinate first among
+//       equal keys; its first need2 entries are kept, which fixes T and the coordinate cut, and each of
+//       them adds one to its tile's count of kept candidates;
+//   threshold == tie key: every listed element is kept and the first need_ties tie-key elements in
+//       coordinate order: a running sum of the per-tile tie counts says how many each tile admits;
+//   then the kept counts of the segment's tiles are summed up into the tiles' first message slots.
+__device__ __noinline__ void finish_segment(const FastParams& P, uint32_t prob) {
+    __shared__ unsigned long long srt[LIST2_CAP];
+    __shared__ uint32_t s_scan[WARPS + 1];
+    const Layout& L = P.L;
+    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    const SegEntry seg = L.segs[s];
+    FastState st = load_state_l2(P.state + prob);
+    if (st.path != PATH_FAST) return;
+    const uint32_t ntiles = L.segs[s + 1].tile_begin - seg.tile_begin;
+    const size_t item0 = (size_t)w * L.tiles_per_worker + seg.tile_begin;
+    const bool admit = st.need_ties != 0u;
+    const uint32_t mis = misalign_of(P.residuals + (size_t)w * L.n_total + seg.offset);   // tiles lie on the 128-byte grid of the row
+    // candidates that did not fit their tile's slice (rare): those of the threshold's bin join the short list
+    const uint32_t ncov = min(st.cov_used, seg.cov_cap);
+    const uint2* cover = P.cand + (size_t)w * L.cand_per_worker + seg.cov_begin;
+    if (st.need2 && ncov) {
+        uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
+        for (uint32_t i = threadIdx.x; i < ncov; i += THREADS) {
+            const uint2 c = __ldcg(cover + i);
+            if (c.x >= st.lo2 && c.x <= st.hi2) {
+                const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
+                if (pos < LIST2_CAP) out[pos] = c;
+            }
+        }
+        __threadfence();
+        __syncthreads();
+        st.cnt2 = __ldcg(&P.state[prob].cnt2);
+    }
+    if (st.need2) {
+        const uint32_t cnt = st.cnt2;
+        if (cnt != st.expect2 || cnt > LIST2_CAP || st.need2 > cnt) {  // short list disagrees with the histogram
+            if (threadIdx.x == 0) {
+                st.path = PATH_FAILED; st.fail = FAIL_SHORT_LIST;
+                P.state[prob] = st;
+                atomicAdd(P.counters, 1u);
+            }
+            return;
+        }
+        uint32_t size = 1;
+        while (size < cnt) size <<= 1;
+        const uint2* in = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
+        for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
+            unsigned long long v = 0;                                   // padding sorts last
+            if (i < cnt) { const uint2 c = __ldcg(in + i); v = ((unsigned long long)c.x << 32) | (0xFFFFFFFFu - c.y); }
+            srt[i] = v;
+        }
+        __syncthreads();
+        // bitonic sort, descending: larger key first, equal keys: lower coordinate first
+        for (uint32_t k2 = 2; k2 <= size; k2 <<= 1) {
+            for (uint32_t j = k2 >> 1; j > 0; j >>= 1) {
+                for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
+                    const uint32_t ixj = i ^ j;
+                    if (ixj > i) {
+                        const unsigned long long a = srt[i], b = srt[ixj];
+                        const bool desc = (i & k2) == 0;
+                        if (desc ? (a < b) : (a > b)) { srt[i] = b; srt[ixj] = a; }
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        const unsigned long long v = srt[st.need2 - 1u];
+        st.T = (uint32_t)(v >> 32);
+        st.icut = (0xFFFFFFFFu - (uint32_t)v) + 1u;                    // coordinates below this are kept among the ties
+        if (st.icut == 0) st.icut = 0xFFFFFFFFu;                       // (coordinate 2^32-1 cannot occur: n < 2^32)
+        // the kept entries of the short list, counted into their tiles
+        for (uint32_t i = threadIdx.x; i < st.need2; i += THREADS) {
+            const uint32_t coord = 0xFFFFFFFFu - (uint32_t)srt[i];
+            atomicAdd(P.tile_csum + item0 + (coord + mis) / TILE, 1u);
+        }
+        __threadfence();
+        __syncthreads();
+    }
+    if (ncov && (admit || st.need2)) {                                 // kept overflow candidates, counted into their tiles
+        uint32_t* counts = admit ? P.tile_ccnt : P.tile_csum;          // (every candidate is kept when ties are admitted)
+        for (uint32_t i = threadIdx.x; i < ncov; i += THREADS) {
+            const uint2 c = __ldcg(cover + i);
+            if (admit || c.x > st.hi2) atomicAdd(counts + item0 + (c.y + mis) / TILE, 1u);
+        }
+        __threadfence();
+        __syncthreads();
+    }
+    // ---- kept count per tile, exclusive sum over the segment's tiles ------------------------------
+    constexpr uint32_t PER = 8;                                         // tiles per thread and round
+    uint32_t* off = P.offsets + (size_t)w * (L.tiles_per_worker + 1) + seg.tile_begin;
+    uint32_t kept_run = 0, tie_run = 0;
+    for (uint32_t base = 0; base < ntiles; base += THREADS * PER) {
+        const uint32_t t0 = base + threadIdx.x * PER;
+        uint32_t kept[PER], adm[PER], tsum = 0;
+#pragma unroll
+        for (uint32_t i = 0; i < PER; ++i) {
+            kept[i] = 0; adm[i] = 0;
+            if (t0 + i < ntiles) {
+                kept[i] = __ldcg(P.tile_sure + item0 + t0 + i);
+                if (admit) { kept[i] += __ldcg(P.tile_ccnt + item0 + t0 + i); adm[i] = __ldcg(P.tile_tie + item0 + t0 + i); }
+                else kept[i] += __ldcg(P.tile_csum + item0 + t0 + i) & 0xFFFFu;
+                tsum += adm[i];
+            }
+        }
+        if (admit) {                                                   // ties before each tile decide how many it admits
+            uint32_t total;
+            uint32_t before = tie_run + block_exclusive_scan(tsum, s_scan, &total);
+            tie_run += total;
+#pragma unroll
+            for (uint32_t i = 0; i < PER; ++i) {
+                const uint32_t room = st.need_ties > before ? st.need_ties - before : 0u;
+                const uint32_t a = min(adm[i], room);
+                before += adm[i];
+                kept[i] += a;
+                if (t0 + i < ntiles) P.tile_csum[item0 + t0 + i] = a;
+            }
+        }
+        uint32_t ksum = 0;
+#pragma unroll
+        for (uint32_t i = 0; i < PER; ++i) ksum += kept[i];
+        uint32_t total;
+        uint32_t ex = kept_run + block_exclusive_scan(ksum, s_scan, &total);
+        kept_run += total;
+#pragma unroll
+        for (uint32_t i = 0; i < PER; ++i) {
+            if (t0 + i < ntiles) off[t0 + i] = ex;
+            ex += kept[i];
+        }
+    }
+    if (threadIdx.x == 0) {
+        if (kept_run != seg.k) atomicMin(P.status, ST_DEVICE_CHECK);   // counts and k disagree
+        P.state[prob] = st;
+    }
+}
+
+// ---- resolve: copy the candidates of the threshold's bin into the short list; finish segments -----
 __global__ void __launch_bounds__(THREADS)
-topk_candfilter_kernel(FastParams P) {
+topk_resolve_kernel(const __grid_constant__ FastParams P) {
+    __shared__ uint32_t s_prob[FILTER_TILES_PER_CTA];
+    __shared__ uint32_t s_fin[FILTER_TILES_PER_CTA];
+    __shared__ uint32_t s_nfin;
     const Layout& L = P.L;
     const uint32_t sub = threadIdx.x & 7u;
     const uint32_t item0 = ((blockIdx.x * THREADS + threadIdx.x) >> 3) * TILES_PER_GROUP;
+    if (threadIdx.x == 0) s_nfin = 0;
     CandSlice t[TILES_PER_GROUP];
-    cand_slices<true>(P, item0, sub, t);
+    cand_slices(P, item0, sub, t);
 #pragma unroll
     for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
         // candidates above the threshold's bin are kept whatever the exact threshold turns out to be; those
-        // inside the bin go to the short list.  Both counts are left for the per-tile kept count, which then
-        // reads a tile's candidates again only if some of them lie inside the bin (a few thousand tiles at most).
+        // inside the bin go to the short list, and the segment's last step adds the kept ones to the count
         uint32_t above = 0, inbin = 0;
         if (t[u].list && t[u].cnt) {
             const FastState* stp = P.state + t[u].prob;
@@ -618,88 +903,32 @@ topk_candfilter_kernel(FastParams P) {
         both += __shfl_xor_sync(0xFFFFFFFFu, both, 1);
         both += __shfl_xor_sync(0xFFFFFFFFu, both, 2);
         both += __shfl_xor_sync(0xFFFFFFFFu, both, 4);
-        if (sub == 0u && item0 + u < P.total_items) P.tile_csum[item0 + u] = both;
+        if (sub == 0u) {
+            if (item0 + u < P.total_items) P.tile_csum[item0 + u] = both;
+            s_prob[(threadIdx.x >> 3) * TILES_PER_GROUP + u] = t[u].counts ? t[u].prob : 0xFFFFFFFFu;
+        }
     }
-}
-
-// ---- resolve 2: sort the short list, read off the threshold and the tie cut -------------------
-__global__ void __launch_bounds__(THREADS)
-topk_final_kernel(FastParams P) {
-    __shared__ unsigned long long srt[LIST2_CAP];
-    const Layout& L = P.L;
-    uint32_t w, s;
-    const uint32_t prob = fast_problem(L, blockIdx.x, w, s);
-    FastState st = P.state[prob];
-    if (st.path != PATH_FAST || st.need2 == 0) return;
-    const uint32_t cnt = st.cnt2;
-    if (cnt != st.T || cnt > LIST2_CAP || st.need2 > cnt) {            // short list disagrees with the histogram
-        if (threadIdx.x == 0) { P.state[prob].path = PATH_FAILED; atomicAdd(P.n_slow, 1u); atomicAdd(P.n_failed, 1u); }
-        return;
-    }
-    uint32_t size = 1;
-    while (size < cnt) size <<= 1;
-    const uint2* in = P.list2 + ((size_t)w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
-    for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
-        unsigned long long v = 0;                                       // padding sorts last
-        if (i < cnt) { const uint2 c = in[i]; v = ((unsigned long long)c.x << 32) | (0xFFFFFFFFu - c.y); }
-        srt[i] = v;
+    // ---- which segments did this CTA complete?  One addition per run of tiles of the same segment.
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x < FILTER_TILES_PER_CTA) {
+        const uint32_t p = s_prob[threadIdx.x];
+        if (p != 0xFFFFFFFFu && (threadIdx.x == 0 || s_prob[threadIdx.x - 1] != p)) {
+            uint32_t run = 1;
+            while (threadIdx.x + run < FILTER_TILES_PER_CTA && s_prob[threadIdx.x + run] == p) ++run;
+            const uint32_t s = p % L.nseg;
+            const uint32_t ntiles = L.segs[s + 1].tile_begin - L.segs[s].tile_begin;
+            const uint32_t before = atomicAdd(&P.state[p].tiles_filter, run);
+            if (before + run == ntiles) s_fin[atomicAdd(&s_nfin, 1u)] = p;
+        }
     }
     __syncthreads();
-    // bitonic sort, descending: larger key first, equal keys: lower coordinate first
-    for (uint32_t k2 = 2; k2 <= size; k2 <<= 1) {
-        for (uint32_t j = k2 >> 1; j > 0; j >>= 1) {
-            for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
-                const uint32_t ixj = i ^ j;
-                if (ixj > i) {
-                    const unsigned long long a = srt[i], b = srt[ixj];
-                    const bool desc = (i & k2) == 0;
-                    if (desc ? (a < b) : (a > b)) { srt[i] = b; srt[ixj] = a; }
-                }
-            }
-            __syncthreads();
-        }
+    const uint32_t nfin = s_nfin;
+    for (uint32_t i = 0; i < nfin; ++i) {                              // uniform over the CTA
+        __threadfence();
+        finish_segment(P, s_fin[i]);
+        __syncthreads();
     }
-    if (threadIdx.x == 0) {
-        const unsigned long long v = srt[st.need2 - 1u];
-        st.T = (uint32_t)(v >> 32);
-        st.icut = (0xFFFFFFFFu - (uint32_t)v) + 1u;                  // coordinates below this are kept among the ties
-        if (st.icut == 0) st.icut = 0xFFFFFFFFu;                      // (coordinate 2^32-1 cannot occur: n < 2^32)
-        P.state[prob] = st;
-    }
-}
-
-__device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint32_t icut) {
-    return key > T || (key == T && coord < icut);
-}
-
-// ---- kept count per tile = sure elements + chosen candidates -------------------------------------
-__global__ void __launch_bounds__(THREADS)
-topk_tilecount_kernel(FastParams P) {                                 // one thread per tile
-    const Layout& L = P.L;
-    const uint32_t item = blockIdx.x * THREADS + threadIdx.x;
-    if (item >= P.total_items) return;
-    const uint32_t sure = __ldg(P.tile_sure + item), both = __ldg(P.tile_csum + item);
-    const uint32_t w = item / L.tiles_per_worker;
-    const uint32_t lt = item - w * L.tiles_per_worker;
-    const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-    const SegEntry& seg = L.segs[s];
-    uint32_t kept = 0;
-    if (seg.fast) {
-        const FastState* st = P.state + (size_t)w * L.nseg + s;
-        if (st->path == PATH_FAST) {
-            kept = sure + (both & 0xFFFFu);
-            if (both >> 16) {                                          // candidates inside the threshold's bin: the exact rule
-                const uint32_t T = st->T, icut = st->icut, lo2 = st->lo2, hi2 = st->hi2;
-                const uint2* list = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + P.tile_cbase[item];
-                const uint32_t cnt = P.tile_ccnt[item];
-                for (uint32_t i = 0; i < cnt; ++i) {
-                    const uint2 c = list[i];
-                    if (c.x >= lo2 && c.x <= hi2) kept += fast_kept(c.x, c.y, T, icut) ? 1u : 0u;
-                }
-            }
-        }
-    }
-    P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt] = kept;
 }
 
 // ---- emit: G lanes per tile walk the tile's slice of the flagged list ----------------------------
@@ -707,6 +936,8 @@ topk_tilecount_kernel(FastParams P) {                                 // one thr
 // side by side; long slices take the whole warp and more entries per lane.  One batch covers
 // G x D entries.  (Loading the placement words two tiles ahead and asking L2 for the next slice
 // one tile ahead changed nothing: the kernel is not bound by its chain of dependent loads.)
+// Tiles that admit tie-key elements are skipped here and served by a second loop, in which a whole
+// warp re-reads the tile from the residual (it still holds p there) in coordinate order.
 template <int G, int D>
 __global__ void __launch_bounds__(THREADS)
 topk_emit_kernel(FastParams P) {
@@ -722,8 +953,8 @@ topk_emit_kernel(FastParams P) {
     const uint32_t rounds = (P.total_items + stride - 1) / stride;      // the same for every lane: ballots stay whole
     // per-(worker, segment) constants stay in registers while the group's tiles belong to the same one
     uint32_t cw = 0xFFFFFFFFu, cs = 0xFFFFFFFFu, c_tile_end = 0;        // cached worker, segment, end of its tile range
-    uint32_t T = 0, icut = 0, hi = 0, seg_k = 0, idx0 = 0, tile_begin = 0, off_begin = 0;
-    bool live = false;
+    uint32_t T = 0, icut = 0, hi = 0, seg_k = 0, idx0 = 0, tile_begin = 0;
+    bool live = false, admits = false;
     const uint2* flist0 = nullptr;
     float* e = nullptr;
     float* ovals = nullptr;
@@ -741,23 +972,19 @@ topk_emit_kernel(FastParams P) {
                 tile_begin = seg.tile_begin; c_tile_end = L.segs[cs + 1].tile_begin;
                 const FastState* st = P.state + (size_t)w * L.nseg + cs;
                 live = seg.fast && st->path == PATH_FAST;
-                T = st->T; icut = st->icut; hi = st->hi; seg_k = seg.k; idx0 = (uint32_t)seg.offset;
-                off_begin = P.offsets[(size_t)w * (L.tiles_per_worker + 1) + tile_begin];
+                admits = st->need_ties != 0u;
+                T = st->T; icut = st->icut; seg_k = seg.k; idx0 = (uint32_t)seg.offset;
+                hi = st->tie_key != TIE_NONE ? 0x7FFFFFFFu : st->hi;    // with a tie key the streaming pass zeroed nothing
                 flist0 = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
                 e = P.residuals + (size_t)w * L.n_total + seg.offset;
                 ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
                 oidx = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
             }
             if (live) {
-                // the four words that place this tile: independent loads, one round trip
-                const uint32_t* o = P.offsets + (size_t)w * (L.tiles_per_worker + 1) + lt;
+                // the words that place this tile: independent loads, one round trip
                 cnt = __ldg(P.tile_fcnt + item); base = __ldg(P.tile_fbase + item);
-                const uint32_t o0 = __ldg(o), o1 = __ldg(o + 1);
-                running = o0 - off_begin;                               // kept coordinates of the segment before this tile
-                if (cnt && (unsigned long long)running + (o1 - o0) > seg_k) {   // counts and k disagree: write nothing
-                    if (gl == 0) atomicMin(P.status, ST_DEVICE_CHECK);
-                    cnt = 0;
-                }
+                running = __ldg(P.offsets + (size_t)w * (L.tiles_per_worker + 1) + lt);   // kept coordinates of the segment before this tile
+                if (admits && __ldg(P.tile_csum + item) != 0u) cnt = 0;                  // served by the second loop
             }
         }
         const uint32_t maxcnt = __reduce_max_sync(0xFFFFFFFFu, cnt);
@@ -777,21 +1004,79 @@ topk_emit_kernel(FastParams P) {
                 const uint32_t bal = (__ballot_sync(0xFFFFFFFFu, sel) >> gshift) & gmask;
                 if (sel) {
                     const uint32_t r = pos + __popc(bal & lt_mask);
-                    ovals[r] = __uint_as_float(a[u].x);
-                    oidx[r] = idx0 + a[u].y;
-                    if (key <= hi) e[a[u].y] = 0.0f;                    // a kept candidate: the main pass left p there
+                    if (r < seg_k) {
+                        ovals[r] = __uint_as_float(a[u].x);
+                        oidx[r] = idx0 + a[u].y;
+                    } else {                                            // counts and k disagree
+                        atomicMin(P.status, ST_DEVICE_CHECK);
+                    }
+                    if (key <= hi) e[a[u].y] = 0.0f;                    // the streaming pass left p there
                 }
                 pos += __popc(bal);
+            }
+        }
+    }
+    // ---- tiles that admit tie-key elements (none at all unless some segment's threshold is its tie key) ------
+    if (__ldg(P.counters + 1) == 0u) return;
+    const uint32_t warps_total = gridDim.x * WARPS;
+    for (uint32_t it = blockIdx.x * WARPS + (threadIdx.x >> 5); it < P.total_items; it += warps_total) {
+        const uint32_t w = it / L.tiles_per_worker;
+        const uint32_t lt = it - w * L.tiles_per_worker;
+        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+        const SegEntry& seg = L.segs[s];
+        if (!seg.fast) continue;
+        const FastState* st = P.state + (size_t)w * L.nseg + s;
+        if (st->path != PATH_FAST || st->need_ties == 0u) continue;
+        const uint32_t adm = P.tile_csum[it];
+        if (adm == 0u) continue;
+        const uint32_t tkey = st->T;                                    // == tie key
+        float* er = P.residuals + (size_t)w * L.n_total + seg.offset;
+        float* ov = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
+        uint32_t* oi = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
+        const long long first = (long long)(lt - seg.tile_begin) * TILE - misalign_of(er);
+        uint32_t pos = P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt];
+        uint32_t ties_seen = 0;
+        for (uint32_t r = 0; r < TILE / 128; ++r) {                     // 128 coordinates per step, a quad per lane
+            const long long qb = first + 128 * r + 4 * lane;
+            float p[4];
+            const uint32_t valid = load_quad(er, qb, seg.n, p);
+            uint32_t above = 0, tie = 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t key = key_of(p[c]), v = (valid >> c) & 1u;
+                above |= (v & (uint32_t)(key > tkey)) << c;
+                tie |= (v & (uint32_t)(key == tkey)) << c;
+            }
+            const uint32_t tinc = warp_inclusive_scan(__popc(tie), lane);
+            uint32_t trank = ties_seen + tinc - __popc(tie);            // tie-key elements of the tile before this quad
+            uint32_t keep = above;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if ((tie >> c) & 1u) { if (trank < adm) keep |= 1u << c; ++trank; }
+            ties_seen += __shfl_sync(0xFFFFFFFFu, tinc, 31);
+            const uint32_t kinc = warp_inclusive_scan(__popc(keep), lane);
+            uint32_t slot = pos + kinc - __popc(keep);
+            pos += __shfl_sync(0xFFFFFFFFu, kinc, 31);
+            if (keep) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if ((keep >> c) & 1u) {
+                        if (slot < seg.k) { ov[slot] = p[c]; oi[slot] = (uint32_t)seg.offset + (uint32_t)(qb + c); }
+                        else atomicMin(P.status, ST_DEVICE_CHECK);
+                        ++slot;
+                        p[c] = 0.0f;
+                    }
+                }
+                store_quad(er, qb, valid, p);
             }
         }
     }
 }
 
 // ---- restore: a segment fell back; put the sure values back so that the residual holds p ------
-__global__ void __launch_bounds__(THREADS)
-topk_restore_kernel(FastParams P) {
+// (called by every CTA of the fall-back kernel before the radix select)
+__device__ inline void restore_failed_segments(const FastParams& P) {
     const Layout& L = P.L;
-    if (*P.n_failed == 0u) return;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warps_total = gridDim.x * WARPS;
     for (uint32_t item = blockIdx.x * WARPS + (threadIdx.x >> 5); item < P.total_items; item += warps_total) {
@@ -801,7 +1086,7 @@ topk_restore_kernel(FastParams P) {
         const SegEntry seg = L.segs[s];
         if (!seg.fast) continue;
         const FastState* st = P.state + (size_t)w * L.nseg + s;
-        if (st->path != PATH_FAILED) continue;
+        if (st->path != PATH_FAILED || st->tie_key != TIE_NONE) continue;   // with a tie key nothing was zeroed
         const uint32_t base = P.tile_fbase[item], cnt = P.tile_fcnt[item], hi = st->hi;
         if (base == 0xFFFFFFFFu || cnt == 0u) continue;                 // nothing was written, nothing was zeroed
         const uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + base;

@@ -61,6 +61,9 @@ def test_c4_lstm_shape_topk_ten_percent_full(scope):
     run_step_both(ctx, sc.SC_TOPK, g, e, segs, [0] * W)
     counts = ctx.sc_topk_path_counts()
     assert sum(counts) == W * len(segs)
+    assert counts[2] == 0, ctx.sc_topk_path_detail()        # massive ties and crowded tiles are served in one pass
+    if scope == "layerwise":
+        assert ctx.sc_topk_path_detail()["ties_admitted"] == 2 * W      # both embeddings: the threshold is zero
     ctx.close()
 
 

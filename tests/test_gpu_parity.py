@@ -243,20 +243,34 @@ def test_topk_large_segment_misaligned_rows_and_mixed_table(ctx):
     run_step_both(ctx, sc.SC_TOPK, g2, e2, segs, [0, 0], use="host")
 
 
-def test_topk_large_segment_degenerate_values_fall_back(ctx):
-    """Inputs on which a sampled bracket cannot isolate the threshold (all equal, mostly
-    zero, few distinct values): the exact result must not depend on that."""
+def test_topk_large_segment_massive_ties_in_one_pass(ctx):
+    """Inputs whose threshold sits on one massive key value (all equal, mostly zero, few distinct values):
+    the sample shows that value, its elements are counted per tile instead of listed, and the lowest
+    coordinates among them are admitted; no second pass over the segment."""
     n = BIG + 77
     e = torch.zeros(1, n)
     eq = torch.full((1, n), -0.5)
-    for k in (1, n // 100, n - 3):
+    for k in (1, n // 100, n - 3, n):
         run_step_both(ctx, sc.SC_TOPK, eq, e, [(0, n, k)], [0])
-        assert ctx.sc_topk_path_counts() == (0, 0, 1)           # every element ties: the bracket cannot hold
+        assert ctx.sc_topk_path_counts() == (0, 1, 0)
+        d = ctx.sc_topk_path_detail()
+        assert d["tie_key_seen"] == 1 and d["ties_admitted"] == 1, (k, d)
     z = torch.zeros(1, n)
     nz = torch.randperm(n, generator=torch.Generator().manual_seed(1))[: n // 20]
     z[0, nz] = rand(n // 20, 13)
-    for k in (n // 100, n // 20 - 1, n // 20, n // 20 + 1, n // 10):
+    for k in (n // 100, n // 20 - 1, n // 20, n // 20 + 1, n // 10, n // 2):
         run_step_both(ctx, sc.SC_TOPK, z, e, [(0, n, k)], [0])
+        assert ctx.sc_topk_path_counts() == (0, 1, 0), k
+        d = ctx.sc_topk_path_detail()
+        assert d["ties_admitted"] == (1 if k > n // 20 else 0), (k, d)
+    # zeros of both signs and a residual that cancels part of the gradient exactly
+    zz = z.clone()
+    zz[0, ::3] = -zz[0, ::3]
+    ee = torch.zeros(1, n)
+    ee[0, nz[: n // 40]] = -zz[0, nz[: n // 40]]                    # p becomes +0 or -0 there
+    for k in (n // 50, n // 30, n // 5):
+        run_step_both(ctx, sc.SC_TOPK, zz, ee, [(0, n, k)], [0])
+        assert ctx.sc_topk_path_counts() == (0, 1, 0), k
     ints = torch.randint(-3, 4, (1, n), generator=torch.Generator().manual_seed(2)).float()
     for k in (10, n // 100, n // 3):
         run_step_both(ctx, sc.SC_TOPK, ints, e, [(0, n, k)], [0])
@@ -264,6 +278,89 @@ def test_topk_large_segment_degenerate_values_fall_back(ctx):
     heavy[0, 17] = float("inf"); heavy[0, 4242] = float("nan")
     for k in (1, 2, 3, n // 1000):
         run_step_both(ctx, sc.SC_TOPK, heavy, e, [(0, n, k)], [0])
+
+
+def test_topk_ties_multiworker_segments_and_steps(ctx):
+    """Tie admission with several workers, several large segments (one of them starting misaligned), short
+    segments in between and the residual carried over three steps (zeros turn into earlier leftovers)."""
+    W = 3
+    sizes = [BIG + 5, 300, 2 * BIG + 4099, 70_000, 5000]
+    segs = wl.segment_table(sizes, 1, 8)
+    n = sum(sizes)
+    res = torch.zeros(W, n)
+    for t in range(3):
+        g = torch.zeros(W, n)
+        for w in range(W):
+            gen = torch.Generator().manual_seed(100 * t + w)
+            rows = torch.rand(n // 64 + 1, generator=gen) < 0.06      # runs of 64 non-zero coordinates, the rest exact zeros
+            mask = rows.repeat_interleave(64)[:n]
+            g[w] = torch.randn(n, generator=gen) * 1e-3 * mask
+        res = run_step_both(ctx, sc.SC_TOPK, g, res, segs, [t] * W, use=["step", "split", "step"][t])
+        assert ctx.sc_topk_path_counts()[2] == 0
+
+
+def test_topk_large_segment_two_massive_values_fall_back(ctx):
+    """A threshold that falls between two massive key values cannot be isolated by the sample (the upper one
+    would have to be listed as candidates and does not fit): the radix select serves the segment, and the
+    result must not depend on that."""
+    n = BIG + 77
+    e = torch.zeros(1, n)
+    v = torch.ones(1, n)
+    perm = torch.randperm(n, generator=torch.Generator().manual_seed(7))
+    c3 = n * 3 // 10
+    v[0, perm[:c3]] = -3.0
+    v[0, perm[c3:2 * c3]] = 2.0
+    for k in (c3 - 5, c3, c3 + 5):
+        run_step_both(ctx, sc.SC_TOPK, v, e, [(0, n, k)], [0])
+        assert ctx.sc_topk_path_counts() == (0, 0, 1), k
+        assert ctx.sc_topk_path_detail()["failed_list_overflow"] + ctx.sc_topk_path_detail()["failed_bracket"] == 1
+    # several workers, only one of which fails; a failed and a fine segment side by side
+    W = 3
+    g = torch.stack([v[0], rand(n, 31), rand(n, 32)])
+    run_step_both(ctx, sc.SC_TOPK, g, torch.zeros(W, n), [(0, n, c3 + 5)], [0] * W)
+    assert ctx.sc_topk_path_counts() == (0, 2, 1)
+    half = n // 2
+    run_step_both(ctx, sc.SC_TOPK, g, torch.zeros(W, n), [(0, half, half * 3 // 10), (half, n - half, 1000)], [0] * W)
+    assert ctx.sc_topk_path_counts()[0] == 0
+
+
+def test_topk_crowded_tiles_continue_in_the_pool(ctx):
+    """All large values in one stretch of the segment: the tiles there hold far more bracket elements than
+    their share of the list, and continue in the pool behind the regions (no fall-back)."""
+    n = 3 * BIG + 123
+    W = 2
+    g = torch.stack([rand(n, 41 + w, scale=1e-6) for w in range(W)])
+    g[:, BIG:BIG + BIG // 2] = torch.stack([rand(BIG // 2, 51 + w, scale=1.0) for w in range(W)])
+    e = torch.zeros(W, n)
+    for k in (n // 100, n // 10, BIG // 2 - 1000):
+        run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, k)], [0] * W)
+        assert ctx.sc_topk_path_counts() == (0, W, 0), k
+    # the same with one region per tile (a segment of few tiles) inside a table of several segments
+    segs = [(0, 2 * BIG, BIG // 3), (2 * BIG, n - 2 * BIG, 1000)]
+    run_step_both(ctx, sc.SC_TOPK, g, e, segs, [0] * W)
+    assert ctx.sc_topk_path_counts() == (0, 2 * W, 0)
+
+
+def test_bounded_waits_run_out_and_the_context_stays_usable(ctx):
+    """The fall-back kernel's two waits (grid barrier, look-back of the pack phase), run where what they wait
+    for never arrives: each gives up after the limit, the status word reports the time-out once, and the next
+    call is bit-exact again."""
+    n = BIG + 77
+    g, e = rand(n, 61).view(1, n), torch.zeros(1, n)
+    ctx.sc_debug_set_poll_limits(2000, 2000)
+    try:
+        for which in (0, 1):
+            ctx.sc_debug_wait_probe(which)
+            assert ctx.sc_sync_status() == -5
+            assert sc.strerror(-5) == "bounded device wait timed out"
+            assert ctx.sc_sync_status() == 0                              # reported once, then cleared
+            run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, n // 100)], [0])
+    finally:
+        ctx.sc_debug_set_poll_limits(0, 0)
+    # with the default limits the fall-back itself (barriers and look-backs that do complete) is bit-exact
+    v = torch.ones(1, n)
+    v[0, : n // 3] = 2.0
+    run_step_both(ctx, sc.SC_TOPK, v, e, [(0, n, n // 3 + 5)], [0])
 
 
 def test_aggregate_generic_shared_and_collisions(ctx):
