@@ -65,7 +65,7 @@ struct sc_ctx {
     uint32_t last_topk_problems = 0; // (worker, segment) pairs of the most recent top-k call
     uint32_t max_sample_m = 0, fast_big = 0;
     float gamma = 1.0f;                  // step size of the accumulate line (sc_set_gamma)
-    int occ_main = 1, occ_main_wide = 1, occ_emit_v[4] = {1, 1, 1, 1}, occ_fallback = 1;
+    int occ_main = 1, occ_main_wide = 1, occ_emit_v[4] = {1, 1, 1, 1}, occ_fallback = 1, occ_filter = 1;
     uint32_t lookback_poll_limit = LOOKBACK_POLL_LIMIT, barrier_poll_limit = BARRIER_POLL_LIMIT;
     uint64_t* d_seeds = nullptr;
     int* d_status = nullptr;
@@ -135,11 +135,11 @@ class DeviceGuard {
 };
 
 enum { KIND_SCATTER = 0, KIND_MASK_COUNT, KIND_ROW_SCAN, KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES,
-       KIND_AGG_WARP, KIND_AGG_FINE, KIND_AGG_APPLY, KIND_TINY, KIND_BRACKET, KIND_MAIN, KIND_RESOLVE, KIND_EMIT,
+       KIND_AGG_WARP, KIND_AGG_FINE, KIND_AGG_APPLY, KIND_TINY, KIND_BRACKET, KIND_MAIN, KIND_FILTER, KIND_FINISH, KIND_EMIT,
        KIND_FALLBACK, KIND_COUNT };
 const char* const kKindNames[KIND_COUNT] = {"randk_scatter", "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
                                             "agg_tiles", "agg_warp", "agg_fine", "agg_apply", "topk_tiny", "topk_bracket",
-                                            "topk_main", "topk_resolve", "topk_emit", "topk_fallback"};
+                                            "topk_main", "topk_filter", "topk_finish", "topk_emit", "topk_fallback"};
 
 // Counts a kernel launch and, when profiling is on, brackets it with two events.
 class Launch {
@@ -439,8 +439,19 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               const uint64_t groups_of_tiles = (items + MAIN_GROUP - 1) / MAIN_GROUP;
               if (c->main_wide) topk_main_kernel<1><<<persistent_grid(c, c->occ_main_wide, groups_of_tiles), THREADS, 0, stream>>>(fp);
               else topk_main_kernel<3><<<persistent_grid(c, c->occ_main, groups_of_tiles), THREADS, 0, stream>>>(fp); }
-            { Launch l(c, KIND_RESOLVE, stream);
-              topk_resolve_kernel<<<(items + FILTER_TILES_PER_CTA - 1) / FILTER_TILES_PER_CTA, THREADS, 0, stream>>>(fp); }
+            { Launch l(c, KIND_FILTER, stream);
+              const uint64_t batches = (items + FILTER_TILES_PER_CTA - 1) / FILTER_TILES_PER_CTA;
+              const uint32_t grid = persistent_grid(c, c->occ_filter, batches);
+              const uint32_t per_cta = (uint32_t)((batches + grid - 1) / grid) * FILTER_TILES_PER_CTA;
+              topk_filter_kernel<<<grid, THREADS, 0, stream>>>(fp, per_cta); }
+            { Launch l(c, KIND_FINISH, stream);                        // one cluster per large (worker, segment)
+              cudaLaunchConfig_t cfg = {};
+              cfg.gridDim = dim3(PF * FINISH_CTAS); cfg.blockDim = dim3(THREADS); cfg.stream = stream;
+              cudaLaunchAttribute attr;
+              attr.id = cudaLaunchAttributeClusterDimension;
+              attr.val.clusterDim.x = FINISH_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+              cfg.attrs = &attr; cfg.numAttrs = 1;
+              SC_CUDA(cudaLaunchKernelEx(&cfg, topk_finish_kernel, fp)); }
             { Launch l(c, KIND_EMIT, stream);
               // flagged entries per tile, on average (the list holds the kept elements and a few per cent more)
               const double per_tile = 1.05 * (double)L.K_total * TILE / (double)std::max<size_t>(L.n_total, 1);
@@ -679,6 +690,7 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_main_wide, topk_main_kernel<1>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_tiny_small, topk_tiny_kernel<1>, THREADS, TINY_SMALL_MAX * sizeof(float));
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_fallback, topk_fallback_kernel, THREADS, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_filter, topk_filter_kernel, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[0], topk_emit_kernel<8, 4>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[1], topk_emit_kernel<16, 4>, THREADS, 0);
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_emit_v[2], topk_emit_kernel<32, 4>, THREADS, 0);

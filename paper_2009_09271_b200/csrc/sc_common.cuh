@@ -104,8 +104,7 @@ struct FastState {
                            // counted per tile instead of being listed (massive ties around the threshold)
     uint32_t tie_total;    // elements with key == tie_key
     uint32_t need_ties;    // how many of them are kept, lowest coordinates first (then T == tie_key)
-    uint32_t tiles_main;   // tiles of the segment the streaming pass has finished (the last CTA resolves the bin)
-    uint32_t tiles_filter; // tiles the candidate filter has finished (the last CTA finishes the problem)
+    uint32_t pad0, pad1;
     uint32_t ext_used;     // slots handed out from the flagged list's extension pool
     uint32_t fail;         // FAIL_*: why the one-pass path gave up
     uint32_t expect2;      // entries the short list must hold (from the candidate histogram)

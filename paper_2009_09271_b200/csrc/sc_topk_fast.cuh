@@ -303,17 +303,22 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     if (C > 1) cluster.sync();                                                    // peers stay until CTA 0 has read their histograms
 }
 
-// ---- the bin of the threshold (run by the CTA that finished the segment's last tile) ---------
+// ---- the bin of the threshold --------------------------------------------------------------
 // Exact counts decide whether the bracket held: count(key > hi) <= k <= count(key >= lo) + ties.
 // Then either the k-th key lies among the candidates (its histogram bin is pinned here, the exact
-// key by the resolve step), or every candidate is kept and the rest are tie-key elements.
-__device__ __noinline__ void resolve_bin(const FastParams& P, uint32_t prob) {
+// key by the finish step), or every candidate is kept and the rest are tie-key elements.
+// Called by all threads of a CTA after the streaming pass has ended (all counts are final).  Every
+// CTA that needs a segment's bin works it out for itself (a walk over 2048 words); `owner` (the CTA
+// that holds the segment's first tile) also records it in the segment's state.
+struct BinInfo { uint32_t live, need2, lo2, hi2; };                   // live: the segment is still on the one-pass path
+__device__ __noinline__ BinInfo resolve_bin(const FastParams& P, uint32_t prob, bool owner) {
     __shared__ uint32_t s_tmp[WARPS + 4];
     const Layout& L = P.L;
     const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
     const SegEntry& seg = L.segs[s];
-    FastState st = load_state_l2(P.state + prob);
-    if (st.path != PATH_FAST) return;
+    FastState st = P.state[prob];
+    BinInfo out = {0u, 0u, 0u, 0u};
+    if (st.path != PATH_FAST) return out;
     const size_t fidx = (size_t)w * L.fast_per_worker + seg.fast_index;
     st.cand_total += min(st.cov_used, seg.cov_cap);                   // from here on: every listed candidate
     const uint64_t listed = (uint64_t)st.sure_total + st.cand_total;
@@ -325,30 +330,37 @@ __device__ __noinline__ void resolve_bin(const FastParams& P, uint32_t prob) {
     const uint32_t need = fail ? 0u : seg.k - st.sure_total;
     const bool among_candidates = need != 0u && need <= st.cand_total;
     if (!fail && among_candidates) {
-        const bool found = find_from_top<CAND_BINS>(L2Words{P.cand_hist + fidx * CAND_BINS}, need, s_tmp, bin, need_in, cnt);
+        const bool found = find_from_top<CAND_BINS>(P.cand_hist + fidx * CAND_BINS, need, s_tmp, bin, need_in, cnt);
         if (!found) fail = FAIL_BRACKET;
         else if (cnt > LIST2_CAP) fail = FAIL_SHORT_LIST;
     }
-    if (threadIdx.x == 0) {
-        st.need2 = 0; st.need_ties = 0; st.cnt2 = 0; st.expect2 = 0; st.icut = 0;
-        if (fail) {
-            st.path = PATH_FAILED; st.fail = fail;
-            atomicAdd(P.counters, 1u);
-        } else if (need == 0) {
-            st.T = st.hi;                                              // exactly the sure elements are kept
-        } else if (among_candidates) {
-            st.lo2 = st.lo + (bin << st.shift);
-            const uint64_t top = (uint64_t)st.lo2 + (1ull << st.shift) - 1ull;
-            st.hi2 = bin == CAND_BINS - 1u ? st.hi : (uint32_t)min(top, (uint64_t)st.hi);
-            st.need2 = need_in;
-            st.expect2 = cnt;                                          // length of the short list (checked by the resolve step)
-        } else {                                                       // all candidates, and the first need_ties tie-key elements
-            st.T = st.tie_key;
-            st.need_ties = need - st.cand_total;
-            atomicAdd(P.counters + 1, 1u);
-        }
-        P.state[prob] = st;
+    st.need2 = 0; st.need_ties = 0; st.cnt2 = 0; st.expect2 = 0; st.icut = 0;
+    if (fail) {
+        st.path = PATH_FAILED; st.fail = fail;
+    } else if (need == 0) {
+        st.T = st.hi;                                                  // exactly the sure elements are kept
+    } else if (among_candidates) {
+        st.lo2 = st.lo + (bin << st.shift);
+        const uint64_t top = (uint64_t)st.lo2 + (1ull << st.shift) - 1ull;
+        st.hi2 = bin == CAND_BINS - 1u ? st.hi : (uint32_t)min(top, (uint64_t)st.hi);
+        st.need2 = need_in;
+        st.expect2 = cnt;                                              // length of the short list (checked by the finish step)
+    } else {                                                           // all candidates, and the first need_ties tie-key elements
+        st.T = st.tie_key;
+        st.need_ties = need - st.cand_total;
     }
+    if (owner && threadIdx.x == 0) {
+        if (fail) atomicAdd(P.counters, 1u);
+        else if (st.need_ties) atomicAdd(P.counters + 1, 1u);
+        // only result words are written: other CTAs may be reading the counts above, or adding to the
+        // short-list counter, at this moment
+        FastState* dst = P.state + prob;
+        dst->path = st.path; dst->fail = st.fail; dst->need2 = st.need2;
+        dst->need_ties = st.need_ties; dst->expect2 = st.expect2; dst->icut = st.icut; dst->T = st.T;
+        dst->lo2 = st.lo2; dst->hi2 = st.hi2;
+    }
+    out.live = fail ? 0u : 1u; out.need2 = st.need2; out.lo2 = st.lo2; out.hi2 = st.hi2;
+    return out;
 }
 
 // ---- main streaming pass ---------------------------------------------------------------
@@ -372,7 +384,7 @@ __device__ inline uint32_t bytes_sum(uint32_t v) { return (v & 0xFFu) + ((v >> 8
 struct MainTile {                  // where a work item lives (uniform over the CTA)
     bool have, fast, full;
     uint32_t w, lt, s;
-    SegEntry seg;
+    uint32_t n, tile_begin;        // of the segment
     long long first;               // segment-local coordinate of the tile's first element
     const float* g;
     float* e;
@@ -385,15 +397,28 @@ __device__ inline MainTile main_decode(const FastParams& P, uint32_t item) {
     t.w = item / L.tiles_per_worker;
     t.lt = item - t.w * L.tiles_per_worker;
     t.s = (L.nseg == 1) ? 0u : find_by_tile(L, t.lt);
-    t.seg = L.segs[t.s];
-    t.fast = t.seg.fast != 0;
-    const size_t row = (size_t)t.w * L.n_total + t.seg.offset;
+    const SegEntry* seg = L.segs + t.s;
+    t.fast = seg->fast != 0;
+    t.n = seg->n; t.tile_begin = seg->tile_begin;
+    const size_t row = (size_t)t.w * L.n_total + seg->offset;
     t.g = P.grads + row;
     t.e = P.residuals + row;
-    t.first = (long long)(t.lt - t.seg.tile_begin) * TILE - misalign_of(t.e);
-    t.full = t.first >= 0 && t.first + TILE <= (long long)t.seg.n;
+    t.first = (long long)(t.lt - t.tile_begin) * TILE - misalign_of(t.e);
+    t.full = t.first >= 0 && t.first + TILE <= (long long)t.n;
     return t;
 }
+// What the per-element work of a tile needs to know about its (worker, segment): kept in shared memory
+// (written by thread 0 when the CTA enters the segment, read by everyone after the tile's barrier), so that
+// the streaming part of the loop has the registers to itself.
+struct MainSeg {
+    uint32_t hi, shift, tie_key, ccap;
+    uint32_t flag_cap, region_per_tile, ext_begin, ext_cap;
+    uint32_t ext_chunk, cov_cap, pad0, pad1;
+    uint2* flist;                  // the segment's flagged list of this worker
+    uint2* clist;                  // its candidate list
+    uint2* cover;                  // its candidate overflow list
+    uint32_t* hist;                // its candidate histogram
+};
 // Two builds of the same code: MINB = 3 holds the kernel to 80 registers (three CTAs per SM), which is what
 // many short segments and dense lists want; MINB = 1 lets it take more (two CTAs per SM), which streams long
 // segments with sparse lists 1.4 % faster (350 M x 16 at 1 %: 10.45 against 10.65 ms; at 10 %: 12.1 against
@@ -406,11 +431,11 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
     __shared__ uint16_t s_list[WARPS][512];                            // per warp: its flagged elements, in coordinate order
     __shared__ uint32_t s_wflag[2][WARPS];
     __shared__ uint32_t s_cnt[3][4];                                   // per tile in flight: candidates appended, sure elements, tie-key elements
-    __shared__ uint32_t s_tot[6];                                      // of the current segment in this CTA: candidates, sure, ties, tiles; [4] its tile count
+    __shared__ uint32_t s_tot[4];                                      // of the current segment in this CTA: candidates, sure, ties
     __shared__ uint32_t s_misc[3];                                     // broadcasts of thread 0
+    __shared__ MainSeg s_seg;
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const uint32_t lt_mask = (1u << lane) - 1u;
     const uint32_t off0 = warp * 512u + lane * 4u;                     // this thread's quad of row 0 inside a tile
     // A segment's flagged and candidate lists are cut into regions: one per CTA of this kernel when the
     // segment has more tiles than CTAs (a tile's slots then follow from running counters), else one
@@ -421,17 +446,16 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
     // Candidates are appended through a shared-memory counter, so their order inside a tile's slice is
     // arbitrary (all later uses count or sort them).  A tile's candidate and sure counts are final once
     // every warp has passed the next barrier; they are written out then ("pending" tile).
-    uint32_t cur_pos = 0, cur_end = 0, run_cand = 0, ccap = 0;
+    uint32_t cur_pos = 0, cur_end = 0, run_cand = 0;
     for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) sh[b] = 0;
     if (threadIdx.x < 12) s_cnt[threadIdx.x >> 2][threadIdx.x & 3] = 0;
-    if (threadIdx.x < 6) s_tot[threadIdx.x] = 0;
+    if (threadIdx.x < 4) s_tot[threadIdx.x] = 0;
     __syncthreads();
-    long long cur_prob = -1;
-    size_t cur_fidx = 0;
-    uint32_t lo = 0, hi = 0, shift = 0, tie_key = TIE_NONE, parity = 0;
+    uint32_t cur_prob = 0xFFFFFFFFu;
+    uint32_t lo = 0, parity = 0;
     uint32_t slot3 = 0;                                                // counter triple of the current tile
     uint32_t pend_item = 0xFFFFFFFFu, pend_slot = 0, pend_room = 0;    // tile whose counts are not written yet
-    bool pend_accumulates = false, pool_dry = false;
+    bool pool_dry = false;
     const float gamma = L.gamma;
     const uint32_t group_step = (gridDim.x - 1u) * MAIN_GROUP + 1u;    // from a group's last tile to the next group's first
     MainTile T{};
@@ -443,60 +467,62 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
         if (ig != 0u && T.have && T.lt + 1u < seg_tile_end) {
             T.lt += 1u;
             T.first += TILE;
-            T.full = T.first >= 0 && T.first + TILE <= (long long)T.seg.n;
+            T.full = T.first >= 0 && T.first + TILE <= (long long)T.n;
         } else {
             T = main_decode(P, item);
             seg_tile_end = T.have ? L.segs[T.s + 1].tile_begin : 0u;
         }
         // ---- flush the per-segment accumulators when the segment changes ---------------------------
-        const long long prob = T.have ? (long long)T.w * L.nseg + T.s : -2;
-        if (prob != cur_prob && cur_prob >= 0) {                       // uniform over the CTA
+        const uint32_t prob = T.have ? T.w * L.nseg + T.s : 0xFFFFFFFEu;
+        if (prob != cur_prob && cur_prob != 0xFFFFFFFFu) {             // uniform over the CTA
             __syncthreads();                                           // the last tile's counts are final
             if (threadIdx.x == 0 && pend_item != 0xFFFFFFFFu) {
                 const uint32_t c = min(s_cnt[pend_slot][0], pend_room), su = s_cnt[pend_slot][1], ti = s_cnt[pend_slot][2];
                 P.tile_ccnt[pend_item] = c; P.tile_sure[pend_item] = su;
-                if (tie_key != TIE_NONE) P.tile_tie[pend_item] = ti;
+                if (s_seg.tie_key != TIE_NONE) P.tile_tie[pend_item] = ti;
                 s_tot[0] += c; s_tot[1] += su; s_tot[2] += ti;
             }
             pend_item = 0xFFFFFFFFu;
-            for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
-                const uint32_t c = sh[b];
-                if (c) { atomicAdd(P.cand_hist + cur_fidx * CAND_BINS + b, c); sh[b] = 0; }
+            {
+                uint32_t* gh = s_seg.hist;
+                for (uint32_t b = threadIdx.x; b < CAND_BINS; b += THREADS) {
+                    const uint32_t c = sh[b];
+                    if (c) { atomicAdd(gh + b, c); sh[b] = 0; }
+                }
             }
-            __threadfence();                                           // this thread's additions are in L2 before the count below
             __syncthreads();
             if (threadIdx.x == 0) {
                 FastState* st = P.state + cur_prob;
                 if (s_tot[1]) atomicAdd(&st->sure_total, s_tot[1]);
                 if (s_tot[0]) atomicAdd(&st->cand_total, s_tot[0]);
                 if (s_tot[2]) atomicAdd(&st->tie_total, s_tot[2]);
-                __threadfence();
-                const uint32_t before = atomicAdd(&st->tiles_main, s_tot[3]);
-                s_misc[0] = (before + s_tot[3] == s_tot[4]) ? 1u : 0u;  // this CTA finished the segment's last tile
-                s_tot[0] = 0; s_tot[1] = 0; s_tot[2] = 0; s_tot[3] = 0;
+                s_tot[0] = 0; s_tot[1] = 0; s_tot[2] = 0;
             }
             if (threadIdx.x < 12) s_cnt[threadIdx.x >> 2][threadIdx.x & 3] = 0;
             __syncthreads();
-            if (s_misc[0]) {                                           // uniform: every other CTA's counts are in
-                __threadfence();
-                resolve_bin(P, (uint32_t)cur_prob);
-                __syncthreads();
-            }
             run_cand = 0;
-            cur_prob = -1;
+            cur_prob = 0xFFFFFFFFu;
         }
         if (!T.have) break;
         if (!T.fast) continue;                                         // uniform over the CTA
-        const SegEntry& seg = T.seg;
         if (prob != cur_prob) {
             cur_prob = prob;
-            cur_fidx = (size_t)T.w * L.fast_per_worker + seg.fast_index;
-            const FastState st = P.state[prob];
-            lo = st.lo; hi = st.hi; shift = st.shift; tie_key = st.tie_key;
-            ccap = seg.cand_cap;                                       // region size
-            cur_pos = blockIdx.x * seg.flag_cap; cur_end = cur_pos + seg.flag_cap;
+            lo = P.state[prob].lo;
+            const SegEntry* seg = L.segs + T.s;
+            cur_pos = blockIdx.x * seg->flag_cap; cur_end = cur_pos + seg->flag_cap;
             pool_dry = false;
-            if (threadIdx.x == 0) s_tot[4] = seg_tile_end - seg.tile_begin;
+            if (threadIdx.x == 0) {                                    // (no warp still reads the previous segment's block)
+                const FastState* st = P.state + prob;
+                MainSeg m;
+                m.hi = st->hi; m.shift = st->shift; m.tie_key = st->tie_key; m.ccap = seg->cand_cap;
+                m.flag_cap = seg->flag_cap; m.region_per_tile = seg->region_per_tile; m.ext_begin = seg->ext_begin; m.ext_cap = seg->ext_cap;
+                m.ext_chunk = seg->ext_chunk; m.cov_cap = seg->cov_cap; m.pad0 = 0; m.pad1 = 0;
+                m.flist = P.flagged + (size_t)T.w * L.flag_per_worker + seg->flag_begin;
+                m.clist = P.cand + (size_t)T.w * L.cand_per_worker + seg->cand_begin;
+                m.cover = P.cand + (size_t)T.w * L.cand_per_worker + seg->cov_begin;
+                m.hist = P.cand_hist + ((size_t)T.w * L.fast_per_worker + seg->fast_index) * CAND_BINS;
+                s_seg = m;
+            }
         }
         parity ^= 1u;
         slot3 = slot3 == 2u ? 0u : slot3 + 1u;
@@ -527,8 +553,8 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
             for (int j = 0; j < QUADS; ++j) {
                 const long long base = mine + 128 * j;
                 float p[4], gq[4];
-                const uint32_t valid = load_quad(e, base, seg.n, p);
-                load_quad_stream(T.g, base, seg.n, gq);
+                const uint32_t valid = load_quad(e, base, T.n, p);
+                load_quad_stream(T.g, base, T.n, gq);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     p[c] = accumulate(gamma, gq[c], p[c]);
@@ -581,6 +607,8 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
             fwbase += (i < (int)warp) ? f : 0u;
             tflag += f;
         }
+        const uint32_t tie_key = s_seg.tie_key, ccap = s_seg.ccap, flag_cap = s_seg.flag_cap;
+        const bool per_tile = s_seg.region_per_tile != 0u;
         // the previous tile's counts are final now (every warp has left its per-element loop)
         if (pend_item != 0xFFFFFFFFu) {
             const uint32_t c = min(s_cnt[pend_slot][0], pend_room);
@@ -590,26 +618,25 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
                 if (tie_key != TIE_NONE) P.tile_tie[pend_item] = ti;
                 s_tot[0] += c; s_tot[1] += su; s_tot[2] += ti;
             }
-            if (pend_accumulates) run_cand += c;
+            run_cand += c;
         }
         // this CTA's regions of the two lists, and where this tile's entries go inside them
-        const uint32_t tseg = T.lt - seg.tile_begin;                   // tile inside the segment
-        if (seg.region_per_tile) { cur_pos = tseg * seg.flag_cap; cur_end = cur_pos + seg.flag_cap; run_cand = 0; }
+        const uint32_t tseg = T.lt - T.tile_begin;                     // tile inside the segment
+        if (per_tile) { cur_pos = tseg * flag_cap; cur_end = cur_pos + flag_cap; run_cand = 0; }
         bool fits = cur_pos + tflag <= cur_end;
         if (!fits && !pool_dry) {                                      // uniform: the region is full, continue in the pool
             if (threadIdx.x == 0) {
-                const uint32_t want = max(tflag, seg.ext_chunk);
+                const uint32_t want = max(tflag, s_seg.ext_chunk);
                 const uint32_t got = atomicAdd(&P.state[prob].ext_used, want);
-                s_misc[1] = ((uint64_t)got + want <= seg.ext_cap) ? got : 0xFFFFFFFFu;
+                s_misc[1] = ((uint64_t)got + want <= s_seg.ext_cap) ? got : 0xFFFFFFFFu;
                 s_misc[2] = want;
             }
             __syncthreads();
             const uint32_t got = s_misc[1];
-            if (got != 0xFFFFFFFFu) { cur_pos = seg.ext_begin + got; cur_end = cur_pos + s_misc[2]; fits = true; }
+            if (got != 0xFFFFFFFFu) { cur_pos = s_seg.ext_begin + got; cur_end = cur_pos + s_misc[2]; fits = true; }
             else pool_dry = true;
         }
-        const uint32_t region = seg.region_per_tile ? tseg : blockIdx.x;
-        const uint32_t fbase = cur_pos, cbase = region * ccap + run_cand;
+        const uint32_t fbase = cur_pos, cbase = (per_tile ? tseg : blockIdx.x) * ccap + run_cand;
         const uint32_t room = ccap - run_cand;                         // candidate slots left for this tile
         if (threadIdx.x == 0) {
             P.tile_fbase[item] = fits ? fbase : 0xFFFFFFFFu;
@@ -618,9 +645,8 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
             if (!fits) P.state[prob].overflow = 1u;                    // the list is full: the segment falls back
             const uint32_t nxt = slot3 == 2u ? 0u : slot3 + 1u;        // counters of the tile after this one
             s_cnt[nxt][0] = 0; s_cnt[nxt][1] = 0; s_cnt[nxt][2] = 0;
-            s_tot[3] += 1u;
         }
-        pend_item = item; pend_slot = slot3; pend_room = fits ? room : 0u; pend_accumulates = !seg.region_per_tile;
+        pend_item = item; pend_slot = slot3; pend_room = fits ? room : 0u;
         if (fits) cur_pos += tflag;
         if (tie_key != TIE_NONE) {                                     // uniform: count this thread's tie-key elements
             uint32_t ties = 0;
@@ -628,8 +654,8 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
             for (int j = 0; j < QUADS; ++j) {
                 const float4 p = *reinterpret_cast<const float4*>(sp + off0 + 128 * j);
                 const uint32_t c0 = (uint32_t)(mine + 128 * j);        // coordinates outside the segment wrap far beyond n
-                ties += (uint32_t)(key_of(p.x) == tie_key && c0 < seg.n) + (uint32_t)(key_of(p.y) == tie_key && c0 + 1u < seg.n) +
-                        (uint32_t)(key_of(p.z) == tie_key && c0 + 2u < seg.n) + (uint32_t)(key_of(p.w) == tie_key && c0 + 3u < seg.n);
+                ties += (uint32_t)(key_of(p.x) == tie_key && c0 < T.n) + (uint32_t)(key_of(p.y) == tie_key && c0 + 1u < T.n) +
+                        (uint32_t)(key_of(p.z) == tie_key && c0 + 2u < T.n) + (uint32_t)(key_of(p.w) == tie_key && c0 + 3u < T.n);
             }
             ties = __reduce_add_sync(0xFFFFFFFFu, ties);
             if (lane == 0 && ties) atomicAdd(&s_cnt[slot3][2], ties);
@@ -639,9 +665,9 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
             // the sure ones in the residual (their values stay in the list, from where a fall-back restores
             // them; with a tie key the residual keeps p everywhere, so that the emit step can still tell a kept
             // element from a tie), append the candidates to the tile's slice and histogram them
-            uint2* flist = P.flagged + (size_t)T.w * L.flag_per_worker + seg.flag_begin + fbase + fwbase;
-            uint2* clist = P.cand + (size_t)T.w * L.cand_per_worker + seg.cand_begin + cbase;
-            uint2* cover = P.cand + (size_t)T.w * L.cand_per_worker + seg.cov_begin;   // where candidates go when the slice is full
+            uint2* flist = s_seg.flist + fbase + fwbase;
+            uint2* clist = s_seg.clist + cbase;
+            const uint32_t hi = s_seg.hi, shift = s_seg.shift;
             const uint32_t first32 = (uint32_t)T.first + warp * 512u;
             const float* spw = sp + warp * 512u;
             const bool zero_now = tie_key == TIE_NONE;
@@ -665,12 +691,12 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
                     if (lane == 0) base = atomicAdd(&s_cnt[slot3][0], (uint32_t)__popc(bc));
                     base = __shfl_sync(0xFFFFFFFFu, base, 0);
                     if (cand) {
-                        const uint32_t pos = base + __popc(bc & lt_mask);
+                        const uint32_t pos = base + __popc(bc & ((1u << lane) - 1u));
                         if (pos < room) {
                             clist[pos] = make_uint2(key, coord);
                         } else {                                       // rare: candidates crowd in this part of the segment
                             const uint32_t gp = atomicAdd(&P.state[prob].cov_used, 1u);
-                            if (gp < seg.cov_cap) cover[gp] = make_uint2(key, coord);
+                            if (gp < s_seg.cov_cap) s_seg.cover[gp] = make_uint2(key, coord);
                             else P.state[prob].overflow = 1u;
                         }
                         atomicAdd(&sh[min((key - lo) >> shift, CAND_BINS - 1u)], 1u);
@@ -682,45 +708,112 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
     }
 }
 
-// ---- per-tile walks over the candidate slices ----------------------------------------------------
-// Eight lanes share TILES_PER_GROUP consecutive tiles.  The filter below is bound by a chain of
-// dependent loads (slice length and base, then the slice), so a group first requests the placement
-// words of all its tiles, then the first eight candidates of every tile, and only then looks at
-// them: four tiles per group cut the number of such chains per launch by four.
+// ---- filter: copy the candidates of the threshold's bin into the short list -------------------
+// Eight lanes share TILES_PER_GROUP consecutive tiles.  The walk is bound by a chain of dependent
+// loads (slice length and base, then the slice), so a group first requests the placement words of
+// all its tiles, then the first eight candidates of every tile, and only then looks at them: four
+// tiles per group cut the number of such chains per launch by four.
+// A CTA serves a contiguous range of tiles, FILTER_TILES_PER_CTA at a time; before each such batch it
+// works out the threshold's bin of every large segment the batch touches (see resolve_bin).
 constexpr uint32_t TILES_PER_GROUP = 4;
 constexpr uint32_t FILTER_TILES_PER_CTA = (THREADS / 8) * TILES_PER_GROUP;
-struct CandSlice {                 // one tile's slice as seen by a lane of its group
-    const uint2* list;             // nullptr: nothing to do for this tile
-    uint32_t cnt, prob, w, lt;
-    bool counts;                   // the tile belongs to a segment on the one-pass path
-    uint2 first;                   // entry `sub` of the slice (if sub < cnt)
-};
-__device__ inline void cand_slices(const FastParams& P, uint32_t item0, uint32_t sub, CandSlice (&t)[TILES_PER_GROUP]) {
+
+__global__ void __launch_bounds__(THREADS)
+topk_filter_kernel(const __grid_constant__ FastParams P, uint32_t items_per_cta) {
+    __shared__ BinInfo s_bin[FILTER_TILES_PER_CTA];                    // by problem index relative to the batch's first
+    __shared__ uint32_t s_range[2];
     const Layout& L = P.L;
-    uint32_t base[TILES_PER_GROUP];
+    const uint32_t sub = threadIdx.x & 7u;
+    const uint32_t chunk_begin = blockIdx.x * items_per_cta;
+    const uint32_t chunk_end = min(chunk_begin + items_per_cta, P.total_items);
+    uint32_t cached_prob = 0xFFFFFFFFu;
+    BinInfo cached = {0u, 0u, 0u, 0u};
+    for (uint32_t batch = chunk_begin; batch < chunk_end; batch += FILTER_TILES_PER_CTA) {
+        const uint32_t batch_end = min(batch + FILTER_TILES_PER_CTA, chunk_end);
+        __syncthreads();                                               // the previous batch is done with the table
+        if (threadIdx.x < 2) {
+            const uint32_t item = threadIdx.x == 0 ? batch : batch_end - 1u;
+            const uint32_t w = item / L.tiles_per_worker;
+            const uint32_t lt = item - w * L.tiles_per_worker;
+            s_range[threadIdx.x] = w * L.nseg + ((L.nseg == 1) ? 0u : find_by_tile(L, lt));
+        }
+        __syncthreads();
+        const uint32_t p_first = s_range[0], p_last = s_range[1];     // at most one problem per tile of the batch
+        for (uint32_t p = p_first; p <= p_last; ++p) {                // uniform over the CTA
+            const uint32_t s = p % L.nseg;
+            if (!L.segs[s].fast) continue;
+            if (p != cached_prob) {
+                // the CTA whose range holds the segment's first tile records the result
+                const uint32_t w = p / L.nseg;
+                const uint32_t first_item = w * L.tiles_per_worker + L.segs[s].tile_begin;
+                cached = resolve_bin(P, p, first_item >= batch && first_item < batch_end);
+                cached_prob = p;
+            }
+            if (threadIdx.x == 0) s_bin[p - p_first] = cached;
+        }
+        __syncthreads();
+        const uint32_t item0 = batch + (threadIdx.x >> 3) * TILES_PER_GROUP;
+        uint32_t cnt[TILES_PER_GROUP], base[TILES_PER_GROUP];
 #pragma unroll
-    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-        const uint32_t item = item0 + u;
-        t[u].list = nullptr; t[u].cnt = 0; base[u] = 0; t[u].counts = false; t[u].prob = 0xFFFFFFFFu;
-        if (item < P.total_items) { t[u].cnt = __ldg(P.tile_ccnt + item); base[u] = __ldg(P.tile_cbase + item); }
-    }
+        for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+            const uint32_t item = item0 + u;
+            cnt[u] = 0; base[u] = 0;
+            if (item < batch_end) { cnt[u] = __ldg(P.tile_ccnt + item); base[u] = __ldg(P.tile_cbase + item); }
+        }
+        const uint2* list[TILES_PER_GROUP];
+        uint2 first[TILES_PER_GROUP];
+        uint32_t prob[TILES_PER_GROUP];
 #pragma unroll
-    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-        const uint32_t item = item0 + u;
-        t[u].first = make_uint2(0u, 0u);
-        if (item >= P.total_items) continue;
-        t[u].w = item / L.tiles_per_worker;
-        t[u].lt = item - t[u].w * L.tiles_per_worker;
-        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, t[u].lt);
-        const SegEntry& seg = L.segs[s];
-        if (!seg.fast) { t[u].cnt = 0; continue; }
-        t[u].prob = t[u].w * L.nseg + s;
-        const FastState* st = P.state + t[u].prob;
-        if (st->path != PATH_FAST) { t[u].cnt = 0; t[u].prob = 0xFFFFFFFFu; continue; }
-        t[u].counts = true;
-        if (st->need2 == 0) { t[u].cnt = 0; continue; }               // no candidate, or every candidate, is kept
-        t[u].list = P.cand + (size_t)t[u].w * L.cand_per_worker + seg.cand_begin + base[u];
-        if (sub < t[u].cnt) t[u].first = __ldg(t[u].list + sub);
+        for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+            const uint32_t item = item0 + u;
+            list[u] = nullptr; first[u] = make_uint2(0u, 0u); prob[u] = 0u;
+            if (item >= batch_end) continue;
+            const uint32_t w = item / L.tiles_per_worker;
+            const uint32_t lt = item - w * L.tiles_per_worker;
+            const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+            const SegEntry& seg = L.segs[s];
+            prob[u] = w * L.nseg + s;
+            if (!seg.fast) continue;
+            const BinInfo bi = s_bin[prob[u] - p_first];
+            if (!bi.live || bi.need2 == 0u || cnt[u] == 0u) continue;  // no candidate, or every candidate, is kept
+            list[u] = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + base[u];
+            if (sub < cnt[u]) first[u] = __ldg(list[u] + sub);
+        }
+#pragma unroll
+        for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+            // candidates above the threshold's bin are kept whatever the exact threshold turns out to be; those
+            // inside the bin go to the short list, and the finish step adds the kept ones to the tile's count
+            uint32_t above = 0, inbin = 0;
+            if (list[u]) {
+                const BinInfo bi = s_bin[prob[u] - p_first];
+                const uint32_t s = prob[u] % L.nseg, w = prob[u] / L.nseg;
+                uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
+                for (uint32_t i0 = sub; i0 < cnt[u]; i0 += 32) {           // four entries in flight per lane
+                    uint2 c4[4];
+#pragma unroll
+                    for (uint32_t v = 0; v < 4; ++v) {
+                        const uint32_t i = i0 + 8u * v;
+                        c4[v] = i == sub ? first[u] : (i < cnt[u] ? __ldg(list[u] + i) : make_uint2(0u, 0u));
+                    }
+#pragma unroll
+                    for (uint32_t v = 0; v < 4; ++v) {
+                        if (i0 + 8u * v >= cnt[u]) continue;
+                        const uint2 c = c4[v];
+                        if (c.x > bi.hi2) ++above;
+                        else if (c.x >= bi.lo2) {
+                            ++inbin;
+                            const uint32_t pos = atomicAdd(&P.state[prob[u]].cnt2, 1u);
+                            if (pos < LIST2_CAP) out[pos] = c;
+                        }
+                    }
+                }
+            }
+            uint32_t both = above | (inbin << 16);                     // a tile holds at most 4096 candidates
+            both += __shfl_xor_sync(0xFFFFFFFFu, both, 1);
+            both += __shfl_xor_sync(0xFFFFFFFFu, both, 2);
+            both += __shfl_xor_sync(0xFFFFFFFFu, both, 4);
+            if (sub == 0u && item0 + u < batch_end) P.tile_csum[item0 + u] = both;
+        }
     }
 }
 
@@ -728,207 +821,198 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
     return key > T || (key == T && coord < icut);
 }
 
-// Last step of a segment (run by the CTA that filtered its last tile): exact threshold from the short
-// list, per-tile kept counts, message offsets.
-//   threshold among the candidates: the short list (the candidates of the threshold's histogram bin,
-//       at most LIST2_CAP) is sorted in shared memory, larger key first and lower coordinate first among
-//       equal keys; its first need2 entries are kept, which fixes T and the coordinate cut, and each of
-//       them adds one to its tile's count of kept candidates;
+// ---- finish: exact threshold, per-tile kept counts, message offsets ----------------------------
+// One thread-block cluster per large (worker, segment).
+//   threshold among the candidates: CTA 0 sorts the short list (the candidates of the threshold's
+//       histogram bin, at most LIST2_CAP) in shared memory, larger key first and lower coordinate first
+//       among equal keys; its first need2 entries are kept, which fixes T and the coordinate cut, and each
+//       of them adds one to its tile's count of kept candidates;
 //   threshold == tie key: every listed element is kept and the first need_ties tie-key elements in
 //       coordinate order: a running sum of the per-tile tie counts says how many each tile admits;
-//   then the kept counts of the segment's tiles are summed up into the tiles' first message slots.
-__device__ __noinline__ void finish_segment(const FastParams& P, uint32_t prob) {
+//   then the kept counts of the segment's tiles are summed up into the tiles' first message slots: every
+//   CTA of the cluster adds up a contiguous share of the tiles, the shares' totals are exchanged through
+//   distributed shared memory, and each CTA scans its share from the sum of the shares before it.
+// The cluster barriers are the hardware's; every CTA runs to the last one.
+constexpr uint32_t FINISH_CTAS = 8;
+constexpr uint32_t FINISH_PER = 8;                                     // tiles per thread and round of a scan
+__device__ inline uint32_t block_sum(uint32_t v, uint32_t* s_scan) {
+    uint32_t total;
+    block_exclusive_scan(v, s_scan, &total);
+    return total;
+}
+__global__ void __launch_bounds__(THREADS)
+topk_finish_kernel(const __grid_constant__ FastParams P) {
+    namespace cg = cooperative_groups;
     __shared__ unsigned long long srt[LIST2_CAP];
     __shared__ uint32_t s_scan[WARPS + 1];
+    __shared__ uint32_t s_share[3];                                    // ties and kept elements of this CTA's share; [2]: CTA 0 gave up
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t rank = cluster.block_rank();
     const Layout& L = P.L;
-    const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
+    uint32_t w, s;
+    const uint32_t prob = fast_problem(L, blockIdx.x / FINISH_CTAS, w, s);
     const SegEntry seg = L.segs[s];
-    FastState st = load_state_l2(P.state + prob);
-    if (st.path != PATH_FAST) return;
+    FastState st = P.state[prob];
+    if (st.path != PATH_FAST) return;                                  // the same answer in every CTA of the cluster
     const uint32_t ntiles = L.segs[s + 1].tile_begin - seg.tile_begin;
     const size_t item0 = (size_t)w * L.tiles_per_worker + seg.tile_begin;
     const bool admit = st.need_ties != 0u;
-    const uint32_t mis = misalign_of(P.residuals + (size_t)w * L.n_total + seg.offset);   // tiles lie on the 128-byte grid of the row
-    // candidates that did not fit their tile's slice (rare): those of the threshold's bin join the short list
-    const uint32_t ncov = min(st.cov_used, seg.cov_cap);
-    const uint2* cover = P.cand + (size_t)w * L.cand_per_worker + seg.cov_begin;
-    if (st.need2 && ncov) {
-        uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
-        for (uint32_t i = threadIdx.x; i < ncov; i += THREADS) {
-            const uint2 c = __ldcg(cover + i);
-            if (c.x >= st.lo2 && c.x <= st.hi2) {
-                const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
-                if (pos < LIST2_CAP) out[pos] = c;
-            }
-        }
-        __threadfence();
-        __syncthreads();
-        st.cnt2 = __ldcg(&P.state[prob].cnt2);
-    }
-    if (st.need2) {
-        const uint32_t cnt = st.cnt2;
-        if (cnt != st.expect2 || cnt > LIST2_CAP || st.need2 > cnt) {  // short list disagrees with the histogram
-            if (threadIdx.x == 0) {
-                st.path = PATH_FAILED; st.fail = FAIL_SHORT_LIST;
-                P.state[prob] = st;
-                atomicAdd(P.counters, 1u);
-            }
-            return;
-        }
-        uint32_t size = 1;
-        while (size < cnt) size <<= 1;
-        const uint2* in = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
-        for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
-            unsigned long long v = 0;                                   // padding sorts last
-            if (i < cnt) { const uint2 c = __ldcg(in + i); v = ((unsigned long long)c.x << 32) | (0xFFFFFFFFu - c.y); }
-            srt[i] = v;
-        }
-        __syncthreads();
-        // bitonic sort, descending: larger key first, equal keys: lower coordinate first
-        for (uint32_t k2 = 2; k2 <= size; k2 <<= 1) {
-            for (uint32_t j = k2 >> 1; j > 0; j >>= 1) {
-                for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
-                    const uint32_t ixj = i ^ j;
-                    if (ixj > i) {
-                        const unsigned long long a = srt[i], b = srt[ixj];
-                        const bool desc = (i & k2) == 0;
-                        if (desc ? (a < b) : (a > b)) { srt[i] = b; srt[ixj] = a; }
-                    }
-                }
-                __syncthreads();
-            }
-        }
-        const unsigned long long v = srt[st.need2 - 1u];
-        st.T = (uint32_t)(v >> 32);
-        st.icut = (0xFFFFFFFFu - (uint32_t)v) + 1u;                    // coordinates below this are kept among the ties
-        if (st.icut == 0) st.icut = 0xFFFFFFFFu;                       // (coordinate 2^32-1 cannot occur: n < 2^32)
-        // the kept entries of the short list, counted into their tiles
-        for (uint32_t i = threadIdx.x; i < st.need2; i += THREADS) {
-            const uint32_t coord = 0xFFFFFFFFu - (uint32_t)srt[i];
-            atomicAdd(P.tile_csum + item0 + (coord + mis) / TILE, 1u);
-        }
-        __threadfence();
-        __syncthreads();
-    }
-    if (ncov && (admit || st.need2)) {                                 // kept overflow candidates, counted into their tiles
-        uint32_t* counts = admit ? P.tile_ccnt : P.tile_csum;          // (every candidate is kept when ties are admitted)
-        for (uint32_t i = threadIdx.x; i < ncov; i += THREADS) {
-            const uint2 c = __ldcg(cover + i);
-            if (admit || c.x > st.hi2) atomicAdd(counts + item0 + (c.y + mis) / TILE, 1u);
-        }
-        __threadfence();
-        __syncthreads();
-    }
-    // ---- kept count per tile, exclusive sum over the segment's tiles ------------------------------
-    constexpr uint32_t PER = 8;                                         // tiles per thread and round
-    uint32_t* off = P.offsets + (size_t)w * (L.tiles_per_worker + 1) + seg.tile_begin;
-    uint32_t kept_run = 0, tie_run = 0;
-    for (uint32_t base = 0; base < ntiles; base += THREADS * PER) {
-        const uint32_t t0 = base + threadIdx.x * PER;
-        uint32_t kept[PER], adm[PER], tsum = 0;
-#pragma unroll
-        for (uint32_t i = 0; i < PER; ++i) {
-            kept[i] = 0; adm[i] = 0;
-            if (t0 + i < ntiles) {
-                kept[i] = __ldcg(P.tile_sure + item0 + t0 + i);
-                if (admit) { kept[i] += __ldcg(P.tile_ccnt + item0 + t0 + i); adm[i] = __ldcg(P.tile_tie + item0 + t0 + i); }
-                else kept[i] += __ldcg(P.tile_csum + item0 + t0 + i) & 0xFFFFu;
-                tsum += adm[i];
-            }
-        }
-        if (admit) {                                                   // ties before each tile decide how many it admits
-            uint32_t total;
-            uint32_t before = tie_run + block_exclusive_scan(tsum, s_scan, &total);
-            tie_run += total;
-#pragma unroll
-            for (uint32_t i = 0; i < PER; ++i) {
-                const uint32_t room = st.need_ties > before ? st.need_ties - before : 0u;
-                const uint32_t a = min(adm[i], room);
-                before += adm[i];
-                kept[i] += a;
-                if (t0 + i < ntiles) P.tile_csum[item0 + t0 + i] = a;
-            }
-        }
-        uint32_t ksum = 0;
-#pragma unroll
-        for (uint32_t i = 0; i < PER; ++i) ksum += kept[i];
-        uint32_t total;
-        uint32_t ex = kept_run + block_exclusive_scan(ksum, s_scan, &total);
-        kept_run += total;
-#pragma unroll
-        for (uint32_t i = 0; i < PER; ++i) {
-            if (t0 + i < ntiles) off[t0 + i] = ex;
-            ex += kept[i];
-        }
-    }
-    if (threadIdx.x == 0) {
-        if (kept_run != seg.k) atomicMin(P.status, ST_DEVICE_CHECK);   // counts and k disagree
-        P.state[prob] = st;
-    }
-}
-
-// ---- resolve: copy the candidates of the threshold's bin into the short list; finish segments -----
-__global__ void __launch_bounds__(THREADS)
-topk_resolve_kernel(const __grid_constant__ FastParams P) {
-    __shared__ uint32_t s_prob[FILTER_TILES_PER_CTA];
-    __shared__ uint32_t s_fin[FILTER_TILES_PER_CTA];
-    __shared__ uint32_t s_nfin;
-    const Layout& L = P.L;
-    const uint32_t sub = threadIdx.x & 7u;
-    const uint32_t item0 = ((blockIdx.x * THREADS + threadIdx.x) >> 3) * TILES_PER_GROUP;
-    if (threadIdx.x == 0) s_nfin = 0;
-    CandSlice t[TILES_PER_GROUP];
-    cand_slices(P, item0, sub, t);
-#pragma unroll
-    for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-        // candidates above the threshold's bin are kept whatever the exact threshold turns out to be; those
-        // inside the bin go to the short list, and the segment's last step adds the kept ones to the count
-        uint32_t above = 0, inbin = 0;
-        if (t[u].list && t[u].cnt) {
-            const FastState* stp = P.state + t[u].prob;
-            const uint32_t lo2 = stp->lo2, hi2 = stp->hi2;
-            const uint32_t s = t[u].prob - t[u].w * L.nseg;
-            uint2* out = P.list2 + ((size_t)t[u].w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
-            for (uint32_t i = sub; i < t[u].cnt; i += 8) {
-                const uint2 c = i == sub ? t[u].first : t[u].list[i];
-                if (c.x > hi2) ++above;
-                else if (c.x >= lo2) {
-                    ++inbin;
-                    const uint32_t pos = atomicAdd(&P.state[t[u].prob].cnt2, 1u);
+    if (rank == 0) {
+        bool failed = false;
+        const uint32_t mis = misalign_of(P.residuals + (size_t)w * L.n_total + seg.offset);   // tiles lie on the 128-byte grid of the row
+        // candidates that did not fit their tile's slice (rare): those of the threshold's bin join the short list
+        const uint32_t ncov = min(st.cov_used, seg.cov_cap);
+        const uint2* cover = P.cand + (size_t)w * L.cand_per_worker + seg.cov_begin;
+        if (st.need2 && ncov) {
+            uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
+            for (uint32_t i = threadIdx.x; i < ncov; i += THREADS) {
+                const uint2 c = cover[i];
+                if (c.x >= st.lo2 && c.x <= st.hi2) {
+                    const uint32_t pos = atomicAdd(&P.state[prob].cnt2, 1u);
                     if (pos < LIST2_CAP) out[pos] = c;
                 }
             }
+            __threadfence();
+            __syncthreads();
+            st.cnt2 = __ldcg(&P.state[prob].cnt2);
         }
-        uint32_t both = above | (inbin << 16);                         // a tile holds at most 4096 candidates
-        both += __shfl_xor_sync(0xFFFFFFFFu, both, 1);
-        both += __shfl_xor_sync(0xFFFFFFFFu, both, 2);
-        both += __shfl_xor_sync(0xFFFFFFFFu, both, 4);
-        if (sub == 0u) {
-            if (item0 + u < P.total_items) P.tile_csum[item0 + u] = both;
-            s_prob[(threadIdx.x >> 3) * TILES_PER_GROUP + u] = t[u].counts ? t[u].prob : 0xFFFFFFFFu;
+        if (st.need2) {
+            const uint32_t cnt = st.cnt2;
+            if (cnt != st.expect2 || cnt > LIST2_CAP || st.need2 > cnt) {  // short list disagrees with the histogram
+                failed = true;
+                if (threadIdx.x == 0) {
+                    P.state[prob].path = PATH_FAILED; P.state[prob].fail = FAIL_SHORT_LIST;
+                    atomicAdd(P.counters, 1u);
+                }
+            } else {
+                uint32_t size = 1;
+                while (size < cnt) size <<= 1;
+                const uint2* in = P.list2 + ((size_t)w * L.fast_per_worker + seg.fast_index) * LIST2_CAP;
+                for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
+                    unsigned long long v = 0;                           // padding sorts last
+                    if (i < cnt) { const uint2 c = __ldcg(in + i); v = ((unsigned long long)c.x << 32) | (0xFFFFFFFFu - c.y); }
+                    srt[i] = v;
+                }
+                __syncthreads();
+                // bitonic sort, descending: larger key first, equal keys: lower coordinate first
+                for (uint32_t k2 = 2; k2 <= size; k2 <<= 1) {
+                    for (uint32_t j = k2 >> 1; j > 0; j >>= 1) {
+                        for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
+                            const uint32_t ixj = i ^ j;
+                            if (ixj > i) {
+                                const unsigned long long a = srt[i], b = srt[ixj];
+                                const bool desc = (i & k2) == 0;
+                                if (desc ? (a < b) : (a > b)) { srt[i] = b; srt[ixj] = a; }
+                            }
+                        }
+                        __syncthreads();
+                    }
+                }
+                const unsigned long long v = srt[st.need2 - 1u];
+                st.T = (uint32_t)(v >> 32);
+                st.icut = (0xFFFFFFFFu - (uint32_t)v) + 1u;            // coordinates below this are kept among the ties
+                if (st.icut == 0) st.icut = 0xFFFFFFFFu;               // (coordinate 2^32-1 cannot occur: n < 2^32)
+                if (threadIdx.x == 0) { P.state[prob].T = st.T; P.state[prob].icut = st.icut; }
+                // the kept entries of the short list, counted into their tiles
+                for (uint32_t i = threadIdx.x; i < st.need2; i += THREADS) {
+                    const uint32_t coord = 0xFFFFFFFFu - (uint32_t)srt[i];
+                    atomicAdd(P.tile_csum + item0 + (coord + mis) / TILE, 1u);
+                }
+            }
         }
-    }
-    // ---- which segments did this CTA complete?  One addition per run of tiles of the same segment.
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x < FILTER_TILES_PER_CTA) {
-        const uint32_t p = s_prob[threadIdx.x];
-        if (p != 0xFFFFFFFFu && (threadIdx.x == 0 || s_prob[threadIdx.x - 1] != p)) {
-            uint32_t run = 1;
-            while (threadIdx.x + run < FILTER_TILES_PER_CTA && s_prob[threadIdx.x + run] == p) ++run;
-            const uint32_t s = p % L.nseg;
-            const uint32_t ntiles = L.segs[s + 1].tile_begin - L.segs[s].tile_begin;
-            const uint32_t before = atomicAdd(&P.state[p].tiles_filter, run);
-            if (before + run == ntiles) s_fin[atomicAdd(&s_nfin, 1u)] = p;
+        if (!failed && ncov && (admit || st.need2)) {                  // kept overflow candidates, counted into their tiles
+            uint32_t* counts = admit ? P.tile_ccnt : P.tile_csum;      // (every candidate is kept when ties are admitted)
+            for (uint32_t i = threadIdx.x; i < ncov; i += THREADS) {
+                const uint2 c = cover[i];
+                if (admit || c.x > st.hi2) atomicAdd(counts + item0 + (c.y + mis) / TILE, 1u);
+            }
         }
+        if (threadIdx.x == 0) s_share[2] = failed ? 1u : 0u;
+        __threadfence();                                               // the counts above are in L2 before the peers read them
     }
-    __syncthreads();
-    const uint32_t nfin = s_nfin;
-    for (uint32_t i = 0; i < nfin; ++i) {                              // uniform over the CTA
-        __threadfence();
-        finish_segment(P, s_fin[i]);
-        __syncthreads();
+    cluster.sync();
+    const bool give_up = *cluster.map_shared_rank(&s_share[2], 0) != 0u;
+    if (!give_up) {
+        // ---- kept count per tile, exclusive sum over the segment's tiles ------------------------------
+        constexpr uint32_t ROUND = THREADS * FINISH_PER;
+        const uint32_t per = ((ntiles + FINISH_CTAS - 1) / FINISH_CTAS + ROUND - 1) / ROUND * ROUND;
+        const uint32_t begin = min(rank * per, ntiles), end = min(begin + per, ntiles);
+        uint32_t* off = P.offsets + (size_t)w * (L.tiles_per_worker + 1) + seg.tile_begin;
+        uint32_t tie_run = 0;                                          // tie-key elements of the segment before the current tile
+        if (admit) {
+            uint32_t tsum = 0;
+            for (uint32_t t = begin + threadIdx.x; t < end; t += THREADS) tsum += __ldcg(P.tile_tie + item0 + t);
+            tsum = block_sum(tsum, s_scan);
+            if (threadIdx.x == 0) s_share[0] = tsum;
+            cluster.sync();
+            for (uint32_t r = 0; r < rank; ++r) tie_run += *cluster.map_shared_rank(&s_share[0], r);
+        }
+        // first round over the share: how many ties each tile admits, and the share's kept total
+        uint32_t ksum = 0;
+        for (uint32_t base = begin; base < end; base += ROUND) {
+            const uint32_t t0 = base + threadIdx.x * FINISH_PER;
+            uint32_t kept[FINISH_PER];
+#pragma unroll
+            for (uint32_t i = 0; i < FINISH_PER; ++i) {
+                kept[i] = 0;
+                if (t0 + i < end) {
+                    kept[i] = __ldcg(P.tile_sure + item0 + t0 + i);
+                    kept[i] += admit ? __ldcg(P.tile_ccnt + item0 + t0 + i) : (__ldcg(P.tile_csum + item0 + t0 + i) & 0xFFFFu);
+                }
+            }
+            if (admit) {
+                uint32_t adm[FINISH_PER], tsum = 0;
+#pragma unroll
+                for (uint32_t i = 0; i < FINISH_PER; ++i) {
+                    adm[i] = t0 + i < end ? __ldcg(P.tile_tie + item0 + t0 + i) : 0u;
+                    tsum += adm[i];
+                }
+                uint32_t total;
+                uint32_t before = tie_run + block_exclusive_scan(tsum, s_scan, &total);
+                tie_run += total;
+#pragma unroll
+                for (uint32_t i = 0; i < FINISH_PER; ++i) {
+                    const uint32_t room = st.need_ties > before ? st.need_ties - before : 0u;
+                    const uint32_t a = min(adm[i], room);
+                    before += adm[i];
+                    kept[i] += a;
+                    if (t0 + i < end) P.tile_csum[item0 + t0 + i] = a;
+                }
+            }
+#pragma unroll
+            for (uint32_t i = 0; i < FINISH_PER; ++i) ksum += kept[i];
+        }
+        ksum = block_sum(ksum, s_scan);
+        if (threadIdx.x == 0) s_share[1] = ksum;
+        cluster.sync();
+        uint32_t kept_run = 0;
+        for (uint32_t r = 0; r < rank; ++r) kept_run += *cluster.map_shared_rank(&s_share[1], r);
+        // second round: the tiles' first message slots
+        for (uint32_t base = begin; base < end; base += ROUND) {
+            const uint32_t t0 = base + threadIdx.x * FINISH_PER;
+            uint32_t kept[FINISH_PER], sum = 0;
+#pragma unroll
+            for (uint32_t i = 0; i < FINISH_PER; ++i) {
+                kept[i] = 0;
+                if (t0 + i < end) {
+                    kept[i] = __ldcg(P.tile_sure + item0 + t0 + i);
+                    if (admit) kept[i] += __ldcg(P.tile_ccnt + item0 + t0 + i) + __ldcg(P.tile_csum + item0 + t0 + i);
+                    else kept[i] += __ldcg(P.tile_csum + item0 + t0 + i) & 0xFFFFu;
+                }
+                sum += kept[i];
+            }
+            uint32_t total;
+            uint32_t ex = kept_run + block_exclusive_scan(sum, s_scan, &total);
+            kept_run += total;
+#pragma unroll
+            for (uint32_t i = 0; i < FINISH_PER; ++i) {
+                if (t0 + i < end) off[t0 + i] = ex;
+                ex += kept[i];
+            }
+        }
+        if (rank == FINISH_CTAS - 1u && threadIdx.x == 0 && kept_run != seg.k) atomicMin(P.status, ST_DEVICE_CHECK);   // counts and k disagree
     }
+    cluster.sync();                                                    // a peer's totals must outlive their readers
 }
 
 // ---- emit: G lanes per tile walk the tile's slice of the flagged list ----------------------------
