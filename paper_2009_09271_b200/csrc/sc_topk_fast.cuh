@@ -713,107 +713,117 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
 // loads (slice length and base, then the slice), so a group first requests the placement words of
 // all its tiles, then the first eight candidates of every tile, and only then looks at them: four
 // tiles per group cut the number of such chains per launch by four.
-// A CTA serves a contiguous range of tiles, FILTER_TILES_PER_CTA at a time; before each such batch it
-// works out the threshold's bin of every large segment the batch touches (see resolve_bin).
+// A CTA serves a contiguous range of tiles.  It first works out the threshold's bin of every large
+// segment its range touches (see resolve_bin; FILTER_TABLE segments at a time), then its lane groups
+// walk the range without meeting again.
 constexpr uint32_t TILES_PER_GROUP = 4;
-constexpr uint32_t FILTER_TILES_PER_CTA = (THREADS / 8) * TILES_PER_GROUP;
+constexpr uint32_t FILTER_TILES_PER_CTA = (THREADS / 8) * TILES_PER_GROUP;   // tiles one sweep of the lane groups covers
+constexpr uint32_t FILTER_TABLE = 64;
+
+__device__ inline uint32_t problem_of_item(const Layout& L, uint32_t item) {
+    const uint32_t w = item / L.tiles_per_worker;
+    const uint32_t lt = item - w * L.tiles_per_worker;
+    return w * L.nseg + ((L.nseg == 1) ? 0u : find_by_tile(L, lt));
+}
 
 __global__ void __launch_bounds__(THREADS)
 topk_filter_kernel(const __grid_constant__ FastParams P, uint32_t items_per_cta) {
-    __shared__ BinInfo s_bin[FILTER_TILES_PER_CTA];                    // by problem index relative to the batch's first
+    __shared__ BinInfo s_bin[FILTER_TABLE];                            // by problem index relative to the first of the table
     __shared__ uint32_t s_range[2];
     const Layout& L = P.L;
     const uint32_t sub = threadIdx.x & 7u;
     const uint32_t chunk_begin = blockIdx.x * items_per_cta;
     const uint32_t chunk_end = min(chunk_begin + items_per_cta, P.total_items);
-    uint32_t cached_prob = 0xFFFFFFFFu;
-    BinInfo cached = {0u, 0u, 0u, 0u};
-    for (uint32_t batch = chunk_begin; batch < chunk_end; batch += FILTER_TILES_PER_CTA) {
-        const uint32_t batch_end = min(batch + FILTER_TILES_PER_CTA, chunk_end);
-        __syncthreads();                                               // the previous batch is done with the table
-        if (threadIdx.x < 2) {
-            const uint32_t item = threadIdx.x == 0 ? batch : batch_end - 1u;
-            const uint32_t w = item / L.tiles_per_worker;
-            const uint32_t lt = item - w * L.tiles_per_worker;
-            s_range[threadIdx.x] = w * L.nseg + ((L.nseg == 1) ? 0u : find_by_tile(L, lt));
-        }
-        __syncthreads();
-        const uint32_t p_first = s_range[0], p_last = s_range[1];     // at most one problem per tile of the batch
-        for (uint32_t p = p_first; p <= p_last; ++p) {                // uniform over the CTA
-            const uint32_t s = p % L.nseg;
-            if (!L.segs[s].fast) continue;
-            if (p != cached_prob) {
-                // the CTA whose range holds the segment's first tile records the result
-                const uint32_t w = p / L.nseg;
-                const uint32_t first_item = w * L.tiles_per_worker + L.segs[s].tile_begin;
-                cached = resolve_bin(P, p, first_item >= batch && first_item < batch_end);
-                cached_prob = p;
+    for (uint32_t pos = chunk_begin; pos < chunk_end; ) {
+        __syncthreads();                                               // the previous part is done with the table
+        if (threadIdx.x == 0) {
+            const uint32_t p_first = problem_of_item(L, pos);
+            const uint32_t p_stop = p_first + FILTER_TABLE;            // first problem the table has no room for
+            uint32_t part_end = chunk_end;
+            if (problem_of_item(L, chunk_end - 1u) >= p_stop) {        // the range goes on beyond the table: stop at that problem's first tile
+                const uint32_t w = p_stop / L.nseg, s = p_stop - w * L.nseg;
+                part_end = w * L.tiles_per_worker + L.segs[s].tile_begin;
             }
-            if (threadIdx.x == 0) s_bin[p - p_first] = cached;
+            s_range[0] = p_first; s_range[1] = part_end;
         }
         __syncthreads();
-        const uint32_t item0 = batch + (threadIdx.x >> 3) * TILES_PER_GROUP;
-        uint32_t cnt[TILES_PER_GROUP], base[TILES_PER_GROUP];
-#pragma unroll
-        for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-            const uint32_t item = item0 + u;
-            cnt[u] = 0; base[u] = 0;
-            if (item < batch_end) { cnt[u] = __ldg(P.tile_ccnt + item); base[u] = __ldg(P.tile_cbase + item); }
+        const uint32_t p_first = s_range[0], part_end = s_range[1];
+        const uint32_t p_last = problem_of_item(L, part_end - 1u);
+        for (uint32_t p = p_first; p <= p_last; ++p) {                // uniform over the CTA
+            const uint32_t w = p / L.nseg, s = p - w * L.nseg;
+            if (!L.segs[s].fast) continue;
+            // the CTA whose range holds the segment's first tile records the result
+            const uint32_t first_item = w * L.tiles_per_worker + L.segs[s].tile_begin;
+            const BinInfo bi = resolve_bin(P, p, first_item >= pos && first_item < part_end);
+            if (threadIdx.x == 0) s_bin[p - p_first] = bi;
         }
-        const uint2* list[TILES_PER_GROUP];
-        uint2 first[TILES_PER_GROUP];
-        uint32_t prob[TILES_PER_GROUP];
+        __syncthreads();
+        // (the loop bound is the same for all lanes of a warp: its shuffles stay whole)
+        for (uint32_t warp0 = pos + (threadIdx.x >> 5) * 4u * TILES_PER_GROUP; warp0 < part_end; warp0 += FILTER_TILES_PER_CTA) {
+            const uint32_t item0 = warp0 + ((threadIdx.x >> 3) & 3u) * TILES_PER_GROUP;
+            uint32_t cnt[TILES_PER_GROUP], base[TILES_PER_GROUP];
 #pragma unroll
-        for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-            const uint32_t item = item0 + u;
-            list[u] = nullptr; first[u] = make_uint2(0u, 0u); prob[u] = 0u;
-            if (item >= batch_end) continue;
-            const uint32_t w = item / L.tiles_per_worker;
-            const uint32_t lt = item - w * L.tiles_per_worker;
-            const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-            const SegEntry& seg = L.segs[s];
-            prob[u] = w * L.nseg + s;
-            if (!seg.fast) continue;
-            const BinInfo bi = s_bin[prob[u] - p_first];
-            if (!bi.live || bi.need2 == 0u || cnt[u] == 0u) continue;  // no candidate, or every candidate, is kept
-            list[u] = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + base[u];
-            if (sub < cnt[u]) first[u] = __ldg(list[u] + sub);
-        }
+            for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+                const uint32_t item = item0 + u;
+                cnt[u] = 0; base[u] = 0;
+                if (item < part_end) { cnt[u] = __ldg(P.tile_ccnt + item); base[u] = __ldg(P.tile_cbase + item); }
+            }
+            const uint2* list[TILES_PER_GROUP];
+            uint2 first[TILES_PER_GROUP];
+            uint32_t prob[TILES_PER_GROUP];
 #pragma unroll
-        for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
-            // candidates above the threshold's bin are kept whatever the exact threshold turns out to be; those
-            // inside the bin go to the short list, and the finish step adds the kept ones to the tile's count
-            uint32_t above = 0, inbin = 0;
-            if (list[u]) {
+            for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+                const uint32_t item = item0 + u;
+                list[u] = nullptr; first[u] = make_uint2(0u, 0u); prob[u] = 0u;
+                if (item >= part_end) continue;
+                const uint32_t w = item / L.tiles_per_worker;
+                const uint32_t lt = item - w * L.tiles_per_worker;
+                const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+                const SegEntry& seg = L.segs[s];
+                prob[u] = w * L.nseg + s;
+                if (!seg.fast) continue;
                 const BinInfo bi = s_bin[prob[u] - p_first];
-                const uint32_t s = prob[u] % L.nseg, w = prob[u] / L.nseg;
-                uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
-                for (uint32_t i0 = sub; i0 < cnt[u]; i0 += 32) {           // four entries in flight per lane
-                    uint2 c4[4];
+                if (!bi.live || bi.need2 == 0u || cnt[u] == 0u) continue;  // no candidate, or every candidate, is kept
+                list[u] = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + base[u];
+                if (sub < cnt[u]) first[u] = __ldg(list[u] + sub);
+            }
 #pragma unroll
-                    for (uint32_t v = 0; v < 4; ++v) {
-                        const uint32_t i = i0 + 8u * v;
-                        c4[v] = i == sub ? first[u] : (i < cnt[u] ? __ldg(list[u] + i) : make_uint2(0u, 0u));
-                    }
+            for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+                // candidates above the threshold's bin are kept whatever the exact threshold turns out to be; those
+                // inside the bin go to the short list, and the finish step adds the kept ones to the tile's count
+                uint32_t above = 0, inbin = 0;
+                if (list[u]) {
+                    const BinInfo bi = s_bin[prob[u] - p_first];
+                    const uint32_t w = prob[u] / L.nseg, s = prob[u] - w * L.nseg;
+                    uint2* out = P.list2 + ((size_t)w * L.fast_per_worker + L.segs[s].fast_index) * LIST2_CAP;
+                    for (uint32_t i0 = sub; i0 < cnt[u]; i0 += 32) {       // four entries in flight per lane
+                        uint2 c4[4];
 #pragma unroll
-                    for (uint32_t v = 0; v < 4; ++v) {
-                        if (i0 + 8u * v >= cnt[u]) continue;
-                        const uint2 c = c4[v];
-                        if (c.x > bi.hi2) ++above;
-                        else if (c.x >= bi.lo2) {
-                            ++inbin;
-                            const uint32_t pos = atomicAdd(&P.state[prob[u]].cnt2, 1u);
-                            if (pos < LIST2_CAP) out[pos] = c;
+                        for (uint32_t v = 0; v < 4; ++v) {
+                            const uint32_t i = i0 + 8u * v;
+                            c4[v] = i == sub ? first[u] : (i < cnt[u] ? __ldg(list[u] + i) : make_uint2(0u, 0u));
+                        }
+#pragma unroll
+                        for (uint32_t v = 0; v < 4; ++v) {
+                            if (i0 + 8u * v >= cnt[u]) continue;
+                            const uint2 c = c4[v];
+                            if (c.x > bi.hi2) ++above;
+                            else if (c.x >= bi.lo2) {
+                                ++inbin;
+                                const uint32_t pos2 = atomicAdd(&P.state[prob[u]].cnt2, 1u);
+                                if (pos2 < LIST2_CAP) out[pos2] = c;
+                            }
                         }
                     }
                 }
+                uint32_t both = above | (inbin << 16);                 // a tile holds at most 4096 candidates
+                both += __shfl_xor_sync(0xFFFFFFFFu, both, 1);
+                both += __shfl_xor_sync(0xFFFFFFFFu, both, 2);
+                both += __shfl_xor_sync(0xFFFFFFFFu, both, 4);
+                if (sub == 0u && item0 + u < part_end) P.tile_csum[item0 + u] = both;
             }
-            uint32_t both = above | (inbin << 16);                     // a tile holds at most 4096 candidates
-            both += __shfl_xor_sync(0xFFFFFFFFu, both, 1);
-            both += __shfl_xor_sync(0xFFFFFFFFu, both, 2);
-            both += __shfl_xor_sync(0xFFFFFFFFu, both, 4);
-            if (sub == 0u && item0 + u < batch_end) P.tile_csum[item0 + u] = both;
         }
+        pos = part_end;
     }
 }
 
@@ -834,7 +844,8 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
 //   distributed shared memory, and each CTA scans its share from the sum of the shares before it.
 // The cluster barriers are the hardware's; every CTA runs to the last one.
 constexpr uint32_t FINISH_CTAS = 8;
-constexpr uint32_t FINISH_PER = 8;                                     // tiles per thread and round of a scan
+constexpr uint32_t FINISH_PER = 16;                                    // tiles per thread and round of a scan
+constexpr uint32_t FINISH_SOLO_TILES = 4096;                           // below this many tiles CTA 0 serves the segment alone
 __device__ inline uint32_t block_sum(uint32_t v, uint32_t* s_scan) {
     uint32_t total;
     block_exclusive_scan(v, s_scan, &total);
@@ -855,6 +866,9 @@ topk_finish_kernel(const __grid_constant__ FastParams P) {
     FastState st = P.state[prob];
     if (st.path != PATH_FAST) return;                                  // the same answer in every CTA of the cluster
     const uint32_t ntiles = L.segs[s + 1].tile_begin - seg.tile_begin;
+    const bool solo = ntiles < FINISH_SOLO_TILES;                      // no cluster barrier at all then
+    if (solo && rank != 0) return;
+    const uint32_t ranks = solo ? 1u : FINISH_CTAS;
     const size_t item0 = (size_t)w * L.tiles_per_worker + seg.tile_begin;
     const bool admit = st.need_ties != 0u;
     if (rank == 0) {
@@ -930,12 +944,12 @@ topk_finish_kernel(const __grid_constant__ FastParams P) {
         if (threadIdx.x == 0) s_share[2] = failed ? 1u : 0u;
         __threadfence();                                               // the counts above are in L2 before the peers read them
     }
-    cluster.sync();
-    const bool give_up = *cluster.map_shared_rank(&s_share[2], 0) != 0u;
+    if (solo) __syncthreads(); else cluster.sync();
+    const bool give_up = (solo ? s_share[2] : *cluster.map_shared_rank(&s_share[2], 0)) != 0u;
     if (!give_up) {
         // ---- kept count per tile, exclusive sum over the segment's tiles ------------------------------
         constexpr uint32_t ROUND = THREADS * FINISH_PER;
-        const uint32_t per = ((ntiles + FINISH_CTAS - 1) / FINISH_CTAS + ROUND - 1) / ROUND * ROUND;
+        const uint32_t per = ((ntiles + ranks - 1) / ranks + ROUND - 1) / ROUND * ROUND;
         const uint32_t begin = min(rank * per, ntiles), end = min(begin + per, ntiles);
         uint32_t* off = P.offsets + (size_t)w * (L.tiles_per_worker + 1) + seg.tile_begin;
         uint32_t tie_run = 0;                                          // tie-key elements of the segment before the current tile
@@ -944,7 +958,7 @@ topk_finish_kernel(const __grid_constant__ FastParams P) {
             for (uint32_t t = begin + threadIdx.x; t < end; t += THREADS) tsum += __ldcg(P.tile_tie + item0 + t);
             tsum = block_sum(tsum, s_scan);
             if (threadIdx.x == 0) s_share[0] = tsum;
-            cluster.sync();
+            if (!solo) cluster.sync();
             for (uint32_t r = 0; r < rank; ++r) tie_run += *cluster.map_shared_rank(&s_share[0], r);
         }
         // first round over the share: how many ties each tile admits, and the share's kept total
@@ -984,7 +998,7 @@ topk_finish_kernel(const __grid_constant__ FastParams P) {
         }
         ksum = block_sum(ksum, s_scan);
         if (threadIdx.x == 0) s_share[1] = ksum;
-        cluster.sync();
+        if (!solo) cluster.sync();
         uint32_t kept_run = 0;
         for (uint32_t r = 0; r < rank; ++r) kept_run += *cluster.map_shared_rank(&s_share[1], r);
         // second round: the tiles' first message slots
@@ -1010,9 +1024,9 @@ topk_finish_kernel(const __grid_constant__ FastParams P) {
                 ex += kept[i];
             }
         }
-        if (rank == FINISH_CTAS - 1u && threadIdx.x == 0 && kept_run != seg.k) atomicMin(P.status, ST_DEVICE_CHECK);   // counts and k disagree
+        if (rank == ranks - 1u && threadIdx.x == 0 && kept_run != seg.k) atomicMin(P.status, ST_DEVICE_CHECK);   // counts and k disagree
     }
-    cluster.sync();                                                    // a peer's totals must outlive their readers
+    if (!solo) cluster.sync();                                         // a peer's totals must outlive their readers
 }
 
 // ---- emit: G lanes per tile walk the tile's slice of the flagged list ----------------------------
