@@ -135,6 +135,30 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
     }
 }
 
+// The part of one worker's slice that the register rounds of the two kernels below do not cover (dense
+// stretches of a message: ties admitted from the lowest coordinate up, a block of the block scheme).  Eight
+// rounds of 32 entries are requested together, so that the loop costs one memory latency per 256 entries
+// instead of one per 32; the entries of one worker have distinct coordinates, so their order does not matter.
+__device__ inline void add_rest_of_slice(const uint32_t* __restrict__ idx_row, const float* __restrict__ val_row, uint32_t from,
+                                         uint32_t to, uint32_t base, uint32_t cnt_here, float* acc, uint32_t lane) {
+    constexpr int U = 8;
+    for (uint32_t j0 = from + lane; j0 < to; j0 += 32u * U) {
+        uint32_t ix[U];
+        float vv[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t j = j0 + 32u * u;
+            ix[u] = 0xFFFFFFFFu; vv[u] = 0.0f;
+            if (j < to) { ix[u] = __ldg(idx_row + j); vv[u] = __ldg(val_row + j); }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t loc = ix[u] - base;
+            if (loc < cnt_here) acc[loc] = acc[loc] + vv[u];
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Sparse messages with different coordinates per worker (top-k at the usual densities): one WARP
 // owns 1024 coordinates.  It reads, for eight workers at a time, the workers' slices of the
@@ -143,6 +167,7 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
 // No shared staging area, no CTA-wide barrier: the warps of a CTA never wait for each other.
 // ---------------------------------------------------------------------------------------------
 constexpr uint32_t AWARP = 1024;                 // coordinates per warp
+
 constexpr uint32_t AWARP_BATCH = 8;              // workers whose slices are fetched together
 constexpr uint32_t AWARP_MAX_SLICE = 64;         // entries of one worker in one 4096-tile served by the fast loop
 
@@ -196,13 +221,9 @@ agg_warp_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ idx
                     const uint32_t loc = ix[u][h] - base;
                     if (loc < cnt_here) acc[loc] = acc[loc] + vv[u][h];
                 }
-                if (hi[u] - lo[u] > AWARP_MAX_SLICE) {                    // a long slice: finish it before the next worker
-                    const size_t row = (size_t)(w0 + u) * K;
-                    for (uint32_t j = lo[u] + AWARP_MAX_SLICE + lane; j < hi[u]; j += 32) {
-                        const uint32_t loc = __ldg(idx + row + j) - base;
-                        if (loc < cnt_here) acc[loc] = acc[loc] + __ldg(vals + row + j);
-                    }
-                }
+                if (hi[u] - lo[u] > AWARP_MAX_SLICE)                      // a long slice: finish it before the next worker
+                    add_rest_of_slice(idx + (size_t)(w0 + u) * K, vals + (size_t)(w0 + u) * K, lo[u] + AWARP_MAX_SLICE, hi[u],
+                                      base, cnt_here, acc, lane);
                 __syncwarp();
             }
         }
@@ -311,13 +332,9 @@ agg_warp_fine_kernel(const float* __restrict__ vals, const uint32_t* __restrict_
                     const uint32_t loc = ix[u][h] - base;
                     if (loc < cnt_here) acc[loc] = acc[loc] + vv[u][h];
                 }
-                if (hi[u] - lo[u] > 32u * H) {                               // a long slice: finish it before the next worker
-                    const size_t row = (size_t)(w0 + u) * K;
-                    for (uint32_t j = lo[u] + 32u * H + lane; j < hi[u]; j += 32) {
-                        const uint32_t loc = __ldg(idx + row + j) - base;
-                        if (loc < cnt_here) acc[loc] = acc[loc] + __ldg(vals + row + j);
-                    }
-                }
+                if (hi[u] - lo[u] > 32u * H)                                 // a long slice: finish it before the next worker
+                    add_rest_of_slice(idx + (size_t)(w0 + u) * K, vals + (size_t)(w0 + u) * K, lo[u] + 32u * H, hi[u],
+                                      base, cnt_here, acc, lane);
                 __syncwarp();
             }
         }

@@ -104,7 +104,9 @@ struct FastState {
                            // counted per tile instead of being listed (massive ties around the threshold)
     uint32_t tie_total;    // elements with key == tie_key
     uint32_t need_ties;    // how many of them are kept, lowest coordinates first (then T == tie_key)
-    uint32_t pad0, pad1;
+    uint32_t zcut;         // the streaming pass zeroes flagged elements with key > zcut at once (the sample's estimate of
+                           // the threshold; the emit step corrects the few it got wrong)
+    uint32_t pad1;
     uint32_t ext_used;     // slots handed out from the flagged list's extension pool
     uint32_t fail;         // FAIL_*: why the one-pass path gave up
     uint32_t expect2;      // entries the short list must hold (from the candidate histogram)

@@ -9,8 +9,8 @@
 //            probability.  A key value that holds a large share of the sample at the lower order
 //            statistic (exact zeros of a sparse gradient, a constant tensor) becomes the "tie key":
 //            its elements are counted per tile instead of being listed;
-//   main     the streaming pass forms p = g + e and writes the residual at once: 0 for the
-//            "sure" elements (key > hi), p for the rest.  Every element with key >= lo is
+//   main     the streaming pass forms p = g + e and writes the residual at once: 0 for the elements
+//            above the sample's own estimate of the threshold, p for the rest.  Every element with key >= lo is
 //            appended, in coordinate order inside its tile, to a "flagged" list (value,
 //            coordinate); the few candidates (lo <= key <= hi) also go to a candidate list
 //            and into a 2048-bin histogram.  The CTA that finishes a segment's last tile reads
@@ -21,8 +21,10 @@
 //            cut for ties), admits tie-key elements by coordinate order if the threshold is the
 //            tie key, and scans the per-tile kept counts into message offsets;
 //   emit     a pass over the flagged list only: kept entries go to the message in ascending
-//            coordinate order, kept candidates are zeroed in the residual; tiles that admit
-//            tie-key elements are re-read from the residual instead.
+//            coordinate order; the few entries between the estimated and the exact threshold are
+//            corrected in the residual (scattered accesses to DRAM cost a row cycle each, so as few
+//            as possible are left for this step); tiles that admit tie-key elements are re-read from
+//            the residual instead.
 // Every count is exact, so the result equals the plain definition; the sample only decides how
 // much work that takes.  If the bracket is wrong (counts prove it) or a list overflows, the
 // segment falls back to the radix select on the parked p.
@@ -142,9 +144,9 @@ __global__ void __launch_bounds__(THREADS)
 topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     namespace cg = cooperative_groups;
     __shared__ uint32_t h0[HIST0_BINS];
-    __shared__ uint32_t hA[1024], hB[1024], hC[1024];
+    __shared__ uint32_t hA[1024], hB[1024], hC[1024], hM[1024];
     __shared__ uint32_t s_tmp[WARPS + 4];
-    __shared__ uint32_t s_bins[8];                                     // valid in CTA 0: binA, binB, needA, needB, round 3?, prefix B
+    __shared__ uint32_t s_bins[8];                                     // valid in CTA 0: binA, binB, needA, needB, round 3?, prefix B, binM, needM
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t rank = C > 1 ? cluster.block_rank() : 0u;
     const Layout& L = P.L;
@@ -167,7 +169,7 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     const bool have_hi = j_hi >= 1, have_lo = j_lo <= (long long)m;
 
     for (uint32_t b = threadIdx.x; b < HIST0_BINS; b += THREADS) h0[b] = 0;
-    for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) { hA[b] = 0; hB[b] = 0; hC[b] = 0; }
+    for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) { hA[b] = 0; hB[b] = 0; hC[b] = 0; hM[b] = 0; }
     __syncthreads();
     {   // ---- the sample: sector c of the sample is sector floor(c sectors / S) of the segment's aligned part
         const size_t row = (size_t)w * L.n_total + seg.offset;
@@ -217,14 +219,17 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
         }
         __syncthreads();
         const uint32_t rankA = have_hi ? (uint32_t)j_hi : 1u, rankB = have_lo ? (uint32_t)j_lo : m;
-        uint32_t binA = 0, needA = 0, binB = 0, needB = 0, cnt = 0;
+        // the sample's own estimate of the k-th key: the statistic in the middle
+        const uint32_t rankM = (uint32_t)min(max((long long)llround(centre), 1ll), (long long)m);
+        uint32_t binA = 0, needA = 0, binB = 0, needB = 0, binM = 0, needM = 0, cnt = 0;
         find_from_top<HIST0_BINS>(h0, rankA, s_tmp, binA, needA, cnt);
         find_from_top<HIST0_BINS>(h0, rankB, s_tmp, binB, needB, cnt);
-        if (threadIdx.x == 0) { s_bins[0] = binA; s_bins[1] = binB; s_bins[2] = needA; s_bins[3] = needB; }
+        find_from_top<HIST0_BINS>(h0, rankM, s_tmp, binM, needM, cnt);
+        if (threadIdx.x == 0) { s_bins[0] = binA; s_bins[1] = binB; s_bins[2] = needA; s_bins[3] = needB; s_bins[6] = binM; s_bins[7] = needM; }
     }
     if (C > 1) cluster.sync(); else __syncthreads();
     const uint32_t* bins0 = C > 1 ? cluster.map_shared_rank(s_bins, 0) : s_bins;
-    const uint32_t binA = bins0[0], binB = bins0[1];
+    const uint32_t binA = bins0[0], binB = bins0[1], binM = bins0[6];
     for (uint32_t c = c_begin + threadIdx.x; c < c_end; c += THREADS) {
         const uint4 k0 = smp[2 * (size_t)c], k1 = smp[2 * (size_t)c + 1];
         const uint32_t kk[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
@@ -232,24 +237,27 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
         for (int i = 0; i < 8; ++i) {
             if ((kk[i] >> 20) == binA) atomicAdd(&hA[(kk[i] >> 10) & 1023u], 1u);
             if ((kk[i] >> 20) == binB) atomicAdd(&hB[(kk[i] >> 10) & 1023u], 1u);
+            if ((kk[i] >> 20) == binM) atomicAdd(&hM[(kk[i] >> 10) & 1023u], 1u);
         }
     }
     if (C > 1) cluster.sync(); else __syncthreads();
-    uint32_t bin1A = 0, need2A = 0, bin1B = 0, need2B = 0;             // valid in CTA 0
-    bool okA = false, okB = false;
+    uint32_t bin1A = 0, need2A = 0, bin1B = 0, need2B = 0, bin1M = 0;  // valid in CTA 0
+    bool okA = false, okB = false, okM = false;
     if (rank == 0) {
         for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) {
-            uint32_t va = hA[b], vb = hB[b];
+            uint32_t va = hA[b], vb = hB[b], vm = hM[b];
             for (uint32_t r = 1; r < C; ++r) {
                 va += cluster.map_shared_rank(hA, r)[b];
                 vb += cluster.map_shared_rank(hB, r)[b];
+                vm += cluster.map_shared_rank(hM, r)[b];
             }
-            hA[b] = va; hB[b] = vb;
+            hA[b] = va; hB[b] = vb; hM[b] = vm;
         }
         __syncthreads();
-        uint32_t cntA = 0, cntB = 0;
+        uint32_t cntA = 0, cntB = 0, cntM = 0, need2M = 0;
         okA = find_from_top<1024>(hA, s_bins[2], s_tmp, bin1A, need2A, cntA);
         okB = find_from_top<1024>(hB, s_bins[3], s_tmp, bin1B, need2B, cntB);
+        okM = find_from_top<1024>(hM, s_bins[7], s_tmp, bin1M, need2M, cntM);
         if (threadIdx.x == 0) {
             s_bins[4] = (okB && massive_in_sample(cntB, m)) ? 1u : 0u;
             s_bins[5] = (binB << 10) | bin1B;
@@ -297,6 +305,8 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
             FastState st = {};
             st.path = PATH_FAST; st.lo = lo; st.hi = hi; st.shift = bits > 11u ? bits - 11u : 0u;
             st.tie_key = tie_key;
+            // with a tie key the residual has to keep p everywhere (the emit step re-reads tiles from it)
+            st.zcut = tie_key != TIE_NONE ? 0x7FFFFFFFu : (okM ? min((binM << 20) | (bin1M << 10) | 511u, hi) : hi);
             P.state[prob] = st;
         }
     }
@@ -413,7 +423,7 @@ __device__ inline MainTile main_decode(const FastParams& P, uint32_t item) {
 struct MainSeg {
     uint32_t hi, shift, tie_key, ccap;
     uint32_t flag_cap, region_per_tile, ext_begin, ext_cap;
-    uint32_t ext_chunk, cov_cap, pad0, pad1;
+    uint32_t ext_chunk, cov_cap, zcut, pad1;
     uint2* flist;                  // the segment's flagged list of this worker
     uint2* clist;                  // its candidate list
     uint2* cover;                  // its candidate overflow list
@@ -516,7 +526,7 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
                 MainSeg m;
                 m.hi = st->hi; m.shift = st->shift; m.tie_key = st->tie_key; m.ccap = seg->cand_cap;
                 m.flag_cap = seg->flag_cap; m.region_per_tile = seg->region_per_tile; m.ext_begin = seg->ext_begin; m.ext_cap = seg->ext_cap;
-                m.ext_chunk = seg->ext_chunk; m.cov_cap = seg->cov_cap; m.pad0 = 0; m.pad1 = 0;
+                m.ext_chunk = seg->ext_chunk; m.cov_cap = seg->cov_cap; m.zcut = st->zcut; m.pad1 = 0;
                 m.flist = P.flagged + (size_t)T.w * L.flag_per_worker + seg->flag_begin;
                 m.clist = P.cand + (size_t)T.w * L.cand_per_worker + seg->cand_begin;
                 m.cover = P.cand + (size_t)T.w * L.cand_per_worker + seg->cov_begin;
@@ -662,15 +672,14 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
         }
         if (fits && wflag) {
             // the tile's entries fit: write them (entry r of the warp's slice by lane r % 32: coalesced), zero
-            // the sure ones in the residual (their values stay in the list, from where a fall-back restores
-            // them; with a tie key the residual keeps p everywhere, so that the emit step can still tell a kept
-            // element from a tie), append the candidates to the tile's slice and histogram them
+            // the ones above the estimated threshold in the residual while the tile's lines are still in L2 (their
+            // values stay in the list, from where the emit step or a fall-back puts back what should not have
+            // been zeroed), append the candidates to the tile's slice and histogram them
             uint2* flist = s_seg.flist + fbase + fwbase;
             uint2* clist = s_seg.clist + cbase;
-            const uint32_t hi = s_seg.hi, shift = s_seg.shift;
+            const uint32_t hi = s_seg.hi, shift = s_seg.shift, zcut = s_seg.zcut;
             const uint32_t first32 = (uint32_t)T.first + warp * 512u;
             const float* spw = sp + warp * 512u;
-            const bool zero_now = tie_key == TIE_NONE;
             uint32_t sure_w = 0;
             for (uint32_t r0 = 0; r0 < wflag; r0 += 32) {
                 const uint32_t r = r0 + lane;
@@ -682,7 +691,7 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
                 const bool sure = active && key > hi;
                 const bool cand = active && key <= hi;
                 if (active) flist[r] = make_uint2(__float_as_uint(v), coord);
-                if (sure && zero_now) e[coord] = 0.0f;
+                if (active && key > zcut) e[coord] = 0.0f;
                 const uint32_t bs = __ballot_sync(0xFFFFFFFFu, sure);
                 const uint32_t bc = __ballot_sync(0xFFFFFFFFu, cand);
                 sure_w += __popc(bs);
@@ -1051,7 +1060,7 @@ topk_emit_kernel(FastParams P) {
     const uint32_t rounds = (P.total_items + stride - 1) / stride;      // the same for every lane: ballots stay whole
     // per-(worker, segment) constants stay in registers while the group's tiles belong to the same one
     uint32_t cw = 0xFFFFFFFFu, cs = 0xFFFFFFFFu, c_tile_end = 0;        // cached worker, segment, end of its tile range
-    uint32_t T = 0, icut = 0, hi = 0, seg_k = 0, idx0 = 0, tile_begin = 0;
+    uint32_t T = 0, icut = 0, zcut = 0, seg_k = 0, idx0 = 0, tile_begin = 0;
     bool live = false, admits = false;
     const uint2* flist0 = nullptr;
     float* e = nullptr;
@@ -1072,7 +1081,7 @@ topk_emit_kernel(FastParams P) {
                 live = seg.fast && st->path == PATH_FAST;
                 admits = st->need_ties != 0u;
                 T = st->T; icut = st->icut; seg_k = seg.k; idx0 = (uint32_t)seg.offset;
-                hi = st->tie_key != TIE_NONE ? 0x7FFFFFFFu : st->hi;    // with a tie key the streaming pass zeroed nothing
+                zcut = st->zcut;                                        // the streaming pass zeroed the entries above this key
                 flist0 = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin;
                 e = P.residuals + (size_t)w * L.n_total + seg.offset;
                 ovals = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
@@ -1108,7 +1117,9 @@ topk_emit_kernel(FastParams P) {
                     } else {                                            // counts and k disagree
                         atomicMin(P.status, ST_DEVICE_CHECK);
                     }
-                    if (key <= hi) e[a[u].y] = 0.0f;                    // the streaming pass left p there
+                    if (key <= zcut) e[a[u].y] = 0.0f;                  // the streaming pass left p there
+                } else if (key > zcut) {
+                    e[a[u].y] = __uint_as_float(a[u].x);                // zeroed by the streaming pass, but not kept
                 }
                 pos += __popc(bal);
             }
@@ -1184,14 +1195,14 @@ __device__ inline void restore_failed_segments(const FastParams& P) {
         const SegEntry seg = L.segs[s];
         if (!seg.fast) continue;
         const FastState* st = P.state + (size_t)w * L.nseg + s;
-        if (st->path != PATH_FAILED || st->tie_key != TIE_NONE) continue;   // with a tie key nothing was zeroed
-        const uint32_t base = P.tile_fbase[item], cnt = P.tile_fcnt[item], hi = st->hi;
+        if (st->path != PATH_FAILED) continue;
+        const uint32_t base = P.tile_fbase[item], cnt = P.tile_fcnt[item], zcut = st->zcut;
         if (base == 0xFFFFFFFFu || cnt == 0u) continue;                 // nothing was written, nothing was zeroed
         const uint2* flist = P.flagged + (size_t)w * L.flag_per_worker + seg.flag_begin + base;
         float* e = P.residuals + (size_t)w * L.n_total + seg.offset;
         for (uint32_t i = lane; i < cnt; i += 32) {
             const uint2 a = flist[i];
-            if ((a.x & 0x7FFFFFFFu) > hi) e[a.y] = __uint_as_float(a.x);
+            if ((a.x & 0x7FFFFFFFu) > zcut) e[a.y] = __uint_as_float(a.x);
         }
     }
 }
