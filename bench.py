@@ -528,6 +528,21 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             torch.cuda.synchronize()
             ctx.sc_set_gamma(1.0)
             return round(a.elapsed_time(b) / 3, 4)
+        def timed_step_apply(code):
+            e_tmp = res[schemes[-1]]
+            xm = torch.zeros(n, device=dev)
+            ctx.sc_step_apply(code, grads[0], e_tmp, seg_t, seeds(0), vals, idx, xm)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for t in range(3):
+                ctx.sc_step_apply(code, grads[t % pool], e_tmp, seg_t, seeds(t + 1), vals, idx, xm)
+            b.record()
+            torch.cuda.synchronize()
+            return round(a.elapsed_time(b) / 3, 4)
+        for s_ in schemes:
+            tim[f"{s_}_step_apply_ms"] = timed_step_apply(sc.SCHEMES[s_])
+        tim["note_step_apply"] = ("sc_step_apply: the whole step with x <- x - average applied at the sent coordinates "
+                                  "instead of writing the dense average (compare per_scheme.*.ms)")
         tim["randblock_wrap_step_ms"] = timed_step(sc.SC_RANDBLOCK_WRAP, 1.0)
         tim["topk_step_gamma_0.1_ms"] = timed_step(sc.SC_TOPK, 0.1)
         tim["note_steps"] = ("whole sc_step (compress + aggregate) on this workload: wrap-around block scheme; "

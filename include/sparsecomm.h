@@ -192,6 +192,14 @@ int sc_step(sc_ctx* ctx, int scheme, int W, const float* grads, float* residuals
             const sc_segment* segs, int nseg, const uint64_t* h_seeds,
             float* out_vals, uint32_t* out_idx, float* out, void* stream);
 
+/* One whole step of Algorithm 1 without the dense average: sc_compress_batch followed by the
+ * model-update line applied at the sent coordinates only, x[i] <- x[i] - (sum over w, in order, from
+ * +0.0, of q^w[i]) / W (the same bits as sc_step followed by x - out, see sc_aggregate_apply).  x[n] is
+ * updated in place; no dense vector of n elements is written or read besides g, e and the touched x. */
+int sc_step_apply(sc_ctx* ctx, int scheme, int W, const float* grads, float* residuals, size_t n,
+                  const sc_segment* segs, int nseg, const uint64_t* h_seeds,
+                  float* out_vals, uint32_t* out_idx, float* x, void* stream);
+
 /* One whole step with the step's inputs and result in HOST memory: h_grads
  * (W rows of n, ideally pinned) is copied to device staging owned by the
  * context, worker by worker, overlapped with the compression of the previous

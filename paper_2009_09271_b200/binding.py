@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libsparsecomm.so")
 EXPORTS = ["sc_create", "sc_destroy", "sc_strerror", "sc_sync_status", "sc_set_gamma", "sc_scratch_bytes", "sc_launch_count",
            "sc_topk_path_counts", "sc_topk_path_detail", "sc_debug_set_poll_limits", "sc_debug_wait_probe", "sc_profile", "sc_profile_kinds", "sc_profile_name", "sc_profile_read",
            "sc_compress", "sc_compress_batch", "sc_aggregate", "sc_aggregate_shared", "sc_aggregate_static", "sc_aggregate_apply",
-           "sc_aggregate_apply_shared", "sc_step", "sc_step_host"]
+           "sc_aggregate_apply_shared", "sc_step", "sc_step_apply", "sc_step_host"]
 
 
 class ScSegment(ctypes.Structure):
@@ -94,6 +94,8 @@ def load_library() -> ctypes.CDLL:
     lib.sc_step.argtypes = [vp, ci, ci, vp, vp, sz, ctypes.POINTER(ScSegment), ci, ctypes.POINTER(u64),
                             vp, vp, vp, vp]
     lib.sc_step.restype = ci
+    lib.sc_step_apply.argtypes = lib.sc_step.argtypes
+    lib.sc_step_apply.restype = ci
     lib.sc_step_host.argtypes = [vp, ci, ci, vp, vp, sz, ctypes.POINTER(ScSegment), ci, ctypes.POINTER(u64),
                                  vp, vp]
     lib.sc_step_host.restype = ci
@@ -277,6 +279,20 @@ class Context:
         _check(self._lib.sc_step(self._h, scheme, W, _ptr(grads), _ptr(residuals), n, _segments(segs), len(segs),
                                  _seeds(seeds), _ptr(out_vals), _ptr(out_idx), _ptr(out), _stream(stream)),
                "sc_step")
+
+    def sc_step_apply(self, scheme: int, grads, residuals, segs, seeds, out_vals, out_idx, x, stream=None) -> None:
+        """Compress W workers, then x <- x - average of their messages at the sent coordinates only."""
+        W, n = grads.shape
+        _want(grads, torch.float32, "grads"), _want(residuals, torch.float32, "residuals")
+        _want(out_vals, torch.float32, "out_vals"), _want(out_idx, torch.int32, "out_idx")
+        _want(x, torch.float32, "x")
+        K = sum((s.k if hasattr(s, "k") else s[2]) for s in segs)
+        if (residuals.shape != grads.shape or len(seeds) != W or out_vals.numel() < W * K
+                or out_idx.numel() < W * K or x.numel() < n):
+            raise ValueError("buffer sizes do not match W, n and the segment table")
+        _check(self._lib.sc_step_apply(self._h, scheme, W, _ptr(grads), _ptr(residuals), n, _segments(segs), len(segs),
+                                       _seeds(seeds), _ptr(out_vals), _ptr(out_idx), _ptr(x), _stream(stream)),
+               "sc_step_apply")
 
     def sc_step_host(self, scheme: int, h_grads, residuals, segs, seeds, h_out, stream=None) -> None:
         W, n = h_grads.shape

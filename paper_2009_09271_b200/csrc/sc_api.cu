@@ -602,6 +602,29 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
     return SC_OK;
 }
 
+// x <- x - average of the W messages, at the coordinates that were sent only.
+int apply_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, bool shared_idx, size_t k, size_t n, float* x,
+               cudaStream_t st) {
+    if (n == 0 || k == 0) return SC_OK;
+    if (shared_idx) {
+        Launch l(c, KIND_AGG_APPLY, st);
+        const uint64_t blocks = (k + THREADS - 1) / THREADS;
+        agg_apply_shared_kernel<<<persistent_grid(c, 8, blocks), THREADS, 0, st>>>(
+            vals, idx, (uint32_t)W, (uint32_t)k, (uint32_t)n, x, c->d_status);
+    } else {
+        const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
+        const uint64_t threads = (uint64_t)W * (ntiles + 1ull);
+        { Launch l(c, KIND_AGG_BOUNDS, st);
+          agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, st>>>(
+              idx, (uint32_t)W, (uint32_t)k, ntiles, ATILE, c->d_bounds); }
+        { Launch l(c, KIND_AGG_APPLY, st);
+          agg_apply_tiles_kernel<ATILE><<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, st>>>(
+              vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, x, c->d_status); }
+    }
+    SC_CUDA(cudaGetLastError());
+    return SC_OK;
+}
+
 int check_aggregate_args(const sc_ctx* c, int W, const void* vals, const void* idx, size_t k, size_t n, const void* out) {
     if (!c) return SC_ERR_INVALID;
     if (W < 1 || W > c->max_W) return SC_ERR_RANGE;
@@ -890,34 +913,16 @@ int sc_aggregate_apply(sc_ctx* c, int W, const float* vals, const uint32_t* idx,
                        float* x, void* stream) {
     int rc = check_aggregate_args(c, W, vals, idx, k, n, x);
     if (rc != SC_OK) return rc;
-    if (n == 0 || k == 0) return SC_OK;
     DeviceGuard guard(c->device);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const uint32_t ntiles = (uint32_t)((n + ATILE - 1) / ATILE);
-    const uint64_t threads = (uint64_t)W * (ntiles + 1ull);
-    { Launch l(c, KIND_AGG_BOUNDS, st);
-      agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, st>>>(
-          idx, (uint32_t)W, (uint32_t)k, ntiles, ATILE, c->d_bounds); }
-    { Launch l(c, KIND_AGG_APPLY, st);
-      agg_apply_tiles_kernel<ATILE><<<persistent_grid(c, c->occ_agg, ntiles), THREADS, 0, st>>>(
-          vals, idx, c->d_bounds, (uint32_t)W, (uint32_t)k, (uint32_t)n, ntiles, x, c->d_status); }
-    SC_CUDA(cudaGetLastError());
-    return SC_OK;
+    return apply_rows(c, W, vals, idx, false, k, n, x, static_cast<cudaStream_t>(stream));
 }
 
 int sc_aggregate_apply_shared(sc_ctx* c, int W, const float* vals, const uint32_t* idx, size_t k, size_t n,
                               float* x, void* stream) {
     int rc = check_aggregate_args(c, W, vals, idx, k, n, x);
     if (rc != SC_OK) return rc;
-    if (n == 0 || k == 0) return SC_OK;
     DeviceGuard guard(c->device);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    { Launch l(c, KIND_AGG_APPLY, st);
-      const uint64_t blocks = (k + THREADS - 1) / THREADS;
-      agg_apply_shared_kernel<<<persistent_grid(c, 8, blocks), THREADS, 0, st>>>(
-          vals, idx, (uint32_t)W, (uint32_t)k, (uint32_t)n, x, c->d_status); }
-    SC_CUDA(cudaGetLastError());
-    return SC_OK;
+    return apply_rows(c, W, vals, idx, true, k, n, x, static_cast<cudaStream_t>(stream));
 }
 
 int sc_step(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
@@ -933,6 +938,21 @@ int sc_step(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, 
     if ((rc = compress_rows(c, scheme, W, grads, residuals, n, h_seeds, shared, false, out_vals, out_idx, st)) != SC_OK)
         return rc;
     return aggregate_rows(c, W, out_vals, out_idx, shared && scheme != SC_TOPK, c->layout.K_total, n, out, st);
+}
+
+int sc_step_apply(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
+                  const sc_segment* segs, int nseg, const uint64_t* h_seeds,
+                  float* out_vals, uint32_t* out_idx, float* x, void* stream) {
+    int rc = check_batch_args(c, scheme, W, grads, residuals, n, segs, nseg, h_seeds, out_vals, out_idx);
+    if (rc != SC_OK) return rc;
+    if ((n > 0 && !x) || !aligned16(x)) return SC_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = prepare_layout(c, n, segs, nseg, st)) != SC_OK) return rc;
+    const bool shared = all_equal(h_seeds, W);
+    if ((rc = compress_rows(c, scheme, W, grads, residuals, n, h_seeds, shared, false, out_vals, out_idx, st)) != SC_OK)
+        return rc;
+    return apply_rows(c, W, out_vals, out_idx, shared && scheme != SC_TOPK, c->layout.K_total, n, x, st);
 }
 
 int sc_step_host(sc_ctx* c, int scheme, int W, const float* h_grads, float* residuals, size_t n,

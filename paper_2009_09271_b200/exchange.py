@@ -3,7 +3,9 @@
 The paper exchanges the sparse messages with allGather when the workers kept different
 coordinates and with allReduce when they kept the same ones (Methodology, third parameter).
 Here the collectives are torch.distributed (NCCL over NVLink on GPUs); the received
-messages land in this GPU's own memory and the aggregate kernels read them from there.
+messages land in this GPU's own memory, already in the W x k row layout the aggregate kernels
+read, and the aggregate is enqueued on the caller's stream right behind the collective: torch
+orders the two with a stream event, the host never waits in between.
 
     vals, idx  : this rank's message, k entries (from sc_compress / sc_compress_batch with W = 1)
     exchange_messages(...) -> (vals_all [W, k], idx rows) ready for sc_aggregate / sc_aggregate_shared
@@ -63,3 +65,13 @@ def exchange_and_aggregate(ctx, vals: torch.Tensor, idx: torch.Tensor, n: int, o
         ctx.sc_aggregate_shared(rows, v, i.view(-1), k, n, out)
     else:
         ctx.sc_aggregate(rows, v, i, k, n, out)
+
+
+def exchange_and_apply(ctx, vals: torch.Tensor, idx: torch.Tensor, n: int, x: torch.Tensor,
+                       shared_coordinates: bool, mode: str = "allgather",
+                       group: Optional[dist.ProcessGroup] = None) -> None:
+    """Algorithm 1, exchange + aggregate + model-update lines on one rank: x[n] <- x - average of all ranks'
+    messages, touching only the coordinates some rank sent (no dense vector is formed)."""
+    k = vals.numel()
+    v, i, rows = exchange_messages(vals, idx, shared_coordinates, mode, group)
+    ctx.sc_aggregate_apply(rows, v, i.view(-1), k, n, x, shared=shared_coordinates)

@@ -583,3 +583,25 @@ def test_aggregate_apply_denormal_sums(W):
     assert c.sc_sync_status() == 0
     assert_bits_equal(xs, O.aggregate_apply(x0, list(vals), [idx[0]] * W), "apply shared, denormals")
     c.close()
+
+
+@pytest.mark.parametrize("scheme", SCHEMES)
+def test_step_apply_matches_step_then_update(ctx, scheme):
+    """sc_step_apply: compress, then x <- x - average at the sent coordinates; the same bits as the dense form."""
+    W, sizes = 4, [70_001, 300, 4099, 131_072 + 9]
+    segs = [(s.offset, s.n, s.k) for s in wl.segment_table(sizes, 1, 50)]
+    n, K = sum(sizes), sum(s[2] for s in segs)
+    x0 = rand(n, 1500, scale=1.0)
+    for seeds in ([3] * W, [3, 4, 5, 6]):
+        g = torch.stack([rand(n, 1510 + w) for w in range(W)])
+        e0 = torch.stack([rand(n, 1520 + w, scale=1e-4) for w in range(W)])
+        e = e0.cuda().clone()
+        x = x0.cuda().clone()
+        vals = torch.empty(W, K, device="cuda"); idx = torch.empty(W, K, device="cuda", dtype=torch.int32)
+        ctx.sc_step_apply(scheme, g.cuda(), e, segs, seeds, vals, idx, x)
+        assert ctx.sc_sync_status() == 0
+        ov, oi, oe, _ = O.step(scheme, [g[w].numpy() for w in range(W)], [e0[w].numpy() for w in range(W)], segs, seeds)
+        for w in range(W):
+            assert_bits_equal(e[w], oe[w], f"residual[w={w}]")
+            assert_bits_equal(idx[w], oi[w], f"idx[w={w}]")
+        assert_bits_equal(x, O.aggregate_apply(x0.numpy(), ov, oi), "model")
