@@ -63,7 +63,7 @@ struct sc_ctx {
     size_t flagged_slots = 0;
     size_t max_fast_per_worker = 0, max_cand_per_worker = 0;
     uint32_t last_topk_problems = 0; // (worker, segment) pairs of the most recent top-k call
-    uint32_t max_sample_m = 0, fast_big = 0;
+    uint32_t max_sample_m = 0, fast_big = 0, fast_huge = 0;   // of the fast list: the first fast_huge are long segments, the first fast_big have large samples
     float gamma = 1.0f;                  // step size of the accumulate line (sc_set_gamma)
     int occ_main = 1, occ_main_wide = 1, occ_emit_v[4] = {1, 1, 1, 1}, occ_fallback = 1, occ_filter = 1;
     uint32_t lookback_poll_limit = LOOKBACK_POLL_LIMIT, barrier_poll_limit = BARRIER_POLL_LIMIT;
@@ -94,6 +94,8 @@ struct sc_ctx {
     float* d_stage_out = nullptr;
     size_t stage_grads_elems = 0, stage_msg_elems = 0, stage_out_elems = 0;
     cudaStream_t copy_stream = nullptr;
+    cudaStream_t aux_stream = nullptr;   // short top-k segments run here, beside the large ones
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaEvent_t ev_start = nullptr;
     std::vector<cudaEvent_t> ev_worker;
 };
@@ -219,6 +221,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             uint64_t m = (uint64_t)std::max(balance, capacity);
             m = std::min<uint64_t>(std::min<uint64_t>(m, g.n / 16), SAMPLE_MAX);
             m = std::max<uint64_t>(m, SAMPLE_MIN) & ~7ull;
+            if (seg_tiles >= FINISH_SOLO_TILES) m = std::max<uint64_t>(m, BRACKET_BIG_SAMPLE);   // a long segment: clusters throughout
             e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
             e.sample_begin = smp; smp += m;
             fast_list.push_back((uint32_t)s);
@@ -270,16 +273,21 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     // The fast list starts with the segments whose sample is large enough for a cluster of CTAs to pay
     // (the bracket kernel takes them eight CTAs at a time, the rest one CTA each); the position in the
     // list is the segment's fast index, and the sample keys are stored in list order.
-    std::stable_sort(fast_list.begin(), fast_list.end(), [&](uint32_t a, uint32_t b) {
-        return (h[a].sample_m >= BRACKET_BIG_SAMPLE) > (h[b].sample_m >= BRACKET_BIG_SAMPLE);
-    });
-    uint32_t big_count = 0;
+    // Before them come the long segments (which always have such a sample): the finish kernel takes those a
+    // cluster at a time.
+    auto rank_of = [&](uint32_t a) {
+        const uint64_t t = ((uint64_t)h[a].n + 31 + TILE - 1) / TILE;
+        return t >= FINISH_SOLO_TILES ? 2 : h[a].sample_m >= BRACKET_BIG_SAMPLE ? 1 : 0;
+    };
+    std::stable_sort(fast_list.begin(), fast_list.end(), [&](uint32_t a, uint32_t b) { return rank_of(a) > rank_of(b); });
+    uint32_t big_count = 0, huge_count = 0;
     smp = 0;
     for (size_t i = 0; i < fast_list.size(); ++i) {
         SegEntry& e = h[fast_list[i]];
         e.fast_index = (uint32_t)i;
         e.sample_begin = smp; smp += e.sample_m;
         if (e.sample_m >= BRACKET_BIG_SAMPLE) ++big_count;
+        if (rank_of(fast_list[i]) == 2) ++huge_count;
     }
     if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
     if (fast_count > c->max_fast_per_worker) return SC_ERR_RANGE;
@@ -319,7 +327,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     L.cand_per_worker = cand; L.flag_per_worker = flag; L.sample_per_worker = smp; L.fast_per_worker = fast_count;
     c->layout = L;
     c->main_wide = main_wide; c->max_main_grid = max_main_grid;
-    c->fast_big = big_count; c->max_sample_m = max_m;
+    c->fast_big = big_count; c->fast_huge = huge_count; c->max_sample_m = max_m;
     c->cached_segs.assign(segs, segs + nseg);
     c->cached_n = n;
     c->layout_valid = true;
@@ -392,10 +400,21 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
         SC_CUDA(cudaMemsetAsync(c->d_zero, 0, 64 + state_bytes + (size_t)PF * CAND_BINS * sizeof(uint32_t), stream));
         c->d_fstate = fstate;
         c->last_topk_problems = P;
+        bool forked = false;
         if (c->tiny_small || c->tiny_large) {                          // short segments: one CTA each, in shared memory
             TinyParams tp{};
             tp.L = L; tp.grads = grads; tp.residuals = residuals; tp.out_vals = out_vals; tp.out_idx = out_idx;
             tp.state = fstate; tp.W = (uint32_t)W; tp.status = c->d_status;
+            // They touch other segments than the one-pass path below (which is mostly waiting for memory in its
+            // small kernels): when the table has both kinds, the short ones run beside it on a stream of their own.
+            cudaStream_t main_stream = stream;
+            if (L.fast_per_worker && c->aux_stream) {
+                SC_CUDA(cudaEventRecord(c->ev_fork, main_stream));
+                SC_CUDA(cudaStreamWaitEvent(c->aux_stream, c->ev_fork, 0));
+                stream = c->aux_stream;
+                forked = true;
+            }
+            {
             Launch l(c, KIND_TINY, stream);
             if (c->tiny_small) {
                 tp.list = c->d_tiny_list; tp.count = c->tiny_small;
@@ -414,6 +433,9 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
                 cfg.attrs = &attr; cfg.numAttrs = 1;
                 SC_CUDA(cudaLaunchKernelEx(&cfg, topk_tiny_kernel<TINY_CTAS>, tp));
             }
+            }
+            if (forked) SC_CUDA(cudaEventRecord(c->ev_join, stream));
+            stream = main_stream;
         }
         if (L.fast_per_worker) {
             FastParams fp{};
@@ -444,14 +466,18 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               const uint32_t grid = persistent_grid(c, c->occ_filter, batches);
               const uint32_t per_cta = (uint32_t)((batches + grid - 1) / grid) * FILTER_TILES_PER_CTA;
               topk_filter_kernel<<<grid, THREADS, 0, stream>>>(fp, per_cta); }
-            { Launch l(c, KIND_FINISH, stream);                        // one cluster per large (worker, segment)
-              cudaLaunchConfig_t cfg = {};
-              cfg.gridDim = dim3(PF * FINISH_CTAS); cfg.blockDim = dim3(THREADS); cfg.stream = stream;
-              cudaLaunchAttribute attr;
-              attr.id = cudaLaunchAttributeClusterDimension;
-              attr.val.clusterDim.x = FINISH_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-              cfg.attrs = &attr; cfg.numAttrs = 1;
-              SC_CUDA(cudaLaunchKernelEx(&cfg, topk_finish_kernel, fp)); }
+            { Launch l(c, KIND_FINISH, stream);
+              const uint32_t huge = c->fast_huge, rest = L.fast_per_worker - huge;
+              if (huge) {                                              // one cluster per long (worker, segment)
+                  cudaLaunchConfig_t cfg = {};
+                  cfg.gridDim = dim3(huge * (uint32_t)W * FINISH_CTAS); cfg.blockDim = dim3(THREADS); cfg.stream = stream;
+                  cudaLaunchAttribute attr;
+                  attr.id = cudaLaunchAttributeClusterDimension;
+                  attr.val.clusterDim.x = FINISH_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+                  cfg.attrs = &attr; cfg.numAttrs = 1;
+                  SC_CUDA(cudaLaunchKernelEx(&cfg, topk_finish_kernel<FINISH_CTAS>, fp, 0u, huge));
+              }
+              if (rest) topk_finish_kernel<1><<<rest * (uint32_t)W, THREADS, 0, stream>>>(fp, huge, rest); }
             { Launch l(c, KIND_EMIT, stream);
               // flagged entries per tile, on average (the list holds the kept elements and a few per cent more)
               const double per_tile = 1.05 * (double)L.K_total * TILE / (double)std::max<size_t>(L.n_total, 1);
@@ -483,6 +509,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               const uint32_t grid = (uint32_t)c->sm_count * (uint32_t)std::max(c->occ_fallback, 1);
               SC_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(topk_fallback_kernel), dim3(grid), dim3(THREADS), args, 0, stream)); }
         }
+        if (forked) SC_CUDA(cudaStreamWaitEvent(stream, c->ev_join, 0));
         SC_CUDA(cudaGetLastError());
         return SC_OK;
     }
@@ -741,6 +768,10 @@ int sc_create(sc_ctx** out, size_t max_n, int max_W, int max_segments) {
         c->main_grid_v[1] = (size_t)c->sm_count * (size_t)std::max(c->occ_main_wide, 1);
         c->max_main_grid = c->main_grid_v[0];
     }
+    if (rc == SC_OK && (cudaStreamCreateWithFlags(&c->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
+        rc = SC_ERR_CUDA;
     if (rc != SC_OK) { sc_destroy(c); return rc; }
     *out = c;
     return SC_OK;
@@ -760,6 +791,9 @@ void sc_destroy(sc_ctx* c) {
     for (cudaEvent_t e : c->prof_free) cudaEventDestroy(e);
     if (c->ev_start) cudaEventDestroy(c->ev_start);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->aux_stream) cudaStreamDestroy(c->aux_stream);
     delete c;
 }
 

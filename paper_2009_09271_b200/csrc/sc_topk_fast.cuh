@@ -841,7 +841,9 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
 }
 
 // ---- finish: exact threshold, per-tile kept counts, message offsets ----------------------------
-// One thread-block cluster per large (worker, segment).
+// One thread-block cluster per (worker, segment) of FINISH_SOLO_TILES tiles and more (C = FINISH_CTAS),
+// one CTA for the others (C = 1: no cluster calls at all); `first` and `count` select a range of the fast
+// list, the grid covers count problems of every worker.
 //   threshold among the candidates: CTA 0 sorts the short list (the candidates of the threshold's
 //       histogram bin, at most LIST2_CAP) in shared memory, larger key first and lower coordinate first
 //       among equal keys; its first need2 entries are kept, which fixes T and the coordinate cut, and each
@@ -854,30 +856,31 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
 // The cluster barriers are the hardware's; every CTA runs to the last one.
 constexpr uint32_t FINISH_CTAS = 8;
 constexpr uint32_t FINISH_PER = 16;                                    // tiles per thread and round of a scan
-constexpr uint32_t FINISH_SOLO_TILES = 4096;                           // below this many tiles CTA 0 serves the segment alone
+constexpr uint32_t FINISH_SOLO_TILES = 4096;                           // segments below this many tiles are served by one CTA
 __device__ inline uint32_t block_sum(uint32_t v, uint32_t* s_scan) {
     uint32_t total;
     block_exclusive_scan(v, s_scan, &total);
     return total;
 }
+template <uint32_t C>
 __global__ void __launch_bounds__(THREADS)
-topk_finish_kernel(const __grid_constant__ FastParams P) {
+topk_finish_kernel(const __grid_constant__ FastParams P, uint32_t first, uint32_t count) {
     namespace cg = cooperative_groups;
     __shared__ unsigned long long srt[LIST2_CAP];
     __shared__ uint32_t s_scan[WARPS + 1];
     __shared__ uint32_t s_share[3];                                    // ties and kept elements of this CTA's share; [2]: CTA 0 gave up
     cg::cluster_group cluster = cg::this_cluster();
-    const uint32_t rank = cluster.block_rank();
+    constexpr bool solo = C == 1;
+    constexpr uint32_t ranks = C;
+    const uint32_t rank = solo ? 0u : cluster.block_rank();
     const Layout& L = P.L;
     uint32_t w, s;
-    const uint32_t prob = fast_problem(L, blockIdx.x / FINISH_CTAS, w, s);
+    const uint32_t pidx = blockIdx.x / C;                              // problem of this launch: (worker, position in the range)
+    const uint32_t prob = fast_problem(L, (pidx / count) * L.fast_per_worker + first + pidx % count, w, s);
     const SegEntry seg = L.segs[s];
     FastState st = P.state[prob];
     if (st.path != PATH_FAST) return;                                  // the same answer in every CTA of the cluster
     const uint32_t ntiles = L.segs[s + 1].tile_begin - seg.tile_begin;
-    const bool solo = ntiles < FINISH_SOLO_TILES;                      // no cluster barrier at all then
-    if (solo && rank != 0) return;
-    const uint32_t ranks = solo ? 1u : FINISH_CTAS;
     const size_t item0 = (size_t)w * L.tiles_per_worker + seg.tile_begin;
     const bool admit = st.need_ties != 0u;
     if (rank == 0) {
