@@ -64,30 +64,13 @@ agg_tiles_kernel(const float* __restrict__ vals, const uint32_t* __restrict__ id
         if (shared_idx) {
             const uint32_t lo = bounds[t], hi = bounds[t + 1];
             __syncthreads();
-            // four slots per thread at a time: a tile inside a kept block holds thousands of slots, and one
-            // memory latency per slot and thread would dominate the launch
-            for (uint32_t j0 = lo + threadIdx.x; j0 < hi; j0 += 4 * THREADS) {
-                uint32_t loc[4];
-                float sum[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint32_t j = j0 + u * THREADS;
-                    loc[u] = j < hi ? __ldg(idx + j) - tile_lo : 0xFFFFFFFFu;
-                    sum[u] = 0.0f;
-                }
-                for (uint32_t w = 0; w < W; ++w) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const uint32_t j = j0 + u * THREADS;
-                        if (j < hi) sum[u] = sum[u] + __ldg(vals + (size_t)w * K + j);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (j0 + u * THREADS >= hi) continue;
-                    if (loc[u] < tile_n) acc[loc[u]] = sum[u];
-                    else atomicMin(status, ST_DEVICE_CHECK);
-                }
+            for (uint32_t j = lo + threadIdx.x; j < hi; j += THREADS) {
+                const uint32_t loc = idx[j] - tile_lo;
+                float sum = 0.0f;
+#pragma unroll 8
+                for (uint32_t w = 0; w < W; ++w) sum = sum + vals[(size_t)w * K + j];
+                if (loc < tile_n) acc[loc] = sum;
+                else atomicMin(status, ST_DEVICE_CHECK);
             }
             __syncthreads();
         } else {
