@@ -3,7 +3,9 @@
 // select on p = gamma g + e, which the streaming pass has parked in the residual buffer.
 //
 // ONE persistent kernel per top-k call, launched cooperatively (all its CTAs are resident), which
-// returns in its first instructions unless some segment failed.  Its phases are separated by
+// returns in its first instructions unless some segment failed.  (It also hosts the rare second half
+// of the emit step, the tiles that admit tie-key elements, so that the emit kernel proper keeps its
+// registers for the common case.)  Its phases are separated by
 // grid-wide barriers:
 //   A  put back the values the streaming pass had zeroed, clear the failed segments' histograms
 //   B  histogram of key bits 30..20         C  bucket of the k-th key
@@ -55,6 +57,7 @@ __device__ inline bool grid_barrier(unsigned int* counter, unsigned int& target,
 
 __global__ void __launch_bounds__(THREADS)
 topk_fallback_kernel(const __grid_constant__ FallbackParams P) {
+    if (__ldcg(P.F.counters + 1) != 0u) emit_tie_tiles(P.F);          // some segment's threshold is its tie key
     if (__ldcg(P.F.counters) == 0u) return;                            // no segment failed: the usual case
     const Layout& L = P.F.L;
     const uint32_t nprob = P.W * L.nseg;

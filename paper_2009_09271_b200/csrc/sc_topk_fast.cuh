@@ -1046,8 +1046,7 @@ topk_finish_kernel(const __grid_constant__ FastParams P, uint32_t first, uint32_
 // side by side; long slices take the whole warp and more entries per lane.  One batch covers
 // G x D entries.  (Loading the placement words two tiles ahead and asking L2 for the next slice
 // one tile ahead changed nothing: the kernel is not bound by its chain of dependent loads.)
-// Tiles that admit tie-key elements are skipped here and served by a second loop, in which a whole
-// warp re-reads the tile from the residual (it still holds p there) in coordinate order.
+// Tiles that admit tie-key elements are skipped here (see emit_tie_tiles).
 template <int G, int D>
 __global__ void __launch_bounds__(THREADS)
 topk_emit_kernel(FastParams P) {
@@ -1128,58 +1127,101 @@ topk_emit_kernel(FastParams P) {
             }
         }
     }
-    // ---- tiles that admit tie-key elements (none at all unless some segment's threshold is its tie key) ------
-    if (__ldg(P.counters + 1) == 0u) return;
+}
+
+// ---- tiles that admit tie-key elements ----------------------------------------------------------
+// Run by every CTA of the kernel that follows the emit step (sc_topk_fallback.cuh), and only when some
+// segment's threshold is its tie key.  One warp per tile re-reads the tile from the residual (which
+// still holds p there) in coordinate order: everything above the tie key is kept, and the first `adm`
+// tie-key elements of the tile, as the finish step decided.
+__device__ inline void emit_tie_tiles(const FastParams& P) {
+    const Layout& L = P.L;
+    const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warps_total = gridDim.x * WARPS;
-    for (uint32_t it = blockIdx.x * WARPS + (threadIdx.x >> 5); it < P.total_items; it += warps_total) {
-        const uint32_t w = it / L.tiles_per_worker;
-        const uint32_t lt = it - w * L.tiles_per_worker;
-        const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
-        const SegEntry& seg = L.segs[s];
-        if (!seg.fast) continue;
-        const FastState* st = P.state + (size_t)w * L.nseg + s;
-        if (st->path != PATH_FAST || st->need_ties == 0u) continue;
-        const uint32_t adm = P.tile_csum[it];
-        if (adm == 0u) continue;
-        const uint32_t tkey = st->T;                                    // == tie key
-        float* er = P.residuals + (size_t)w * L.n_total + seg.offset;
-        float* ov = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
-        uint32_t* oi = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
-        const long long first = (long long)(lt - seg.tile_begin) * TILE - misalign_of(er);
-        uint32_t pos = P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt];
-        uint32_t ties_seen = 0;
-        for (uint32_t r = 0; r < TILE / 128; ++r) {                     // 128 coordinates per step, a quad per lane
-            const long long qb = first + 128 * r + 4 * lane;
-            float p[4];
-            const uint32_t valid = load_quad(er, qb, seg.n, p);
-            uint32_t above = 0, tie = 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t key = key_of(p[c]), v = (valid >> c) & 1u;
-                above |= (v & (uint32_t)(key > tkey)) << c;
-                tie |= (v & (uint32_t)(key == tkey)) << c;
+    const uint32_t warp_g = blockIdx.x * WARPS + (threadIdx.x >> 5);
+    for (uint32_t it0 = warp_g; it0 < P.total_items; it0 += warps_total * 32u) {
+        // every lane looks at one tile (neighbouring tiles, which tend to admit ties together, go to different
+        // warps); the warp then serves, one after the other, those that admit ties
+        uint32_t my_adm = 0, my_s = 0;
+        {
+            const unsigned long long it64 = (unsigned long long)it0 + (unsigned long long)lane * warps_total;
+            const uint32_t it = it64 < P.total_items ? (uint32_t)it64 : 0xFFFFFFFFu;
+            if (it != 0xFFFFFFFFu) {
+                const uint32_t w = it / L.tiles_per_worker;
+                const uint32_t lt = it - w * L.tiles_per_worker;
+                my_s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+                if (L.segs[my_s].fast) {
+                    const FastState* st = P.state + (size_t)w * L.nseg + my_s;
+                    if (st->path == PATH_FAST && st->need_ties != 0u) my_adm = P.tile_csum[it];
+                }
             }
-            const uint32_t tinc = warp_inclusive_scan(__popc(tie), lane);
-            uint32_t trank = ties_seen + tinc - __popc(tie);            // tie-key elements of the tile before this quad
-            uint32_t keep = above;
+        }
+        uint32_t todo = __ballot_sync(0xFFFFFFFFu, my_adm != 0u);
+        while (todo) {
+            const uint32_t src = (uint32_t)__ffs((int)todo) - 1u;
+            todo &= todo - 1u;
+            const uint32_t it = it0 + src * warps_total;
+            const uint32_t adm = __shfl_sync(0xFFFFFFFFu, my_adm, src), s = __shfl_sync(0xFFFFFFFFu, my_s, src);
+            const uint32_t w = it / L.tiles_per_worker;
+            const uint32_t lt = it - w * L.tiles_per_worker;
+            const SegEntry& seg = L.segs[s];
+            const uint32_t tkey = P.state[(size_t)w * L.nseg + s].T;   // == tie key
+            float* er = P.residuals + (size_t)w * L.n_total + seg.offset;
+            float* ov = P.out_vals + (size_t)w * L.K_total + seg.msg_off;
+            uint32_t* oi = P.out_idx + (size_t)w * L.K_total + seg.msg_off;
+            const long long first = (long long)(lt - seg.tile_begin) * TILE - misalign_of(er);
+            const bool full = first >= 0 && first + TILE <= (long long)seg.n;
+            uint32_t pos = P.offsets[(size_t)w * (L.tiles_per_worker + 1) + lt];
+            uint32_t ties_seen = 0;
+            for (uint32_t r0 = 0; r0 < TILE / 128; r0 += 8) {           // 128 coordinates per step, a quad per lane; eight steps' loads together
+                float pb[8][4];
+                uint32_t vb[8];
+                if (full) {                                               // uniform: eight independent 128-bit loads
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if ((tie >> c) & 1u) { if (trank < adm) keep |= 1u << c; ++trank; }
-            ties_seen += __shfl_sync(0xFFFFFFFFu, tinc, 31);
-            const uint32_t kinc = warp_inclusive_scan(__popc(keep), lane);
-            uint32_t slot = pos + kinc - __popc(keep);
-            pos += __shfl_sync(0xFFFFFFFFu, kinc, 31);
-            if (keep) {
+                    for (uint32_t u = 0; u < 8; ++u) {
+                        const float4 q = *reinterpret_cast<const float4*>(er + first + 128 * (r0 + u) + 4 * lane);
+                        pb[u][0] = q.x; pb[u][1] = q.y; pb[u][2] = q.z; pb[u][3] = q.w;
+                        vb[u] = 0xFu;
+                    }
+                } else {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if ((keep >> c) & 1u) {
-                        if (slot < seg.k) { ov[slot] = p[c]; oi[slot] = (uint32_t)seg.offset + (uint32_t)(qb + c); }
-                        else atomicMin(P.status, ST_DEVICE_CHECK);
-                        ++slot;
-                        p[c] = 0.0f;
+                    for (uint32_t u = 0; u < 8; ++u) vb[u] = load_quad(er, first + 128 * (r0 + u) + 4 * lane, seg.n, pb[u]);
+                }
+#pragma unroll
+                for (uint32_t u = 0; u < 8; ++u) {
+                    const long long qb = first + 128 * (r0 + u) + 4 * lane;
+                    float* p = pb[u];
+                    const uint32_t valid = vb[u];
+                    uint32_t above = 0, tie = 0;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t key = key_of(p[c]), v = (valid >> c) & 1u;
+                        above |= (v & (uint32_t)(key > tkey)) << c;
+                        tie |= (v & (uint32_t)(key == tkey)) << c;
+                    }
+                    const uint32_t tinc = warp_inclusive_scan(__popc(tie), lane);
+                    uint32_t trank = ties_seen + tinc - __popc(tie);    // tie-key elements of the tile before this quad
+                    uint32_t keep = above;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if ((tie >> c) & 1u) { if (trank < adm) keep |= 1u << c; ++trank; }
+                    ties_seen += __shfl_sync(0xFFFFFFFFu, tinc, 31);
+                    const uint32_t kinc = warp_inclusive_scan(__popc(keep), lane);
+                    uint32_t slot = pos + kinc - __popc(keep);
+                    pos += __shfl_sync(0xFFFFFFFFu, kinc, 31);
+                    if (keep) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            if ((keep >> c) & 1u) {
+                                if (slot < seg.k) { ov[slot] = p[c]; oi[slot] = (uint32_t)seg.offset + (uint32_t)(qb + c); }
+                                else atomicMin(P.status, ST_DEVICE_CHECK);
+                                ++slot;
+                                p[c] = 0.0f;
+                            }
+                        }
+                        store_quad(er, qb, valid, p);
                     }
                 }
-                store_quad(er, qb, valid, p);
             }
         }
     }
