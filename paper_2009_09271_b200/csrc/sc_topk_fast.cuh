@@ -317,13 +317,15 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
 // Exact counts decide whether the bracket held: count(key > hi) <= k <= count(key >= lo) + ties.
 // Then either the k-th key lies among the candidates (its histogram bin is pinned here, the exact
 // key by the finish step), or every candidate is kept and the rest are tie-key elements.
-// Called by all threads of a CTA after the streaming pass has ended (all counts are final).  Every
-// CTA that needs a segment's bin works it out for itself (a walk over 2048 words); `owner` (the CTA
-// that holds the segment's first tile) also records it in the segment's state.
+// Called after the streaming pass has ended (all counts are final).  Every CTA that needs a segment's
+// bin works it out for itself (a walk over 2048 words); `owner` (the CTA that holds the segment's
+// first tile) also records it in the segment's state.
 struct BinInfo { uint32_t live, need2, lo2, hi2; };                   // live: the segment is still on the one-pass path
+// Run by ONE WARP (the warps of a CTA take different segments): lane l adds up 64 bins, a warp scan
+// finds the lane whose bins hold the k-th key, and that lane walks its 64 bins.
 __device__ __noinline__ BinInfo resolve_bin(const FastParams& P, uint32_t prob, bool owner) {
-    __shared__ uint32_t s_tmp[WARPS + 4];
     const Layout& L = P.L;
+    const uint32_t lane = threadIdx.x & 31u;
     const uint32_t w = prob / L.nseg, s = prob - w * L.nseg;
     const SegEntry& seg = L.segs[s];
     FastState st = P.state[prob];
@@ -339,10 +341,38 @@ __device__ __noinline__ BinInfo resolve_bin(const FastParams& P, uint32_t prob, 
     uint32_t bin = 0, need_in = 0, cnt = 0;
     const uint32_t need = fail ? 0u : seg.k - st.sure_total;
     const bool among_candidates = need != 0u && need <= st.cand_total;
-    if (!fail && among_candidates) {
-        const bool found = find_from_top<CAND_BINS>(P.cand_hist + fidx * CAND_BINS, need, s_tmp, bin, need_in, cnt);
-        if (!found) fail = FAIL_BRACKET;
-        else if (cnt > LIST2_CAP) fail = FAIL_SHORT_LIST;
+    if (!fail && among_candidates) {                                   // uniform over the warp
+        static_assert(CAND_BINS == 64 * 32, "64 bins per lane");
+        const uint32_t* mine = P.cand_hist + fidx * CAND_BINS + (CAND_BINS - 64u * (lane + 1u));   // lane 0 owns the top 64 bins
+        uint32_t sum = 0;
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {                                 // (four loads in flight: the filter below wants the registers)
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(mine) + i);
+            sum += v.x + v.y + v.z + v.w;
+        }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+            if (lane >= (uint32_t)d) inc += t;
+        }
+        const uint32_t before = inc - sum;
+        const bool here = before < need && need <= inc;                // at most one lane
+        if (here) {
+            uint32_t acc = before;
+            for (int b = 63; b >= 0; --b) {
+                const uint32_t c = __ldg(mine + b);
+                if (need <= acc + c) { bin = CAND_BINS - 64u * (lane + 1u) + (uint32_t)b; need_in = need - acc; cnt = c; break; }
+                acc += c;
+            }
+        }
+        const uint32_t who = __ballot_sync(0xFFFFFFFFu, here);
+        if (who == 0u) fail = FAIL_BRACKET;
+        else {
+            const int src = __ffs((int)who) - 1;
+            bin = __shfl_sync(0xFFFFFFFFu, bin, src); need_in = __shfl_sync(0xFFFFFFFFu, need_in, src); cnt = __shfl_sync(0xFFFFFFFFu, cnt, src);
+            if (cnt > LIST2_CAP) fail = FAIL_SHORT_LIST;
+        }
     }
     st.need2 = 0; st.need_ties = 0; st.cnt2 = 0; st.expect2 = 0; st.icut = 0;
     if (fail) {
@@ -359,7 +389,7 @@ __device__ __noinline__ BinInfo resolve_bin(const FastParams& P, uint32_t prob, 
         st.T = st.tie_key;
         st.need_ties = need - st.cand_total;
     }
-    if (owner && threadIdx.x == 0) {
+    if (owner && lane == 0) {
         if (fail) atomicAdd(P.counters, 1u);
         else if (st.need_ties) atomicAdd(P.counters + 1, 1u);
         // only result words are written: other CTAs may be reading the counts above, or adding to the
@@ -758,13 +788,13 @@ topk_filter_kernel(const __grid_constant__ FastParams P, uint32_t items_per_cta)
         __syncthreads();
         const uint32_t p_first = s_range[0], part_end = s_range[1];
         const uint32_t p_last = problem_of_item(L, part_end - 1u);
-        for (uint32_t p = p_first; p <= p_last; ++p) {                // uniform over the CTA
+        for (uint32_t p = p_first + (threadIdx.x >> 5); p <= p_last; p += WARPS) {   // one warp per segment
             const uint32_t w = p / L.nseg, s = p - w * L.nseg;
             if (!L.segs[s].fast) continue;
             // the CTA whose range holds the segment's first tile records the result
             const uint32_t first_item = w * L.tiles_per_worker + L.segs[s].tile_begin;
             const BinInfo bi = resolve_bin(P, p, first_item >= pos && first_item < part_end);
-            if (threadIdx.x == 0) s_bin[p - p_first] = bi;
+            if ((threadIdx.x & 31u) == 0u) s_bin[p - p_first] = bi;
         }
         __syncthreads();
         // (the loop bound is the same for all lanes of a warp: its shuffles stay whole)
@@ -780,6 +810,7 @@ topk_filter_kernel(const __grid_constant__ FastParams P, uint32_t items_per_cta)
             const uint2* list[TILES_PER_GROUP];
             uint2 first[TILES_PER_GROUP];
             uint32_t prob[TILES_PER_GROUP];
+            uint32_t s_prev = 0xFFFFFFFFu, w_prev = 0xFFFFFFFFu, end_prev = 0;   // consecutive tiles mostly share their segment
 #pragma unroll
             for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
                 const uint32_t item = item0 + u;
@@ -787,7 +818,11 @@ topk_filter_kernel(const __grid_constant__ FastParams P, uint32_t items_per_cta)
                 if (item >= part_end) continue;
                 const uint32_t w = item / L.tiles_per_worker;
                 const uint32_t lt = item - w * L.tiles_per_worker;
-                const uint32_t s = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+                if (w != w_prev || lt >= end_prev) {
+                    s_prev = (L.nseg == 1) ? 0u : find_by_tile(L, lt);
+                    w_prev = w; end_prev = L.segs[s_prev + 1].tile_begin;
+                }
+                const uint32_t s = s_prev;
                 const SegEntry& seg = L.segs[s];
                 prob[u] = w * L.nseg + s;
                 if (!seg.fast) continue;
