@@ -605,3 +605,31 @@ def test_step_apply_matches_step_then_update(ctx, scheme):
             assert_bits_equal(e[w], oe[w], f"residual[w={w}]")
             assert_bits_equal(idx[w], oi[w], f"idx[w={w}]")
         assert_bits_equal(x, O.aggregate_apply(x0.numpy(), ov, oi), "model")
+
+
+def test_user_stream_short_and_long_segments_side_by_side(ctx):
+    """On a stream of the caller's, with short segments (served on a stream of the library's own, forked from
+    and joined to the caller's) next to long ones: the result is complete when the caller's stream is."""
+    sizes = [3000, BIG + 9, 50_000, 200, 131_072, 17]
+    segs = [(s.offset, s.n, s.k) for s in wl.segment_table(sizes, 1, 64)]
+    n, K, W = sum(sizes), sum(s[2] for s in segs), 3
+    g = torch.stack([rand(n, 1700 + w) for w in range(W)])
+    e0 = torch.stack([rand(n, 1710 + w, scale=1e-4) for w in range(W)])
+    ov, oi, oe, oout = O.step(sc.SC_TOPK, [g[w].numpy() for w in range(W)], [e0[w].numpy() for w in range(W)], segs, [0] * W)
+    stream = torch.cuda.Stream()
+    gd = g.cuda()
+    for _ in range(3):                                                   # back to back: scratch reuse across calls in stream order
+        e = e0.cuda().clone()
+        vals = torch.full((W, K), float("nan"), device="cuda"); idx = torch.full((W, K), -1, device="cuda", dtype=torch.int32)
+        out = torch.full((n,), float("nan"), device="cuda")
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            ctx.sc_step(sc.SC_TOPK, gd, e, segs, [0] * W, vals, idx, out, stream=stream)
+            ctx.sc_step(sc.SC_TOPK, gd, e.clone(), segs, [0] * W, vals.clone(), idx.clone(), out.clone(), stream=stream)
+        stream.synchronize()
+        for w in range(W):
+            assert_bits_equal(idx[w], oi[w], f"idx[w={w}]")
+            assert_bits_equal(vals[w], ov[w], f"vals[w={w}]")
+            assert_bits_equal(e[w], oe[w], f"residual[w={w}]")
+        assert_bits_equal(out, oout, "aggregate")
+    assert ctx.sc_sync_status(stream) == 0
