@@ -137,11 +137,11 @@ class DeviceGuard {
 };
 
 enum { KIND_SCATTER = 0, KIND_MASK_COUNT, KIND_ROW_SCAN, KIND_RANDK_PACK, KIND_RANDBLOCK, KIND_AGG_BOUNDS, KIND_AGG_TILES,
-       KIND_AGG_WARP, KIND_AGG_FINE, KIND_AGG_APPLY, KIND_TINY, KIND_BRACKET, KIND_MAIN, KIND_FILTER, KIND_FINISH, KIND_EMIT,
+       KIND_AGG_WARP, KIND_AGG_FINE, KIND_AGG_APPLY, KIND_TINY, KIND_BRACKET, KIND_MAIN, KIND_FILTER, KIND_FINISH, KIND_RESOLVE_SMALL, KIND_EMIT,
        KIND_FALLBACK, KIND_COUNT };
 const char* const kKindNames[KIND_COUNT] = {"randk_scatter", "mask_count", "row_scan", "randk_pack", "randblock", "agg_bounds",
                                             "agg_tiles", "agg_warp", "agg_fine", "agg_apply", "topk_tiny", "topk_bracket",
-                                            "topk_main", "topk_filter", "topk_finish", "topk_emit", "topk_fallback"};
+                                            "topk_main", "topk_filter", "topk_finish", "topk_resolve_small", "topk_emit", "topk_fallback"};
 
 // Counts a kernel launch and, when profiling is on, brackets it with two events.
 class Launch {
@@ -221,8 +221,12 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             uint64_t m = (uint64_t)std::max(balance, capacity);
             m = std::min<uint64_t>(std::min<uint64_t>(m, g.n / 16), SAMPLE_MAX);
             m = std::max<uint64_t>(m, SAMPLE_MIN) & ~7ull;
-            if (seg_tiles >= FINISH_SOLO_TILES) m = std::max<uint64_t>(m, BRACKET_BIG_SAMPLE);   // a long segment: clusters throughout
-            e.fast = 1; e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
+            // Segments of few tiles whose bracket leaves few candidates are resolved by one CTA each
+            // (topk_resolve_small_kernel); the others go through the filter and finish kernels (see below).
+            const double candidates = 12.0 * std::sqrt(q * (1.0 - q) / (double)m) * (double)g.n;
+            const bool small = seg_tiles <= SMALL_MAX_TILES && candidates <= 16384.0;
+            e.fast = small ? 2u : 1u;
+            e.sample_m = (uint32_t)m; e.fast_index = fast_count++;
             e.sample_begin = smp; smp += m;
             fast_list.push_back((uint32_t)s);
             // The main pass appends to private regions of the segment's flagged and candidate lists:
@@ -234,7 +238,9 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
             const uint64_t regions = per_tile ? seg_tiles : max_main_grid;
             // (a CTA takes groups of MAIN_GROUP consecutive tiles, every regions-th group: the segment overlaps at
             // most seg_tiles / MAIN_GROUP + 2 groups)
-            const uint64_t tiles_per_region = per_tile ? 1 : MAIN_GROUP * ((seg_tiles / MAIN_GROUP + 2 + regions - 1) / regions);
+            uint64_t tiles_per_region = 1;                             // (the pass may take smaller groups when the call has few tiles)
+            for (uint64_t gsz = 1; !per_tile && gsz <= MAIN_GROUP; gsz *= 2)
+                tiles_per_region = std::max(tiles_per_region, gsz * ((seg_tiles / gsz + 2 + regions - 1) / regions));
             const uint64_t cand_region = tiles_per_region * ((slack + seg_tiles - 1) / seg_tiles + 16);
             const uint64_t flag_region = tiles_per_region * ((g.k + slack + seg_tiles - 1) / seg_tiles + 16);
             // Behind the regions lies a pool from which a full region continues (elements above the bracket
@@ -273,12 +279,17 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
     // The fast list starts with the segments whose sample is large enough for a cluster of CTAs to pay
     // (the bracket kernel takes them eight CTAs at a time, the rest one CTA each); the position in the
     // list is the segment's fast index, and the sample keys are stored in list order.
-    // Before them come the long segments (which always have such a sample): the finish kernel takes those a
-    // cluster at a time.
-    auto rank_of = [&](uint32_t a) {
-        const uint64_t t = ((uint64_t)h[a].n + 31 + TILE - 1) / TILE;
-        return t >= FINISH_SOLO_TILES ? 2 : h[a].sample_m >= BRACKET_BIG_SAMPLE ? 1 : 0;
-    };
+    // Before them come the segments that the filter and finish kernels serve (they take the cluster form of the
+    // bracket kernel whatever their sample); the others are resolved by one CTA each.
+    // A table that needs the filter and finish kernels anyway lets a handful of small segments ride along with
+    // them instead of paying for a launch of their own.
+    {
+        uint32_t n_large = 0, n_small = 0;
+        for (uint32_t a : fast_list) (h[a].fast == 1u ? n_large : n_small) += 1u;
+        if (n_large && n_small < 8u)
+            for (uint32_t a : fast_list) h[a].fast = 1u;
+    }
+    auto rank_of = [&](uint32_t a) { return h[a].fast == 1u ? 2 : h[a].sample_m >= BRACKET_BIG_SAMPLE ? 1 : 0; };
     std::stable_sort(fast_list.begin(), fast_list.end(), [&](uint32_t a, uint32_t b) { return rank_of(a) > rank_of(b); });
     uint32_t big_count = 0, huge_count = 0;
     smp = 0;
@@ -286,7 +297,7 @@ int prepare_layout(sc_ctx* c, size_t n, const sc_segment* segs, int nseg, cudaSt
         SegEntry& e = h[fast_list[i]];
         e.fast_index = (uint32_t)i;
         e.sample_begin = smp; smp += e.sample_m;
-        if (e.sample_m >= BRACKET_BIG_SAMPLE) ++big_count;
+        if (rank_of(fast_list[i]) >= 1) ++big_count;               // the cluster form of the bracket kernel serves these
         if (rank_of(fast_list[i]) == 2) ++huge_count;
     }
     if (tiles > c->max_tiles_per_worker || maskw > c->max_mask_words || tiles > 0xFFFFFFFFull) return SC_ERR_RANGE;
@@ -458,26 +469,34 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
               }
               if (small) topk_bracket_kernel<1><<<small * (uint32_t)W, THREADS, 0, stream>>>(fp, big, small); }
             { Launch l(c, KIND_MAIN, stream);
-              const uint64_t groups_of_tiles = (items + MAIN_GROUP - 1) / MAIN_GROUP;
+              // groups of 8 consecutive tiles, fewer when that would leave CTAs without work
+              const uint64_t cap = (uint64_t)c->sm_count * (uint64_t)std::max(c->main_wide ? c->occ_main_wide : c->occ_main, 1);
+              uint32_t group = MAIN_GROUP;
+              while (group > 1u && (items + group - 1) / group < 2 * cap) group /= 2;
+              fp.main_group = group;
+              const uint64_t groups_of_tiles = (items + group - 1) / group;
               if (c->main_wide) topk_main_kernel<1><<<persistent_grid(c, c->occ_main_wide, groups_of_tiles), THREADS, 0, stream>>>(fp);
               else topk_main_kernel<3><<<persistent_grid(c, c->occ_main, groups_of_tiles), THREADS, 0, stream>>>(fp); }
+            const uint32_t huge = c->fast_huge, rest = L.fast_per_worker - huge;
+            if (huge) {
             { Launch l(c, KIND_FILTER, stream);
               const uint64_t batches = (items + FILTER_TILES_PER_CTA - 1) / FILTER_TILES_PER_CTA;
               const uint32_t grid = persistent_grid(c, c->occ_filter, batches);
               const uint32_t per_cta = (uint32_t)((batches + grid - 1) / grid) * FILTER_TILES_PER_CTA;
               topk_filter_kernel<<<grid, THREADS, 0, stream>>>(fp, per_cta); }
-            { Launch l(c, KIND_FINISH, stream);
-              const uint32_t huge = c->fast_huge, rest = L.fast_per_worker - huge;
-              if (huge) {                                              // one cluster per long (worker, segment)
-                  cudaLaunchConfig_t cfg = {};
-                  cfg.gridDim = dim3(huge * (uint32_t)W * FINISH_CTAS); cfg.blockDim = dim3(THREADS); cfg.stream = stream;
-                  cudaLaunchAttribute attr;
-                  attr.id = cudaLaunchAttributeClusterDimension;
-                  attr.val.clusterDim.x = FINISH_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-                  cfg.attrs = &attr; cfg.numAttrs = 1;
-                  SC_CUDA(cudaLaunchKernelEx(&cfg, topk_finish_kernel<FINISH_CTAS>, fp, 0u, huge));
-              }
-              if (rest) topk_finish_kernel<1><<<rest * (uint32_t)W, THREADS, 0, stream>>>(fp, huge, rest); }
+            { Launch l(c, KIND_FINISH, stream);                        // one cluster per long (worker, segment)
+              cudaLaunchConfig_t cfg = {};
+              cfg.gridDim = dim3(huge * (uint32_t)W * FINISH_CTAS); cfg.blockDim = dim3(THREADS); cfg.stream = stream;
+              cudaLaunchAttribute attr;
+              attr.id = cudaLaunchAttributeClusterDimension;
+              attr.val.clusterDim.x = FINISH_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+              cfg.attrs = &attr; cfg.numAttrs = 1;
+              SC_CUDA(cudaLaunchKernelEx(&cfg, topk_finish_kernel<FINISH_CTAS>, fp, 0u, huge)); }
+            }
+            if (rest) {                                                // segments of few tiles: one CTA each does all of it
+                Launch l(c, KIND_RESOLVE_SMALL, stream);
+                topk_resolve_small_kernel<<<rest * (uint32_t)W, THREADS, 0, stream>>>(fp, huge, rest);
+            }
             { Launch l(c, KIND_EMIT, stream);
               // flagged entries per tile, on average (the list holds the kept elements and a few per cent more)
               const double per_tile = 1.05 * (double)L.K_total * TILE / (double)std::max<size_t>(L.n_total, 1);

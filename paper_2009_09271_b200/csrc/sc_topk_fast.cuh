@@ -62,6 +62,7 @@ struct FastParams {
     uint32_t* offsets;         // [W][tiles_per_worker + 1]: kept coordinates of the SEGMENT before the tile
     int* status;
     uint32_t total_items;
+    uint32_t main_group;       // consecutive tiles a CTA of the streaming pass takes at a time (<= MAIN_GROUP)
 };
 
 // The per-segment launches of this path cover the fast segments only: problem index
@@ -497,11 +498,12 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
     uint32_t pend_item = 0xFFFFFFFFu, pend_slot = 0, pend_room = 0;    // tile whose counts are not written yet
     bool pool_dry = false;
     const float gamma = L.gamma;
-    const uint32_t group_step = (gridDim.x - 1u) * MAIN_GROUP + 1u;    // from a group's last tile to the next group's first
+    const uint32_t group = P.main_group;
+    const uint32_t group_step = (gridDim.x - 1u) * group + 1u;         // from a group's last tile to the next group's first
     MainTile T{};
     uint32_t seg_tile_end = 0;                                         // first tile after T's segment
-    for (uint32_t item = blockIdx.x * MAIN_GROUP, ig = 0; ;
-         item += (ig + 1u == MAIN_GROUP ? group_step : 1u), ig = (ig + 1u == MAIN_GROUP ? 0u : ig + 1u)) {
+    for (uint32_t item = blockIdx.x * group, ig = 0; ;
+         item += (ig + 1u == group ? group_step : 1u), ig = (ig + 1u == group ? 0u : ig + 1u)) {
         // inside a group the next tile usually belongs to the same (worker, segment): then only its position
         // changes, and the lookup of the segment (a search over the table) is skipped
         if (ig != 0u && T.have && T.lt + 1u < seg_tile_end) {
@@ -607,7 +609,7 @@ topk_main_kernel(const __grid_constant__ FastParams P) {
         // the loads of this tile have landed: ask L2 for the tile this CTA takes next, so that DRAM stays busy
         // during the per-element work below (measured on 350 M x 16 at 1 %: 12.3 -> 10.85 ms)
         if (SC_PREFETCH_DIST) {
-            const uint32_t ahead = ig + 1u == MAIN_GROUP ? group_step : 1u;    // distance to this CTA's next tile
+            const uint32_t ahead = ig + 1u == group ? group_step : 1u;         // distance to this CTA's next tile
             if (T.full && T.lt + ahead + 1u < seg_tile_end) {
                 prefetch_tile_l2(T.g, e, T.first + (long long)ahead * TILE);
             } else {                                                   // the next tile lies in another segment: locate it
@@ -790,7 +792,7 @@ topk_filter_kernel(const __grid_constant__ FastParams P, uint32_t items_per_cta)
         const uint32_t p_last = problem_of_item(L, part_end - 1u);
         for (uint32_t p = p_first + (threadIdx.x >> 5); p <= p_last; p += WARPS) {   // one warp per segment
             const uint32_t w = p / L.nseg, s = p - w * L.nseg;
-            if (!L.segs[s].fast) continue;
+            if (L.segs[s].fast != 1u) continue;                       // (segments of few tiles are resolved by one CTA each)
             // the CTA whose range holds the segment's first tile records the result
             const uint32_t first_item = w * L.tiles_per_worker + L.segs[s].tile_begin;
             const BinInfo bi = resolve_bin(P, p, first_item >= pos && first_item < part_end);
@@ -825,7 +827,7 @@ topk_filter_kernel(const __grid_constant__ FastParams P, uint32_t items_per_cta)
                 const uint32_t s = s_prev;
                 const SegEntry& seg = L.segs[s];
                 prob[u] = w * L.nseg + s;
-                if (!seg.fast) continue;
+                if (seg.fast != 1u) continue;
                 const BinInfo bi = s_bin[prob[u] - p_first];
                 if (!bi.live || bi.need2 == 0u || cnt[u] == 0u) continue;  // no candidate, or every candidate, is kept
                 list[u] = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin + base[u];
@@ -876,9 +878,9 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
 }
 
 // ---- finish: exact threshold, per-tile kept counts, message offsets ----------------------------
-// One thread-block cluster per (worker, segment) of FINISH_SOLO_TILES tiles and more (C = FINISH_CTAS),
-// one CTA for the others (C = 1: no cluster calls at all); `first` and `count` select a range of the fast
-// list, the grid covers count problems of every worker.
+// One thread-block cluster of C = FINISH_CTAS CTAs per (worker, segment) of more than SMALL_MAX_TILES tiles
+// (the shorter ones take topk_resolve_small_kernel instead); `first` and `count` select a range of the
+// fast list, the grid covers count problems of every worker.
 //   threshold among the candidates: CTA 0 sorts the short list (the candidates of the threshold's
 //       histogram bin, at most LIST2_CAP) in shared memory, larger key first and lower coordinate first
 //       among equal keys; its first need2 entries are kept, which fixes T and the coordinate cut, and each
@@ -891,7 +893,7 @@ __device__ inline bool fast_kept(uint32_t key, uint32_t coord, uint32_t T, uint3
 // The cluster barriers are the hardware's; every CTA runs to the last one.
 constexpr uint32_t FINISH_CTAS = 8;
 constexpr uint32_t FINISH_PER = 16;                                    // tiles per thread and round of a scan
-constexpr uint32_t FINISH_SOLO_TILES = 4096;                           // segments below this many tiles are served by one CTA
+constexpr uint32_t SMALL_MAX_TILES = 1024;                             // one-pass segments of at most this many tiles are resolved by one CTA each
 __device__ inline uint32_t block_sum(uint32_t v, uint32_t* s_scan) {
     uint32_t total;
     block_exclusive_scan(v, s_scan, &total);
@@ -1074,6 +1076,176 @@ topk_finish_kernel(const __grid_constant__ FastParams P, uint32_t first, uint32_
         if (rank == ranks - 1u && threadIdx.x == 0 && kept_run != seg.k) atomicMin(P.status, ST_DEVICE_CHECK);   // counts and k disagree
     }
     if (!solo) cluster.sync();                                         // a peer's totals must outlive their readers
+}
+
+// ---- resolve of a one-pass segment of few tiles: bin, filter, exact threshold and offsets by ONE CTA ---------
+// For segments of at most SMALL_MAX_TILES tiles (4 M elements) the three steps above cost more in launches and
+// in waiting for memory than in work (the tensors of a network, layer by layer: 42 of ResNet-50's per worker).
+// One CTA per (worker, segment) does them back to back: warp 0 works out the threshold's bin, the lane groups
+// walk the tiles' candidate slices (the short list and the per-tile counts stay in shared memory), the list is
+// sorted, ties are admitted, and the kept counts are summed into the tiles' message offsets.
+__global__ void __launch_bounds__(THREADS)
+topk_resolve_small_kernel(const __grid_constant__ FastParams P, uint32_t first, uint32_t count) {
+    __shared__ unsigned long long srt[LIST2_CAP];
+    __shared__ uint32_t s_kept[SMALL_MAX_TILES];                       // kept candidates per tile
+    __shared__ uint32_t s_scan[WARPS + 1];
+    __shared__ BinInfo s_bi;
+    __shared__ uint32_t s_cnt2;
+    const Layout& L = P.L;
+    const uint32_t lane = threadIdx.x & 31u, sub = threadIdx.x & 7u;
+    uint32_t w, s;
+    const uint32_t prob = fast_problem(L, (blockIdx.x / count) * L.fast_per_worker + first + blockIdx.x % count, w, s);
+    const SegEntry seg = L.segs[s];
+    if (P.state[prob].path != PATH_FAST) return;
+    const uint32_t ntiles = L.segs[s + 1].tile_begin - seg.tile_begin;
+    const size_t item0 = (size_t)w * L.tiles_per_worker + seg.tile_begin;
+    if (threadIdx.x < 32) {
+        const BinInfo bi = resolve_bin(P, prob, true);
+        if (lane == 0) { s_bi = bi; s_cnt2 = 0; }
+    }
+    for (uint32_t t = threadIdx.x; t < ntiles; t += THREADS) s_kept[t] = 0;
+    __syncthreads();
+    const BinInfo bi = s_bi;
+    if (!bi.live) return;                                              // the bracket missed: the fall-back serves the segment
+    FastState st = load_state_l2(P.state + prob);                      // with what warp 0 has just recorded
+    const bool admit = st.need_ties != 0u;
+    const uint32_t mis = misalign_of(P.residuals + (size_t)w * L.n_total + seg.offset);   // tiles lie on the 128-byte grid of the row
+    const uint2* clist = P.cand + (size_t)w * L.cand_per_worker + seg.cand_begin;
+    // ---- filter: candidates above the bin are kept, those inside it go to the short list -----------------------
+    if (bi.need2) {
+        for (uint32_t warp0 = (threadIdx.x >> 5) * 4u * TILES_PER_GROUP; warp0 < ntiles; warp0 += FILTER_TILES_PER_CTA) {
+            const uint32_t t0 = warp0 + ((threadIdx.x >> 3) & 3u) * TILES_PER_GROUP;
+            uint32_t cnt[TILES_PER_GROUP], base[TILES_PER_GROUP];
+#pragma unroll
+            for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+                cnt[u] = 0; base[u] = 0;
+                if (t0 + u < ntiles) { cnt[u] = __ldg(P.tile_ccnt + item0 + t0 + u); base[u] = __ldg(P.tile_cbase + item0 + t0 + u); }
+            }
+#pragma unroll
+            for (uint32_t u = 0; u < TILES_PER_GROUP; ++u) {
+                uint32_t above = 0;
+                for (uint32_t i0 = sub; i0 < cnt[u]; i0 += 32) {           // four entries in flight per lane
+                    uint2 c4[4];
+#pragma unroll
+                    for (uint32_t v = 0; v < 4; ++v) {
+                        const uint32_t i = i0 + 8u * v;
+                        c4[v] = i < cnt[u] ? __ldg(clist + base[u] + i) : make_uint2(0u, 0u);
+                    }
+#pragma unroll
+                    for (uint32_t v = 0; v < 4; ++v) {
+                        if (i0 + 8u * v >= cnt[u]) continue;
+                        const uint2 c = c4[v];
+                        if (c.x > bi.hi2) ++above;
+                        else if (c.x >= bi.lo2) {
+                            const uint32_t pos = atomicAdd(&s_cnt2, 1u);
+                            if (pos < LIST2_CAP) srt[pos] = ((unsigned long long)c.x << 32) | (0xFFFFFFFFu - c.y);
+                        }
+                    }
+                }
+                above += __shfl_xor_sync(0xFFFFFFFFu, above, 1);
+                above += __shfl_xor_sync(0xFFFFFFFFu, above, 2);
+                above += __shfl_xor_sync(0xFFFFFFFFu, above, 4);
+                if (sub == 0u && t0 + u < ntiles) s_kept[t0 + u] = above;
+            }
+        }
+    }
+    __syncthreads();
+    // candidates that did not fit their tile's slice (rare)
+    const uint32_t ncov = min(st.cov_used, seg.cov_cap);
+    const uint2* cover = P.cand + (size_t)w * L.cand_per_worker + seg.cov_begin;
+    if (ncov && (admit || bi.need2)) {
+        for (uint32_t i = threadIdx.x; i < ncov; i += THREADS) {
+            const uint2 c = cover[i];
+            if (admit || c.x > bi.hi2) atomicAdd(&s_kept[(c.y + mis) / TILE], 1u);
+            else if (c.x >= bi.lo2) {
+                const uint32_t pos = atomicAdd(&s_cnt2, 1u);
+                if (pos < LIST2_CAP) srt[pos] = ((unsigned long long)c.x << 32) | (0xFFFFFFFFu - c.y);
+            }
+        }
+        __syncthreads();
+    }
+    // ---- exact threshold from the short list ----------------------------------------------------------------
+    if (bi.need2) {
+        const uint32_t cnt = s_cnt2;
+        if (cnt != st.expect2 || cnt > LIST2_CAP || bi.need2 > cnt) {  // short list disagrees with the histogram
+            if (threadIdx.x == 0) {
+                P.state[prob].path = PATH_FAILED; P.state[prob].fail = FAIL_SHORT_LIST;
+                atomicAdd(P.counters, 1u);
+            }
+            return;
+        }
+        uint32_t size = 1;
+        while (size < cnt) size <<= 1;
+        for (uint32_t i = cnt + threadIdx.x; i < size; i += THREADS) srt[i] = 0;   // padding sorts last
+        __syncthreads();
+        // bitonic sort, descending: larger key first, equal keys: lower coordinate first
+        for (uint32_t k2 = 2; k2 <= size; k2 <<= 1) {
+            for (uint32_t j = k2 >> 1; j > 0; j >>= 1) {
+                for (uint32_t i = threadIdx.x; i < size; i += THREADS) {
+                    const uint32_t ixj = i ^ j;
+                    if (ixj > i) {
+                        const unsigned long long a = srt[i], b = srt[ixj];
+                        const bool desc = (i & k2) == 0;
+                        if (desc ? (a < b) : (a > b)) { srt[i] = b; srt[ixj] = a; }
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        const unsigned long long v = srt[bi.need2 - 1u];
+        if (threadIdx.x == 0) {
+            uint32_t icut = (0xFFFFFFFFu - (uint32_t)v) + 1u;          // coordinates below this are kept among the ties
+            if (icut == 0) icut = 0xFFFFFFFFu;                         // (coordinate 2^32-1 cannot occur: n < 2^32)
+            P.state[prob].T = (uint32_t)(v >> 32); P.state[prob].icut = icut;
+        }
+        for (uint32_t i = threadIdx.x; i < bi.need2; i += THREADS) {
+            const uint32_t coord = 0xFFFFFFFFu - (uint32_t)srt[i];
+            atomicAdd(&s_kept[(coord + mis) / TILE], 1u);
+        }
+        __syncthreads();
+    }
+    // ---- kept count per tile, exclusive sum over the segment's tiles (at most four tiles per thread) --------------
+    constexpr uint32_t PER = SMALL_MAX_TILES / THREADS;
+    const uint32_t t0 = threadIdx.x * PER;
+    uint32_t kept[PER];
+#pragma unroll
+    for (uint32_t i = 0; i < PER; ++i) {
+        kept[i] = 0;
+        if (t0 + i < ntiles) {
+            kept[i] = __ldg(P.tile_sure + item0 + t0 + i) + s_kept[t0 + i];
+            if (admit) kept[i] += __ldg(P.tile_ccnt + item0 + t0 + i);   // every candidate is kept (those of the overflow list are in s_kept)
+        }
+    }
+    if (admit) {                                                       // ties before each tile decide how many it admits
+        uint32_t adm[PER], tsum = 0;
+#pragma unroll
+        for (uint32_t i = 0; i < PER; ++i) {
+            adm[i] = t0 + i < ntiles ? __ldg(P.tile_tie + item0 + t0 + i) : 0u;
+            tsum += adm[i];
+        }
+        uint32_t total;
+        uint32_t before = block_exclusive_scan(tsum, s_scan, &total);
+#pragma unroll
+        for (uint32_t i = 0; i < PER; ++i) {
+            const uint32_t room = st.need_ties > before ? st.need_ties - before : 0u;
+            const uint32_t a = min(adm[i], room);
+            before += adm[i];
+            kept[i] += a;
+            if (t0 + i < ntiles) P.tile_csum[item0 + t0 + i] = a;
+        }
+    }
+    uint32_t sum = 0;
+#pragma unroll
+    for (uint32_t i = 0; i < PER; ++i) sum += kept[i];
+    uint32_t total;
+    uint32_t ex = block_exclusive_scan(sum, s_scan, &total);
+    uint32_t* off = P.offsets + (size_t)w * (L.tiles_per_worker + 1) + seg.tile_begin;
+#pragma unroll
+    for (uint32_t i = 0; i < PER; ++i) {
+        if (t0 + i < ntiles) off[t0 + i] = ex;
+        ex += kept[i];
+    }
+    if (threadIdx.x == 0 && total != seg.k) atomicMin(P.status, ST_DEVICE_CHECK);   // counts and k disagree
 }
 
 // ---- emit: G lanes per tile walk the tile's slice of the flagged list ----------------------------
