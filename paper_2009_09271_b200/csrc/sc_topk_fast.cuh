@@ -3,7 +3,8 @@
 //
 // A radix select has to see every key before it knows the threshold, which costs extra
 // passes over HBM.  Here a small systematic sample of |g + e| brackets the threshold first:
-//   bracket  m keys per (worker, segment) are read from evenly spaced 32-byte sectors; two order
+//   bracket  m keys per (worker, segment) are read from 32-byte sectors, one per stretch of the segment
+//            at a hashed place inside the stretch; two order
 //            statistics of the sample, six standard deviations either side of rank k m / n, give
 //            [lo, hi] with count(key > hi) <= k <= count(key >= lo) except with negligible
 //            probability.  A key value that holds a large share of the sample at the lower order
@@ -178,13 +179,18 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
         const float* e = P.residuals + row;
         const uint32_t a0 = (8u - (uint32_t)((reinterpret_cast<uintptr_t>(e) >> 2) & 7u)) & 7u;   // first 32-byte aligned element
         const uint32_t sectors = (seg.n - a0) / 8u;
+        // one sector out of every `stride`, at a hashed place inside its stretch: evenly spread, but not periodic
+        // (a tensor whose large entries repeat with the stride, a hot column of a matrix, would otherwise be
+        // sampled at its large entries only, or never)
+        const uint32_t stride = max(sectors / S, 1u);
         for (uint32_t c0 = c_begin + threadIdx.x; c0 < c_end; c0 += THREADS * SAMPLE_BATCH) {
             float4 ev[SAMPLE_BATCH][2], gv[SAMPLE_BATCH][2];
 #pragma unroll
             for (int u = 0; u < SAMPLE_BATCH; ++u) {
                 const uint32_t c = c0 + u * THREADS;
                 if (c < c_end) {
-                    const size_t at = (size_t)a0 + (size_t)(((uint64_t)c * sectors) / S) * 8u;
+                    const uint32_t jitter = mix32(c * 0x9E3779B9u + 0x85EBCA6Bu) % stride;
+                    const size_t at = (size_t)a0 + ((size_t)(((uint64_t)c * sectors) / S) + jitter) * 8u;
                     ev[u][0] = *reinterpret_cast<const float4*>(e + at); ev[u][1] = *reinterpret_cast<const float4*>(e + at + 4);
                     gv[u][0] = *reinterpret_cast<const float4*>(g + at); gv[u][1] = *reinterpret_cast<const float4*>(g + at + 4);
                 }

@@ -633,3 +633,38 @@ def test_user_stream_short_and_long_segments_side_by_side(ctx):
             assert_bits_equal(e[w], oe[w], f"residual[w={w}]")
         assert_bits_equal(out, oout, "aggregate")
     assert ctx.sc_sync_status(stream) == 0
+
+
+def _sample_keys(n, k):
+    """Sample size the library takes for a large segment (the same arithmetic as its host code; if that changes,
+    the test below still passes but no longer constructs the periodic case it is meant for)."""
+    q = k / n
+    balance = 1048576.0 * ((n / 350e6) * (max(q, 1e-9) / 0.1) ** 0.5) ** (2.0 / 3.0)
+    capacity = 230400.0 * q * (1.0 - q)
+    m = int(max(balance, capacity))
+    m = min(m, n // 16, 1 << 20)
+    return max(m, 4096) & ~7
+
+
+def test_topk_values_periodic_in_the_sampling_stride(ctx):
+    """Large entries exactly one sampling stride apart (a hot column of a row-major matrix): an evenly spaced
+    sample would hold nothing but large entries, or none.  The sample's sectors sit at hashed places inside their
+    stretches, so the bracket holds and the segment is served in one pass."""
+    found = None
+    for n in range(1 << 21, (1 << 22) + 1, 8):
+        k = n // 64
+        S = _sample_keys(n, k) // 8
+        if (n // 8) % S == 0 and (n // 8) // S >= 4:
+            found = (n, k, (n // 8) // S)
+            break
+    assert found is not None
+    n, k, stride = found
+    g = rand(n, 1800, scale=1e-3).view(1, n)
+    big = rand(n // 8 // stride * 8, 1801, scale=10.0)
+    g.view(-1, 8)[::stride] = big.view(-1, 8)                           # every stride-th sector is large
+    e = torch.zeros(1, n)
+    run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, k)], [0])
+    assert ctx.sc_topk_path_counts() == (0, 1, 0)
+    g2 = g.roll(8 * (stride // 2), dims=1)                              # the same pattern, half a stride on
+    run_step_both(ctx, sc.SC_TOPK, g2, e, [(0, n, k)], [0])
+    assert ctx.sc_topk_path_counts() == (0, 1, 0)
