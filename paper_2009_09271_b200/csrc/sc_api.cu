@@ -388,6 +388,30 @@ int launch_row_scan(uint32_t* data, uint32_t rows, uint32_t len, cudaStream_t st
     return SC_OK;
 }
 
+// Top-k of the short segments of the table: one CTA per (worker, segment) up to TINY_SMALL_MAX elements, a
+// cluster of TINY_CTAS CTAs for the longer ones.
+int launch_short_segments(sc_ctx* c, TinyParams tp, int W, cudaStream_t stream) {
+    Launch l(c, KIND_TINY, stream);
+    if (c->tiny_small) {
+        tp.list = c->d_tiny_list; tp.count = c->tiny_small;
+        const uint32_t grid = persistent_grid(c, c->occ_tiny_small, (uint64_t)W * c->tiny_small);
+        topk_tiny_kernel<1><<<grid, THREADS, TINY_SMALL_MAX * sizeof(float), stream>>>(tp);
+    }
+    if (c->tiny_large) {
+        tp.list = c->d_tiny_list + c->tiny_small; tp.count = c->tiny_large;
+        const uint32_t per = (((c->tiny_large_max_n + TINY_CTAS - 1) / TINY_CTAS) + 3u) & ~3u;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((uint32_t)W * c->tiny_large * TINY_CTAS); cfg.blockDim = dim3(THREADS);
+        cfg.dynamicSmemBytes = (size_t)per * sizeof(float); cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = TINY_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr; cfg.numAttrs = 1;
+        SC_CUDA(cudaLaunchKernelEx(&cfg, topk_tiny_kernel<TINY_CTAS>, tp));
+    }
+    return SC_OK;
+}
+
 int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,
                   const uint64_t* h_seeds, bool shared_seeds, bool mask_ready,
                   float* out_vals, uint32_t* out_idx, cudaStream_t stream) {
@@ -425,26 +449,7 @@ int compress_rows(sc_ctx* c, int scheme, int W, const float* grads, float* resid
                 stream = c->aux_stream;
                 forked = true;
             }
-            {
-            Launch l(c, KIND_TINY, stream);
-            if (c->tiny_small) {
-                tp.list = c->d_tiny_list; tp.count = c->tiny_small;
-                const uint32_t grid = persistent_grid(c, c->occ_tiny_small, (uint64_t)W * c->tiny_small);
-                topk_tiny_kernel<1><<<grid, THREADS, TINY_SMALL_MAX * sizeof(float), stream>>>(tp);
-            }
-            if (c->tiny_large) {
-                tp.list = c->d_tiny_list + c->tiny_small; tp.count = c->tiny_large;
-                const uint32_t per = (((c->tiny_large_max_n + TINY_CTAS - 1) / TINY_CTAS) + 3u) & ~3u;
-                cudaLaunchConfig_t cfg = {};
-                cfg.gridDim = dim3((uint32_t)W * c->tiny_large * TINY_CTAS); cfg.blockDim = dim3(THREADS);
-                cfg.dynamicSmemBytes = (size_t)per * sizeof(float); cfg.stream = stream;
-                cudaLaunchAttribute attr;
-                attr.id = cudaLaunchAttributeClusterDimension;
-                attr.val.clusterDim.x = TINY_CTAS; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-                cfg.attrs = &attr; cfg.numAttrs = 1;
-                SC_CUDA(cudaLaunchKernelEx(&cfg, topk_tiny_kernel<TINY_CTAS>, tp));
-            }
-            }
+            if ((rc_scan = launch_short_segments(c, tp, W, stream)) != SC_OK) return rc_scan;
             if (forked) SC_CUDA(cudaEventRecord(c->ev_join, stream));
             stream = main_stream;
         }
