@@ -31,7 +31,7 @@ UNIT = "elements/s"
 CONTRACT_PEAK_GBS = 8000.0        # the nominal B200 HBM figure the target is stated against
 FALLBACK_PEAK_GBS = 6650.0        # used only if MEASURED_PEAKS.json is absent
 # DRAM bytes per gradient element of the streaming kernels, measured once with ncu on a small case
-NCU_DRAM_BYTES_PER_ELEMENT = {"topk_main": 11.85, "randk_pack": 11.94, "randblock": 11.80}
+NCU_DRAM_BYTES_PER_ELEMENT = {"topk_main": 11.84, "randk_pack": 11.94, "randblock": 11.80}
 
 
 def parse_args():
