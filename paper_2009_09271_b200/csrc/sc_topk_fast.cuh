@@ -1348,8 +1348,12 @@ topk_emit_kernel(FastParams P) {
 // still holds p there) in coordinate order: everything above the tie key is kept, and the first `adm`
 // tie-key elements of the tile, as the finish step decided.
 __device__ inline void emit_tie_tiles(const FastParams& P) {
+    __shared__ float s_stage_v[WARPS][128];                            // per warp: the kept entries of one step, in coordinate order
+    __shared__ uint32_t s_stage_i[WARPS][128];
     const Layout& L = P.L;
     const uint32_t lane = threadIdx.x & 31u;
+    float* stage_v = s_stage_v[threadIdx.x >> 5];
+    uint32_t* stage_i = s_stage_i[threadIdx.x >> 5];
     const uint32_t warps_total = gridDim.x * WARPS;
     const uint32_t warp_g = blockIdx.x * WARPS + (threadIdx.x >> 5);
     for (uint32_t it0 = warp_g; it0 < P.total_items; it0 += warps_total * 32u) {
@@ -1420,20 +1424,27 @@ __device__ inline void emit_tie_tiles(const FastParams& P) {
                         if ((tie >> c) & 1u) { if (trank < adm) keep |= 1u << c; ++trank; }
                     ties_seen += __shfl_sync(0xFFFFFFFFu, tinc, 31);
                     const uint32_t kinc = warp_inclusive_scan(__popc(keep), lane);
-                    uint32_t slot = pos + kinc - __popc(keep);
-                    pos += __shfl_sync(0xFFFFFFFFu, kinc, 31);
+                    uint32_t rank = kinc - __popc(keep);                // among the kept elements of this step (at most 128)
+                    const uint32_t step_kept = __shfl_sync(0xFFFFFFFFu, kinc, 31);
                     if (keep) {
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             if ((keep >> c) & 1u) {
-                                if (slot < seg.k) { ov[slot] = p[c]; oi[slot] = (uint32_t)seg.offset + (uint32_t)(qb + c); }
-                                else atomicMin(P.status, ST_DEVICE_CHECK);
-                                ++slot;
+                                stage_v[rank] = p[c]; stage_i[rank] = (uint32_t)seg.offset + (uint32_t)(qb + c);
+                                ++rank;
                                 p[c] = 0.0f;
                             }
                         }
                         store_quad(er, qb, valid, p);
                     }
+                    __syncwarp();
+                    // the step's kept entries go out together: consecutive lanes, consecutive message slots
+                    for (uint32_t i = lane; i < step_kept; i += 32) {
+                        if (pos + i < seg.k) { ov[pos + i] = stage_v[i]; oi[pos + i] = stage_i[i]; }
+                        else atomicMin(P.status, ST_DEVICE_CHECK);
+                    }
+                    __syncwarp();
+                    pos += step_kept;
                 }
             }
         }
