@@ -124,12 +124,12 @@ __device__ inline bool find_from_top(HistPtr h, uint32_t need, uint32_t* s_tmp /
 
 // ---- bracket: sample the segment, take two order statistics of the sample ---------------------
 // One thread-block cluster of BRACKET_CTAS CTAs per problem (one CTA for small samples).  Every CTA
-// reads its share of the sample: one 32-byte sector (8 elements) of g and e per step and thread, from
-// evenly spaced positions; the keys are kept in global memory for the later rounds (each thread reads
-// back only what it wrote itself).  Round 1 histograms key bits 30..20 in shared memory, CTA 0 adds the
+// reads its share of the sample: one 32-byte sector (8 elements) of g and e per step and thread, one
+// sector per stretch of the segment at a hashed place inside it; the keys are kept in global memory for
+// the later histogram passes (each thread reads back only what it wrote itself).  The first pass histograms key bits 30..20 in shared memory, CTA 0 adds the
 // shares up through distributed shared memory, walks the total and hands the two bins back the same
-// way; round 2 refines them by ten more bits.  If the lower order statistic falls on a key prefix that
-// holds a large share of the sample, round 3 resolves the last ten bits: when ONE key value holds that
+// way; the second pass refines them by ten more bits.  If the lower order statistic falls on a key prefix that
+// holds a large share of the sample, a third pass resolves the last ten bits: when ONE key value holds that
 // share it becomes the tie key (counted, not listed, by the streaming pass).
 // The cluster barriers are the hardware's; no CTA leaves before the last one (a peer's shared memory
 // must stay alive while it is read).  `first` and `count` select a range of the fast list; the grid
@@ -148,7 +148,7 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
     __shared__ uint32_t h0[HIST0_BINS];
     __shared__ uint32_t hA[1024], hB[1024], hC[1024], hM[1024];
     __shared__ uint32_t s_tmp[WARPS + 4];
-    __shared__ uint32_t s_bins[8];                                     // valid in CTA 0: binA, binB, needA, needB, round 3?, prefix B, binM, needM
+    __shared__ uint32_t s_bins[8];                                     // valid in CTA 0: binA, binB, needA, needB, third pass?, prefix B, binM, needM
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t rank = C > 1 ? cluster.block_rank() : 0u;
     const Layout& L = P.L;
@@ -271,8 +271,8 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
         }
     }
     if (C > 1) cluster.sync(); else __syncthreads();
-    const bool round3 = bins0[4] != 0u;                                // the same answer in every CTA of the cluster
-    if (round3) {
+    const bool third_pass = bins0[4] != 0u;                                // the same answer in every CTA of the cluster
+    if (third_pass) {
         const uint32_t prefB = bins0[5];
         for (uint32_t c = c_begin + threadIdx.x; c < c_end; c += THREADS) {
             const uint4 k0 = smp[2 * (size_t)c], k1 = smp[2 * (size_t)c + 1];
@@ -288,7 +288,7 @@ topk_bracket_kernel(FastParams P, uint32_t first, uint32_t count) {
         uint32_t top = okA ? ((prefA << 10) | 1023u) : 0x7FFFFFFFu;
         uint32_t lo = (have_lo && okB) ? (prefB << 10) : 0u;
         uint32_t tie_key = TIE_NONE;
-        if (round3) {
+        if (third_pass) {
             for (uint32_t b = threadIdx.x; b < 1024; b += THREADS) {
                 uint32_t v = hC[b];
                 for (uint32_t r = 1; r < C; ++r) v += cluster.map_shared_rank(hC, r)[b];
