@@ -1354,6 +1354,7 @@ __device__ inline void emit_tie_tiles(const FastParams& P) {
     const uint32_t lane = threadIdx.x & 31u;
     float* stage_v = s_stage_v[threadIdx.x >> 5];
     uint32_t* stage_i = s_stage_i[threadIdx.x >> 5];
+    const uint32_t lt_mask = (1u << lane) - 1u;
     const uint32_t warps_total = gridDim.x * WARPS;
     const uint32_t warp_g = blockIdx.x * WARPS + (threadIdx.x >> 5);
     for (uint32_t it0 = warp_g; it0 < P.total_items; it0 += warps_total * 32u) {
@@ -1416,16 +1417,25 @@ __device__ inline void emit_tie_tiles(const FastParams& P) {
                         above |= (v & (uint32_t)(key > tkey)) << c;
                         tie |= (v & (uint32_t)(key == tkey)) << c;
                     }
-                    const uint32_t tinc = warp_inclusive_scan(__popc(tie), lane);
-                    uint32_t trank = ties_seen + tinc - __popc(tie);    // tie-key elements of the tile before this quad
+                    // ranks by four independent ballots (one per position in the quad) instead of a five-step scan:
+                    // this loop is a chain of dependent steps on one warp, and their latency is what it costs
+                    uint32_t trank = ties_seen, ttotal = 0;             // tie-key elements of the tile before this quad
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t b = __ballot_sync(0xFFFFFFFFu, (tie >> c) & 1u);
+                        trank += __popc(b & lt_mask); ttotal += __popc(b);
+                    }
                     uint32_t keep = above;
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
                         if ((tie >> c) & 1u) { if (trank < adm) keep |= 1u << c; ++trank; }
-                    ties_seen += __shfl_sync(0xFFFFFFFFu, tinc, 31);
-                    const uint32_t kinc = warp_inclusive_scan(__popc(keep), lane);
-                    uint32_t rank = kinc - __popc(keep);                // among the kept elements of this step (at most 128)
-                    const uint32_t step_kept = __shfl_sync(0xFFFFFFFFu, kinc, 31);
+                    ties_seen += ttotal;
+                    uint32_t rank = 0, step_kept = 0;                   // among the kept elements of this step (at most 128)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t b = __ballot_sync(0xFFFFFFFFu, (keep >> c) & 1u);
+                        rank += __popc(b & lt_mask); step_kept += __popc(b);
+                    }
                     if (keep) {
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
