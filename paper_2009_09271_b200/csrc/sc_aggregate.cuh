@@ -35,6 +35,33 @@ agg_bounds_kernel(const uint32_t* __restrict__ idx, uint32_t rows, uint32_t K, u
     bounds[gid] = lo;
 }
 
+// The same bounds when the messages come straight from the one-pass top-k of ONE segment that covers the
+// whole row and lies on the aggregate's tile grid: the per-tile message offsets that step has just left ARE
+// the bounds (kept coordinates before tile t = first slot with a coordinate >= t * tile), so a row is a copy
+// instead of a binary search per tile.  A row whose segment was redone by the fall-back is searched as above.
+__global__ void __launch_bounds__(THREADS)
+agg_bounds_from_offsets_kernel(const uint32_t* __restrict__ idx, uint32_t rows, uint32_t K, uint32_t ntiles, uint32_t tile,
+                               uint32_t* __restrict__ bounds, const uint32_t* __restrict__ offsets, uint32_t off_stride,
+                               const FastState* __restrict__ state) {
+    const uint64_t gid = (uint64_t)blockIdx.x * THREADS + threadIdx.x;
+    const uint64_t per_row = (uint64_t)ntiles + 1;
+    if (gid >= per_row * rows) return;
+    const uint32_t r = (uint32_t)(gid / per_row);
+    const uint32_t t = (uint32_t)(gid - (uint64_t)r * per_row);
+    if (state[r].path == PATH_FAST) {
+        bounds[gid] = t < ntiles ? offsets[(size_t)r * off_stride + (size_t)t * (tile / 4096u)] : K;
+        return;
+    }
+    const uint32_t* row = idx + (size_t)r * K;
+    const uint64_t target = (uint64_t)t * tile;
+    uint32_t lo = 0, hi = K;
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        if ((uint64_t)__ldg(row + mid) < target) lo = mid + 1; else hi = mid;
+    }
+    bounds[gid] = lo;
+}
+
 constexpr uint32_t AGG_STAGE = 1536;     // message entries staged in shared memory per round
 
 // One CTA per tile of ATILE coordinates.  The slices of all W messages that fall into the

@@ -600,8 +600,10 @@ inline uint32_t aggregate_tile(int W, size_t k, size_t n) {
     return per_big_tile <= 0.9 * AGG_STAGE ? ATILE_BIG : ATILE;
 }
 
+// `from_topk`: the messages are those the top-k call on this stream has just written for a table of one segment
+// that covers the row on the aggregate's tile grid; its per-tile offsets then serve as the bounds.
 int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, bool shared_idx, size_t k, size_t n,
-                   float* out, cudaStream_t stream) {
+                   float* out, cudaStream_t stream, bool from_topk = false) {
     if (n == 0) return SC_OK;
     // sparse messages with private coordinates: warp-owned quarter tiles (slices of ~k/n*4096 entries)
     const double slice = (double)k * ATILE / (double)std::max<size_t>(n, 1);       // entries of one worker per 4096-tile
@@ -617,8 +619,12 @@ int aggregate_rows(sc_ctx* c, int W, const float* vals, const uint32_t* idx, boo
     const uint32_t rows = shared_idx ? 1u : (uint32_t)W;
     const uint64_t threads = (uint64_t)rows * (ntiles + 1ull);
     { Launch l(c, KIND_AGG_BOUNDS, stream);
-      agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
-          idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds); }
+      if (from_topk && !shared_idx)
+          agg_bounds_from_offsets_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
+              idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds, c->d_offsets, c->layout.tiles_per_worker + 1u, c->d_fstate);
+      else
+          agg_bounds_kernel<<<(uint32_t)((threads + THREADS - 1) / THREADS), THREADS, 0, stream>>>(
+              idx, rows, (uint32_t)k, ntiles, tile, c->d_bounds); }
     { Launch l(c, by_warp ? KIND_AGG_WARP : fine >= 0 ? KIND_AGG_FINE : KIND_AGG_TILES, stream);
       if (by_warp) {
           const uint64_t nparts = (n + AGG_WARP_PART - 1) / AGG_WARP_PART;
@@ -995,7 +1001,11 @@ int sc_step(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, 
     const bool shared = all_equal(h_seeds, W);
     if ((rc = compress_rows(c, scheme, W, grads, residuals, n, h_seeds, shared, false, out_vals, out_idx, st)) != SC_OK)
         return rc;
-    return aggregate_rows(c, W, out_vals, out_idx, shared && scheme != SC_TOPK, c->layout.K_total, n, out, st);
+    // top-k of one large segment that is the whole row, rows on the 128-byte grid: the tiles of the two steps coincide
+    const bool one_segment = scheme == SC_TOPK && nseg == 1 && segs[0].offset == 0 && segs[0].n == n &&
+                             c->layout.fast_per_worker == 1 && n % 32 == 0 &&
+                             (reinterpret_cast<uintptr_t>(residuals) & 127u) == 0;
+    return aggregate_rows(c, W, out_vals, out_idx, shared && scheme != SC_TOPK, c->layout.K_total, n, out, st, one_segment);
 }
 
 int sc_step_apply(sc_ctx* c, int scheme, int W, const float* grads, float* residuals, size_t n,

@@ -668,3 +668,21 @@ def test_topk_values_periodic_in_the_sampling_stride(ctx):
     g2 = g.roll(8 * (stride // 2), dims=1)                              # the same pattern, half a stride on
     run_step_both(ctx, sc.SC_TOPK, g2, e, [(0, n, k)], [0])
     assert ctx.sc_topk_path_counts() == (0, 1, 0)
+
+
+def test_step_of_one_aligned_segment_takes_its_aggregate_bounds_from_the_topk_offsets(ctx):
+    """A table of one large segment that covers rows on the 128-byte grid: sc_step hands the top-k step's
+    per-tile message offsets to the aggregate instead of searching the messages; a worker whose segment was
+    redone by the fall-back is searched as usual.  Sparse and dense messages (both tile sizes of the aggregate)."""
+    n, W = BIG + 64, 3
+    v = torch.ones(n)
+    perm = torch.randperm(n, generator=torch.Generator().manual_seed(9))
+    c3 = n * 3 // 10
+    v[perm[:c3]] = -3.0
+    v[perm[c3:2 * c3]] = 2.0
+    g = torch.stack([rand(n, 1900), v, rand(n, 1901, scale=1.0)])
+    e = torch.zeros(W, n)
+    for k in (c3 + 5, n // 1000, 1, 0, n // 2):
+        run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, k)], [0] * W)
+    run_step_both(ctx, sc.SC_TOPK, g, e, [(0, n, c3 + 5)], [0] * W)
+    assert ctx.sc_topk_path_counts() == (0, 2, 1)
